@@ -1,0 +1,207 @@
+/* gear.h -- C ABI of the B200-native GEAR hot path (arXiv 2403.05527).
+ *
+ * GEAR keeps a KV cache as  X ~= D^ + L + S :  a b-bit uniformly quantized
+ * backbone D^ (Eq. 2, Eq. 5), a head-wise rank-r matrix L_h = A_h B_h^T fitted
+ * to the quantization residual by power iteration (Eq. 6, Algorithm 2) and a
+ * sparse matrix S of filtered outliers (Eq. 4).  New tokens wait in a small
+ * fp16 streaming buffer and are compressed every n_b steps (Algorithm 1).
+ * Decode attention (Eq. 1) reads the compressed cache directly.
+ *
+ * Conventions
+ *  - Every pointer argument says "device" or "host".  Device buffers are
+ *    borrowed for the duration of the work enqueued on `stream`; the library
+ *    never frees or keeps them.  All tensors are contiguous, row-major.
+ *  - The library owns a gear_cache (one per layer): all of its device memory
+ *    is allocated when the cache is created and released by gear_free.
+ *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return
+ *    without synchronising, except where stated (the *_host variants,
+ *    gear_export, gear_last_device_status).
+ *  - Errors are return codes only; arguments are validated on the host before
+ *    anything is launched; no entry point aborts, throws or traps the device.
+ *  - Not thread-safe per cache: calls on one cache must be issued from one
+ *    thread at a time and on one stream (or streams ordered by the caller).
+ *  - Inputs are assumed finite; NaN / Inf give unspecified results, no error.
+ */
+#ifndef GEAR_H_
+#define GEAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t gear_status;
+enum {
+  GEAR_OK = 0,
+  GEAR_FLUSHED = 1,        /* gear_append_buffer: this push filled the buffer and compressed it */
+  GEAR_ERR_ARG = -1,       /* NULL / out-of-range argument */
+  GEAR_ERR_SHAPE = -2,     /* sizes violate the grouping rules */
+  GEAR_ERR_ALIGN = -3,     /* pointer not 16-byte aligned */
+  GEAR_ERR_CAPACITY = -4,  /* max_tokens / arena exhausted */
+  GEAR_ERR_ALLOC = -5,     /* device allocation failed */
+  GEAR_ERR_CUDA = -6,      /* a CUDA runtime call failed */
+  GEAR_ERR_TIMEOUT = -7,   /* a bounded device-side wait gave up (see gear_last_device_status) */
+  GEAR_ERR_STATE = -8      /* call not valid in the cache's current state */
+};
+
+enum {
+  GEAR_FLAG_KEEP_FP32_FACTORS = 1u  /* also keep A, B in fp32 (before the fp16 rounding) for gear_export */
+};
+
+/* Hyper-parameters in the paper's notation (Section 2 and 3; Algorithm 1, 2). */
+typedef struct gear_config {
+  int32_t batch;        /* sequences in the batch                                              */
+  int32_t n_q_heads;    /* H_q query heads; n_q_heads % n_kv_heads == 0                        */
+  int32_t n_kv_heads;   /* H   key/value heads                                                  */
+  int32_t head_dim;     /* d_H; this build supports 128                                         */
+  int32_t bits;         /* b in {2, 4}                                                           */
+  int32_t group;        /* g in {16, 32, 64, 128}: keys are grouped per channel over
+                           min(g, n_c) consecutive tokens of a segment, values per token over
+                           min(g, d_H) consecutive channels (KIVI grouping, Section 2)          */
+  float   outlier_pct;  /* s in percent, 0 <= s <= 10.  Filter_s (Eq. 4) takes
+                           k = ceil(s * len / 200) largest and k smallest entries of every
+                           group of length len; need k <= 8 and 2k < len                        */
+  int32_t buffer_cap;   /* n_b >= 1, multiple of 16: streaming-buffer capacity in tokens         */
+  int32_t rank_flush;   /* r_g: rank used when a full buffer is compressed, 0..16               */
+  int32_t rank_max;     /* largest rank any gear_compress call will use (sizes the arena), 0..16 */
+  int32_t power_iters;  /* L >= 1 loops of Algorithm 2                                           */
+  int64_t max_tokens;   /* capacity in compressed tokens per sequence (arena is sized from it)   */
+  uint64_t seed;        /* start vectors when the caller passes no B0                           */
+  uint32_t flags;       /* GEAR_FLAG_*                                                           */
+  uint32_t reserved;
+} gear_config;
+
+typedef struct gear_cache gear_cache;   /* opaque */
+
+/* Create an empty cache (no segment, empty buffer) on the current device.
+ * Allocates everything the cache will ever use.  *cache must be NULL. */
+gear_status gear_create(gear_cache** cache, const gear_config* cfg);
+
+/* Algorithm 1, prefill body, applied to a block of n tokens: for X in {K, V}
+ *   S = Filter_s(X) (Eq. 4);  D^ = Quant_b(X - S) (Eq. 5);  R = X - D^ - S;
+ *   per head  A_h B_h^T = SVDSolver_rank(R_h) (Eq. 6, Algorithm 2),
+ * and append the result as one compressed segment.
+ *   cache  in/out: *cache == NULL creates the cache from cfg first (cfg may be NULL otherwise).
+ *   K, V   device fp16 [batch, n_kv_heads, n, head_dim], 16-byte aligned.
+ *   n      segment length; multiple of 16, and of `group` when n >= group.
+ *   rank   r for this segment, 0 <= rank <= min(rank_max, n).
+ *   B0     device fp32 [batch, n_kv_heads, 2 (0 = K, 1 = V), head_dim, rank]: the
+ *          power-iteration start (Algorithm 2's random B), or NULL to draw it
+ *          from cfg.seed.
+ * Must not be called while the streaming buffer holds tokens (GEAR_ERR_STATE). */
+gear_status gear_compress(gear_cache** cache, const gear_config* cfg,
+                          const void* K, const void* V, int64_t n, int32_t rank,
+                          const float* B0, void* stream);
+
+/* Algorithm 1, decoding phase: push (k_t, v_t) into the fp16 buffer; when the
+ * push fills it (n_b tokens) compress the buffer with rank r_g as one more
+ * segment and clear it (returns GEAR_FLUSHED).
+ *   k_new, v_new  device fp16 [batch, n_kv_heads, head_dim].
+ *   B0_flush      device fp32 [batch, n_kv_heads, 2, head_dim, rank_flush] or NULL; only
+ *                 read by the call that flushes. */
+gear_status gear_append_buffer(gear_cache* cache, const void* k_new, const void* v_new,
+                               const float* B0_flush, void* stream);
+
+/* Eq. 1 for one query per sequence over the compressed cache, evaluated as
+ *   scores = q . dequant(codes_K)^T + (q B_K) A_K^T + q . S_K^T   (+ q . K_buffer^T)
+ *   out    = softmax(scores * scale) applied to dequant(codes_V) + A_V B_V^T + S_V (+ V_buffer)
+ * with the low-rank terms taken as down- then up-projection (Section 4,
+ * "Implementation optimization"); fp16 K/V are never materialised.
+ *   q     device fp16 [batch, n_q_heads, head_dim];  query head h reads kv head h / (H_q / H).
+ *   out   device fp32 [batch, n_q_heads, head_dim].
+ *   softmax_scale  <= 0 selects 1 / sqrt(head_dim).
+ * The cache must hold at least one token (GEAR_ERR_STATE otherwise). */
+gear_status gear_decode_attn(gear_cache* cache, const void* q, float* out,
+                             float softmax_scale, void* stream);
+
+/* Release the cache and everything it owns.  NULL is allowed. */
+void gear_free(gear_cache* cache);
+
+/* ---- host-buffer variants (copies inside the call; they synchronise `stream`) ---- */
+
+/* gear_append_buffer with k_new, v_new (and B0_flush) in HOST memory. */
+gear_status gear_append_buffer_host(gear_cache* cache, const void* k_new_host, const void* v_new_host,
+                                    const float* B0_flush_host, void* stream);
+/* gear_decode_attn with q and out in HOST memory. */
+gear_status gear_decode_attn_host(gear_cache* cache, const void* q_host, float* out_host,
+                                  float softmax_scale, void* stream);
+
+/* ---- FP16-cache reference point for the same decode step (Eq. 1 on uncompressed K, V) ---- */
+
+/* out = softmax(q K^T * scale) V over an fp16 cache.
+ *   K, V  device fp16 [batch, n_kv_heads, n_alloc, head_dim] of which the first n tokens are used;
+ *   q     device fp16 [batch, n_q_heads, head_dim];  out device fp32 [batch, n_q_heads, head_dim];
+ *   scratch  device, at least gear_fp16_attn_scratch_bytes(...) bytes, 16-byte aligned. */
+gear_status gear_fp16_decode_attn(const void* K, const void* V, const void* q, float* out,
+                                  int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                  int64_t n, int64_t n_alloc, float softmax_scale,
+                                  void* scratch, size_t scratch_bytes, void* stream);
+size_t gear_fp16_attn_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim);
+
+/* ---- test / accounting helpers (not on the timed path; gear_export synchronises) ---- */
+
+enum {                       /* `what` of gear_export; K_ / V_ select the side                      */
+  GEAR_EXP_K_CODES = 0,      /* u8  [B, H, n_c, d_H]            one code per byte                    */
+  GEAR_EXP_V_CODES = 1,
+  GEAR_EXP_K_SCALE = 2,      /* f16 [B, H, n_c / g_K, d_H]      scale (Delta) of every key group     */
+  GEAR_EXP_V_SCALE = 3,      /* f16 [B, H, n_c, d_H / g_V]                                            */
+  GEAR_EXP_K_ZERO = 4,       /* f16, same shape as the scale: zero-point (group minimum)             */
+  GEAR_EXP_V_ZERO = 5,
+  GEAR_EXP_K_OUT_IDX = 6,    /* u8  [B, H, n_c / g_K, d_H, 2k]  in-group token index, ascending      */
+  GEAR_EXP_V_OUT_IDX = 7,    /* u8  [B, H, n_c, d_H / g_V, 2k]  in-group channel index, ascending    */
+  GEAR_EXP_K_OUT_VAL = 8,    /* f16, same shape as the index: the outlier values, same order         */
+  GEAR_EXP_V_OUT_VAL = 9,
+  GEAR_EXP_K_A = 10,         /* f32 [B, H, n_c, r]   as stored (fp16 rounded)                        */
+  GEAR_EXP_V_A = 11,
+  GEAR_EXP_K_B = 12,         /* f32 [B, H, d_H, r]   as stored (fp16 rounded)                        */
+  GEAR_EXP_V_B = 13,
+  GEAR_EXP_K_A_FP32 = 14,    /* f32, before the fp16 rounding (needs GEAR_FLAG_KEEP_FP32_FACTORS)    */
+  GEAR_EXP_V_A_FP32 = 15,
+  GEAR_EXP_K_B_FP32 = 16,
+  GEAR_EXP_V_B_FP32 = 17,
+  GEAR_EXP_K_BUFFER = 18,    /* f16 [B, H, buffer_len, d_H]  (segment argument ignored)              */
+  GEAR_EXP_V_BUFFER = 19
+};
+
+/* Copy one piece of segment `segment` to HOST memory in the canonical
+ * (unpacked) layout above.  `bytes` must equal the piece's size exactly. */
+gear_status gear_export(gear_cache* cache, int32_t segment, int32_t what,
+                        void* host_dst, size_t bytes);
+
+typedef struct gear_info {
+  int32_t n_segments;
+  int32_t buffer_len;        /* tokens waiting in the fp16 buffer */
+  int64_t n_compressed;      /* tokens in compressed segments     */
+} gear_info;
+gear_status gear_cache_info(const gear_cache* cache, gear_info* info);
+
+typedef struct gear_segment_info {
+  int64_t n_c;               /* tokens in the segment                          */
+  int32_t rank;
+  int32_t g_k, g_v;          /* effective group lengths                        */
+  int32_t k_k, k_v;          /* outliers per side per key / value group        */
+} gear_segment_info;
+gear_status gear_segment_info_get(const gear_cache* cache, int32_t segment, gear_segment_info* info);
+
+/* Bytes the decode kernel reads per call, by component (whole batch, all kv
+ * heads): the denominator of the bandwidth figures.  `stored_*` include the
+ * layout's padding; `alloc_total` is what gear_create allocated. */
+typedef struct gear_bytes {
+  int64_t codes, scale_zero, outliers, lowrank_a, lowrank_b, buffer;
+  int64_t stored_total;      /* bytes of records + B factors + buffer actually read */
+  int64_t alloc_total;
+} gear_bytes;
+gear_status gear_cache_bytes(const gear_cache* cache, gear_bytes* out);
+
+/* Read (and clear) the device status word: 0, or a GEAR_ERR_* a kernel recorded
+ * (a bounded wait that gave up, a range check that failed).  Synchronises. */
+gear_status gear_last_device_status(gear_cache* cache, int32_t* code);
+
+const char* gear_strerror(gear_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GEAR_H_ */

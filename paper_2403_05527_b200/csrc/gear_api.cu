@@ -1,0 +1,525 @@
+// C ABI of the library: cache object, argument checks, launch sequences.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/gear.h"
+#include "gear_internal.cuh"
+
+namespace gear {
+int decode_occupancy(int bits, int G, int warps_per_cta, size_t smem);
+}
+using namespace gear;
+
+struct gear_cache {
+  gear_config cfg;
+  CacheConst cc;
+  int device;
+  int sm_count;
+  int G;                         // query heads per kv head
+  int k_k_full;                  // outliers per side for a key group of length g
+  // device memory
+  unsigned char* arena; size_t arena_bytes; size_t arena_used;
+  float* dbg; size_t dbg_bytes; size_t dbg_used;        // fp32 factor copies (GEAR_FLAG_KEEP_FP32_FACTORS)
+  SegDesc* table_dev; int table_cap;
+  void* buf_k; void* buf_v;                              // [BH][n_b][128] fp16
+  unsigned char* flush_ws; size_t flush_ws_bytes;
+  float* partial; size_t partial_bytes; int max_parts;
+  int* tickets; int* status;
+  void* stage_k; void* stage_v; void* stage_q; float* stage_out; float* stage_b0;   // for the *_host calls
+  // host state
+  std::vector<SegDesc> segs;
+  std::vector<long long> dbgA_off, dbgB_off;             // float offsets into dbg (or -1)
+  int buf_len;
+  long long n_compressed;
+  int n_blocks_c;
+  // cached launch plan of the decode kernel (depends on the segments' shapes)
+  int plan_key, plan_warps, plan_grid, plan_stage, plan_warp_smem, plan_max_T, plan_max_rpad;
+  size_t plan_smem;
+};
+
+static int outlier_count(float s_pct, int len) {
+  const long long s_units = llroundf(s_pct * 10000.0f);
+  return (int)((s_units * len + 1999999LL) / 2000000LL);
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static gear_status check_config(const gear_config* c) {
+  if (!c) return GEAR_ERR_ARG;
+  if (c->batch < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1 || c->max_tokens < 16) return GEAR_ERR_ARG;
+  if (c->n_q_heads % c->n_kv_heads) return GEAR_ERR_SHAPE;
+  if (c->head_dim != kHeadDim) return GEAR_ERR_SHAPE;
+  if (c->bits != 2 && c->bits != 4) return GEAR_ERR_ARG;
+  if (c->group != 16 && c->group != 32 && c->group != 64 && c->group != 128) return GEAR_ERR_ARG;
+  if (!(c->outlier_pct >= 0.f) || c->outlier_pct > 10.f) return GEAR_ERR_ARG;
+  if (c->buffer_cap < 16 || c->buffer_cap % 16 || c->buffer_cap > 1024) return GEAR_ERR_ARG;
+  if (c->buffer_cap > c->group && c->buffer_cap % c->group) return GEAR_ERR_SHAPE;
+  if (c->rank_flush < 0 || c->rank_flush > kMaxRank || c->rank_max < 0 || c->rank_max > kMaxRank) return GEAR_ERR_ARG;
+  if (c->rank_flush > c->rank_max) return GEAR_ERR_ARG;
+  if (c->rank_flush > c->buffer_cap) return GEAR_ERR_SHAPE;
+  if (c->power_iters < 1 || c->power_iters > 64) return GEAR_ERR_ARG;
+  const int gv = c->group < kHeadDim ? c->group : kHeadDim;
+  const int kv = outlier_count(c->outlier_pct, gv);
+  if (kv > kMaxOutliers || (kv > 0 && 2 * kv >= gv)) return GEAR_ERR_SHAPE;
+  const int tf = c->buffer_cap < c->group ? c->buffer_cap : c->group;
+  const int kf = outlier_count(c->outlier_pct, tf);
+  if (kf > kMaxOutliers || (kf > 0 && 2 * kf >= tf)) return GEAR_ERR_SHAPE;
+  return GEAR_OK;
+}
+
+static SegDesc shape_segment(const gear_cache* c, int n_c, int rank) {
+  SegDesc s;
+  memset(&s, 0, sizeof(s));
+  s.n_c = n_c;
+  s.T = n_c < c->cfg.group ? n_c : c->cfg.group;
+  s.rank = rank;
+  s.k_k = outlier_count(c->cfg.outlier_pct, s.T);
+  layout_segment(s, c->cc);
+  return s;
+}
+
+extern "C" void gear_free(gear_cache* c) {
+  if (!c) return;
+  cudaFree(c->arena); cudaFree(c->dbg); cudaFree(c->table_dev); cudaFree(c->buf_k); cudaFree(c->buf_v);
+  cudaFree(c->flush_ws); cudaFree(c->partial); cudaFree(c->tickets); cudaFree(c->status);
+  cudaFree(c->stage_k); cudaFree(c->stage_v); cudaFree(c->stage_q); cudaFree(c->stage_out); cudaFree(c->stage_b0);
+  delete c;
+}
+
+#define GEAR_TRY_ALLOC(ptr, bytes)                                                   \
+  do {                                                                               \
+    if (cudaMalloc((void**)&(ptr), (bytes)) != cudaSuccess) {                        \
+      cudaGetLastError();                                                            \
+      gear_free(c);                                                                  \
+      return GEAR_ERR_ALLOC;                                                         \
+    }                                                                                \
+  } while (0)
+
+extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
+  if (!out || *out) return GEAR_ERR_ARG;
+  gear_status st = check_config(cfg);
+  if (st != GEAR_OK) return st;
+  gear_cache* c = new (std::nothrow) gear_cache();
+  if (!c) return GEAR_ERR_ALLOC;
+  c->cfg = *cfg;
+  c->arena = nullptr; c->dbg = nullptr; c->table_dev = nullptr; c->buf_k = c->buf_v = nullptr; c->flush_ws = nullptr;
+  c->partial = nullptr; c->tickets = nullptr; c->status = nullptr;
+  c->stage_k = c->stage_v = c->stage_q = nullptr; c->stage_out = nullptr; c->stage_b0 = nullptr;
+  c->cc.bits = cfg->bits;
+  c->cc.g_v = cfg->group < kHeadDim ? cfg->group : kHeadDim;
+  c->cc.ngv = kHeadDim / c->cc.g_v;
+  c->cc.k_v = outlier_count(cfg->outlier_pct, c->cc.g_v);
+  c->cc.BH = cfg->batch * cfg->n_kv_heads;
+  c->cc.n_b = cfg->buffer_cap;
+  c->G = cfg->n_q_heads / cfg->n_kv_heads;
+  c->buf_len = 0; c->n_compressed = 0; c->n_blocks_c = 0; c->plan_key = -1;
+  if (cudaGetDevice(&c->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) {
+    delete c;
+    return GEAR_ERR_CUDA;
+  }
+  const size_t BH = c->cc.BH;
+  // arena: worst bytes per token over the two segment shapes the cache can see (full groups at rank_max,
+  // flushed buffers at rank_flush), plus the per-segment B factors
+  const int n_b = cfg->buffer_cap;
+  SegDesc sp = shape_segment(c, cfg->group, cfg->rank_max);
+  SegDesc sf = shape_segment(c, n_b, cfg->rank_flush);
+  const double dens_p = (double)sp.rec_bytes / sp.T, dens_f = (double)sf.rec_bytes / sf.T;
+  const double dens = dens_p > dens_f ? dens_p : dens_f;
+  const size_t n_flush_max = (size_t)(cfg->max_tokens / n_b) + 1;
+  size_t per_bh = (size_t)(dens * (double)cfg->max_tokens) + n_flush_max * sf.bfac_bytes + 8 * (size_t)sp.bfac_bytes +
+                  16 * (size_t)(sp.rec_bytes > sf.rec_bytes ? sp.rec_bytes : sf.rec_bytes);
+  c->arena_bytes = align_up(per_bh, 256) * BH + 4096;
+  c->arena_used = 0;
+  GEAR_TRY_ALLOC(c->arena, c->arena_bytes);
+  c->table_cap = (int)(cfg->max_tokens / 16 + 8);
+  GEAR_TRY_ALLOC(c->table_dev, sizeof(SegDesc) * (size_t)c->table_cap);
+  GEAR_TRY_ALLOC(c->buf_k, BH * n_b * kHeadDim * 2);
+  GEAR_TRY_ALLOC(c->buf_v, BH * n_b * kHeadDim * 2);
+  c->flush_ws_bytes = compress_workspace_bytes((int)BH, n_b, cfg->rank_flush);
+  GEAR_TRY_ALLOC(c->flush_ws, c->flush_ws_bytes);
+  if (cfg->flags & GEAR_FLAG_KEEP_FP32_FACTORS) {
+    const size_t rm = cfg->rank_max > 0 ? cfg->rank_max : 1;
+    c->dbg_bytes = (BH * 2 * (size_t)cfg->max_tokens * rm + BH * 2 * kHeadDim * rm * (size_t)c->table_cap) * 4;
+    c->dbg_used = 0;
+    GEAR_TRY_ALLOC(c->dbg, c->dbg_bytes);
+  }
+  // decode scratch: one partial per (unit, warp touching it); upper bound of warps in a launch
+  const int hp = c->G <= 4 ? 4 : 8;
+  const int passes = (c->G + hp - 1) / hp;
+  const size_t units = BH * passes;
+  const size_t nw_max = (size_t)c->sm_count * 16;
+  c->max_parts = (int)(nw_max / units + 3);
+  c->partial_bytes = units * c->max_parts * (size_t)hp * 130 * 4;
+  GEAR_TRY_ALLOC(c->partial, c->partial_bytes);
+  GEAR_TRY_ALLOC(c->tickets, units * 4);
+  GEAR_TRY_ALLOC(c->status, 4);
+  cudaMemset(c->tickets, 0, units * 4);
+  cudaMemset(c->status, 0, 4);
+  const size_t tok_bytes = BH * kHeadDim * 2;
+  GEAR_TRY_ALLOC(c->stage_k, tok_bytes);
+  GEAR_TRY_ALLOC(c->stage_v, tok_bytes);
+  GEAR_TRY_ALLOC(c->stage_q, (size_t)cfg->batch * cfg->n_q_heads * kHeadDim * 2);
+  GEAR_TRY_ALLOC(c->stage_out, (size_t)cfg->batch * cfg->n_q_heads * kHeadDim * 4);
+  GEAR_TRY_ALLOC(c->stage_b0, BH * 2 * kHeadDim * (size_t)(cfg->rank_flush > 0 ? cfg->rank_flush : 1) * 4);
+  if (cudaDeviceSynchronize() != cudaSuccess) { gear_free(c); return GEAR_ERR_CUDA; }
+  *out = c;
+  return GEAR_OK;
+}
+
+// Append one compressed segment built from K, V [BH][n][128] on the device.
+static gear_status compress_segment(gear_cache* c, const void* K, const void* V, int n, int rank, const float* B0,
+                                    bool is_flush, cudaStream_t st) {
+  if ((int)c->segs.size() >= c->table_cap) return GEAR_ERR_CAPACITY;
+  if (c->n_compressed + n > c->cfg.max_tokens) return GEAR_ERR_CAPACITY;
+  SegDesc sd = shape_segment(c, n, rank);
+  if (sd.k_k > kMaxOutliers || (sd.k_k > 0 && 2 * sd.k_k >= sd.T)) return GEAR_ERR_SHAPE;
+  const size_t need = align_up((size_t)sd.bh_stride, 16) * c->cc.BH;
+  sd.bh_stride = (long long)align_up((size_t)sd.bh_stride, 16);
+  if (c->arena_used + need > c->arena_bytes) return GEAR_ERR_CAPACITY;
+  sd.seg_base = (long long)c->arena_used;
+  sd.tok_start = (int)c->n_compressed;
+  sd.blk_start = c->n_blocks_c;
+  sd.dbg_base = -1;
+  float* dbgA = nullptr; float* dbgB = nullptr;
+  long long offA = -1, offB = -1;
+  if (c->dbg && rank > 0) {
+    const size_t nA = (size_t)c->cc.BH * 2 * n * rank, nB = (size_t)c->cc.BH * 2 * kHeadDim * rank;
+    if ((c->dbg_used + nA + nB) * 4 > c->dbg_bytes) return GEAR_ERR_CAPACITY;
+    offA = (long long)c->dbg_used; offB = offA + (long long)nA;
+    dbgA = c->dbg + offA; dbgB = c->dbg + offB;
+  }
+  CompressJob job;
+  job.seg = sd; job.cc = c->cc; job.arena = c->arena;
+  job.K = (const __half*)K; job.V = (const __half*)V; job.B0 = B0;
+  job.dbgA = dbgA; job.dbgB = dbgB;
+  job.seed = c->cfg.seed; job.segment_index = (int)c->segs.size(); job.iters = c->cfg.power_iters;
+
+  cudaError_t e = cudaSuccess;
+  if (is_flush) {
+    e = compress_range(job, 0, c->cc.BH, c->flush_ws, st);
+  } else {
+    // bounded transient workspace, (batch, head) pairs processed in ranges
+    const size_t per_bh = compress_workspace_bytes(1, n, rank);
+    const size_t budget = (size_t)3 << 30;
+    int chunk = (int)(budget / per_bh);
+    if (chunk < 1) chunk = 1;
+    if (chunk > c->cc.BH) chunk = c->cc.BH;
+    unsigned char* ws = nullptr;
+    const size_t ws_bytes = compress_workspace_bytes(chunk, n, rank);
+    if (cudaMallocAsync((void**)&ws, ws_bytes, st) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_ALLOC; }
+    for (int bh0 = 0; bh0 < c->cc.BH && e == cudaSuccess; bh0 += chunk) {
+      const int nbh = bh0 + chunk <= c->cc.BH ? chunk : c->cc.BH - bh0;
+      e = compress_range(job, bh0, nbh, ws, st);
+    }
+    cudaFreeAsync(ws, st);
+  }
+  if (e != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
+  e = launch_write_desc(c->table_dev, (int)c->segs.size(), sd, st);
+  if (e != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
+  c->segs.push_back(sd);
+  c->dbgA_off.push_back(offA); c->dbgB_off.push_back(offB);
+  if (offA >= 0) c->dbg_used += (size_t)c->cc.BH * 2 * n * rank + (size_t)c->cc.BH * 2 * kHeadDim * rank;
+  c->arena_used += need;
+  c->n_compressed += n;
+  c->n_blocks_c += sd.nblk;
+  c->plan_key = -1;
+  return GEAR_OK;
+}
+
+extern "C" gear_status gear_compress(gear_cache** cache, const gear_config* cfg, const void* K, const void* V,
+                                     int64_t n, int32_t rank, const float* B0, void* stream) {
+  if (!cache || !K || !V) return GEAR_ERR_ARG;
+  if (((uintptr_t)K | (uintptr_t)V) & 15) return GEAR_ERR_ALIGN;
+  const gear_config* use = *cache ? &(*cache)->cfg : cfg;
+  if (!use) return GEAR_ERR_ARG;
+  gear_status st = check_config(use);
+  if (st != GEAR_OK) return st;
+  if (n < 16 || n % 16 || n > (1 << 30)) return GEAR_ERR_SHAPE;
+  if (n >= use->group && n % use->group) return GEAR_ERR_SHAPE;
+  if (rank < 0 || rank > use->rank_max || rank > n) return GEAR_ERR_ARG;
+  bool created = false;
+  if (!*cache) {
+    st = gear_create(cache, cfg);
+    if (st != GEAR_OK) return st;
+    created = true;
+  }
+  gear_cache* c = *cache;
+  if (c->buf_len != 0) return GEAR_ERR_STATE;
+  st = compress_segment(c, K, V, (int)n, rank, B0, false, (cudaStream_t)stream);
+  if (st != GEAR_OK && created) { gear_free(c); *cache = nullptr; }
+  return st;
+}
+
+extern "C" gear_status gear_append_buffer(gear_cache* c, const void* k_new, const void* v_new, const float* B0_flush,
+                                          void* stream) {
+  if (!c || !k_new || !v_new) return GEAR_ERR_ARG;
+  if (((uintptr_t)k_new | (uintptr_t)v_new) & 15) return GEAR_ERR_ALIGN;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int n_b = c->cfg.buffer_cap;
+  if (c->buf_len + 1 == n_b) {     // this push will flush: make sure the segment fits before touching anything
+    if (c->n_compressed + n_b > c->cfg.max_tokens || (int)c->segs.size() >= c->table_cap) return GEAR_ERR_CAPACITY;
+  }
+  if (launch_append(c->buf_k, c->buf_v, k_new, v_new, c->cc.BH, n_b, c->buf_len, st) != cudaSuccess) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  c->buf_len += 1;
+  c->plan_key = -1;
+  if (c->buf_len < n_b) return GEAR_OK;
+  gear_status s = compress_segment(c, c->buf_k, c->buf_v, n_b, c->cfg.rank_flush, B0_flush, true, st);
+  if (s != GEAR_OK) { c->buf_len -= 1; return s; }
+  c->buf_len = 0;
+  return GEAR_FLUSHED;
+}
+
+static gear_status plan_decode(gear_cache* c) {
+  const int key = (int)c->segs.size() * 4096 + c->buf_len;
+  if (c->plan_key == key) return GEAR_OK;
+  int max_rec = 0, max_bfac = 0, max_T = 16, max_rpad = 0;
+  for (const SegDesc& s : c->segs) {
+    if (s.rec_bytes > max_rec) max_rec = s.rec_bytes;
+    if (s.bfac_bytes > max_bfac) max_bfac = s.bfac_bytes;
+    if (s.T > max_T) max_T = s.T;
+    if (s.r_pad > max_rpad) max_rpad = s.r_pad;
+  }
+  const int hp = c->G <= 4 ? 4 : 8;
+  int stage = 0, wsm = 0;
+  decode_smem_plan(c->cc.bits, max_rec, max_bfac, max_T, max_rpad, hp, &stage, &wsm);
+  int warps = 4;
+  while (warps > 1 && (size_t)warps * wsm > 220 * 1024) warps >>= 1;
+  const size_t smem = (size_t)warps * wsm;
+  if (smem > 227 * 1024) return GEAR_ERR_SHAPE;
+  int occ = decode_occupancy(c->cc.bits, c->G, warps, smem);
+  if (occ < 1) return GEAR_ERR_CUDA;
+  if (occ * warps > 16) occ = 16 / warps;
+  c->plan_warps = warps; c->plan_grid = c->sm_count * occ; c->plan_stage = stage; c->plan_warp_smem = wsm;
+  c->plan_max_T = max_T; c->plan_max_rpad = max_rpad; c->plan_smem = smem;
+  c->plan_key = key;
+  return GEAR_OK;
+}
+
+extern "C" gear_status gear_decode_attn(gear_cache* c, const void* q, float* out, float softmax_scale, void* stream) {
+  if (!c || !q || !out) return GEAR_ERR_ARG;
+  if (((uintptr_t)q | (uintptr_t)out) & 15) return GEAR_ERR_ALIGN;
+  if (c->n_compressed == 0 && c->buf_len == 0) return GEAR_ERR_STATE;
+  gear_status s = plan_decode(c);
+  if (s != GEAR_OK) return s;
+  DecodeArgs a;
+  a.arena = c->arena; a.table = c->table_dev;
+  a.buf_k = (const __half*)c->buf_k; a.buf_v = (const __half*)c->buf_v;
+  a.q = (const __half*)q; a.out = out; a.partial = c->partial; a.tickets = c->tickets; a.status = c->status;
+  a.cc = c->cc; a.nseg = (int)c->segs.size(); a.n_blocks_c = c->n_blocks_c; a.buf_len = c->buf_len;
+  a.n_kv_heads = c->cfg.n_kv_heads; a.group_heads = c->G; a.max_parts = c->max_parts;
+  a.stage_bytes = c->plan_stage; a.warp_smem = c->plan_warp_smem; a.max_T = c->plan_max_T; a.max_rpad = c->plan_max_rpad;
+  const float sc = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)kHeadDim);
+  a.scale_log2 = sc * 1.4426950408889634f;
+  if (launch_decode(a, c->plan_warps, c->plan_grid, c->plan_smem, (cudaStream_t)stream) != cudaSuccess) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  return GEAR_OK;
+}
+
+extern "C" gear_status gear_append_buffer_host(gear_cache* c, const void* k_host, const void* v_host,
+                                               const float* B0_host, void* stream) {
+  if (!c || !k_host || !v_host) return GEAR_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t tok_bytes = (size_t)c->cc.BH * kHeadDim * 2;
+  if (cudaMemcpyAsync(c->stage_k, k_host, tok_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(c->stage_v, v_host, tok_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  const float* b0 = nullptr;
+  if (B0_host && c->cfg.rank_flush > 0 && c->buf_len + 1 == c->cfg.buffer_cap) {
+    if (cudaMemcpyAsync(c->stage_b0, B0_host, (size_t)c->cc.BH * 2 * kHeadDim * c->cfg.rank_flush * 4,
+                        cudaMemcpyHostToDevice, st) != cudaSuccess) {
+      cudaGetLastError();
+      return GEAR_ERR_CUDA;
+    }
+    b0 = c->stage_b0;
+  }
+  gear_status s = gear_append_buffer(c, c->stage_k, c->stage_v, b0, stream);
+  if (s < 0) return s;
+  if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
+  return s;
+}
+
+extern "C" gear_status gear_decode_attn_host(gear_cache* c, const void* q_host, float* out_host, float softmax_scale,
+                                             void* stream) {
+  if (!c || !q_host || !out_host) return GEAR_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t nq = (size_t)c->cfg.batch * c->cfg.n_q_heads * kHeadDim;
+  if (cudaMemcpyAsync(c->stage_q, q_host, nq * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  gear_status s = gear_decode_attn(c, c->stage_q, c->stage_out, softmax_scale, stream);
+  if (s != GEAR_OK) return s;
+  if (cudaMemcpyAsync(out_host, c->stage_out, nq * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  return GEAR_OK;
+}
+
+extern "C" gear_status gear_fp16_decode_attn(const void* K, const void* V, const void* q, float* out, int32_t batch,
+                                             int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int64_t n,
+                                             int64_t n_alloc, float softmax_scale, void* scratch, size_t scratch_bytes,
+                                             void* stream) {
+  if (!K || !V || !q || !out || !scratch) return GEAR_ERR_ARG;
+  if (batch < 1 || n_kv_heads < 1 || n_q_heads < 1 || n < 1 || n_alloc < n) return GEAR_ERR_ARG;
+  if (head_dim != kHeadDim || n_q_heads % n_kv_heads) return GEAR_ERR_SHAPE;
+  if (((uintptr_t)K | (uintptr_t)V | (uintptr_t)q | (uintptr_t)out | (uintptr_t)scratch) & 15) return GEAR_ERR_ALIGN;
+  if (scratch_bytes < gear_fp16_attn_scratch_bytes(batch, n_q_heads, head_dim)) return GEAR_ERR_CAPACITY;
+  const float sc = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)kHeadDim);
+  if (launch_fp16_attn(K, V, q, out, batch, n_q_heads, n_kv_heads, n, n_alloc, sc, scratch, scratch_bytes,
+                       (cudaStream_t)stream) != cudaSuccess) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  return GEAR_OK;
+}
+
+extern "C" size_t gear_fp16_attn_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim) {
+  (void)head_dim;
+  return fp16_attn_scratch(batch, n_q_heads);
+}
+
+// ------------------------------------------------------------------ helpers
+static size_t export_elems(const gear_cache* c, const SegDesc& s, int what, size_t* elem_bytes) {
+  const size_t BH = c->cc.BH, d = kHeadDim;
+  switch (what) {
+    case GEAR_EXP_K_CODES: case GEAR_EXP_V_CODES: *elem_bytes = 1; return BH * s.n_c * d;
+    case GEAR_EXP_K_SCALE: case GEAR_EXP_K_ZERO: *elem_bytes = 2; return BH * s.nblk * d;
+    case GEAR_EXP_V_SCALE: case GEAR_EXP_V_ZERO: *elem_bytes = 2; return BH * s.n_c * c->cc.ngv;
+    case GEAR_EXP_K_OUT_IDX: *elem_bytes = 1; return BH * s.nblk * d * 2 * s.k_k;
+    case GEAR_EXP_K_OUT_VAL: *elem_bytes = 2; return BH * s.nblk * d * 2 * s.k_k;
+    case GEAR_EXP_V_OUT_IDX: *elem_bytes = 1; return BH * s.n_c * c->cc.ngv * 2 * c->cc.k_v;
+    case GEAR_EXP_V_OUT_VAL: *elem_bytes = 2; return BH * s.n_c * c->cc.ngv * 2 * c->cc.k_v;
+    case GEAR_EXP_K_A: case GEAR_EXP_V_A: case GEAR_EXP_K_A_FP32: case GEAR_EXP_V_A_FP32:
+      *elem_bytes = 4; return BH * s.n_c * s.rank;
+    case GEAR_EXP_K_B: case GEAR_EXP_V_B: case GEAR_EXP_K_B_FP32: case GEAR_EXP_V_B_FP32:
+      *elem_bytes = 4; return BH * d * s.rank;
+    default: *elem_bytes = 0; return 0;
+  }
+}
+
+extern "C" gear_status gear_export(gear_cache* c, int32_t segment, int32_t what, void* host_dst, size_t bytes) {
+  if (!c || (!host_dst && bytes)) return GEAR_ERR_ARG;
+  if (what == GEAR_EXP_K_BUFFER || what == GEAR_EXP_V_BUFFER) {
+    const size_t row = (size_t)c->buf_len * kHeadDim * 2;
+    if (bytes != row * c->cc.BH) return GEAR_ERR_ARG;
+    if (row == 0) return GEAR_OK;
+    const void* src = what == GEAR_EXP_K_BUFFER ? c->buf_k : c->buf_v;
+    if (cudaDeviceSynchronize() != cudaSuccess ||
+        cudaMemcpy2D(host_dst, row, src, (size_t)c->cfg.buffer_cap * kHeadDim * 2, row, c->cc.BH,
+                     cudaMemcpyDeviceToHost) != cudaSuccess) {
+      cudaGetLastError();
+      return GEAR_ERR_CUDA;
+    }
+    return GEAR_OK;
+  }
+  if (segment < 0 || segment >= (int)c->segs.size()) return GEAR_ERR_ARG;
+  const SegDesc& s = c->segs[segment];
+  size_t eb = 0;
+  const size_t n = export_elems(c, s, what, &eb);
+  if (eb == 0) return GEAR_ERR_ARG;
+  if (bytes != n * eb) return GEAR_ERR_ARG;
+  if (n == 0) return GEAR_OK;
+  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
+  if (what >= GEAR_EXP_K_A_FP32 && what <= GEAR_EXP_V_B_FP32) {
+    if (!c->dbg || c->dbgA_off[segment] < 0) return GEAR_ERR_STATE;
+    // stored as [BH][2][rows][rank]; gather the side
+    const int side = what & 1;
+    const bool isA = what == GEAR_EXP_K_A_FP32 || what == GEAR_EXP_V_A_FP32;
+    const size_t rows = isA ? (size_t)s.n_c : (size_t)kHeadDim;
+    const float* base = c->dbg + (isA ? c->dbgA_off[segment] : c->dbgB_off[segment]);
+    const size_t tile = rows * s.rank * 4;
+    if (cudaMemcpy2D(host_dst, tile, base + (size_t)side * rows * s.rank, 2 * tile, tile, c->cc.BH,
+                     cudaMemcpyDeviceToHost) != cudaSuccess) {
+      cudaGetLastError();
+      return GEAR_ERR_CUDA;
+    }
+    return GEAR_OK;
+  }
+  void* tmp = nullptr;
+  if (cudaMalloc(&tmp, bytes) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_ALLOC; }
+  gear_status r = GEAR_OK;
+  if (launch_export(c->arena, s, c->cc, what, tmp, n, 0) != cudaSuccess ||
+      cudaMemcpy(host_dst, tmp, bytes, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    r = GEAR_ERR_CUDA;
+  }
+  cudaFree(tmp);
+  return r;
+}
+
+extern "C" gear_status gear_cache_info(const gear_cache* c, gear_info* info) {
+  if (!c || !info) return GEAR_ERR_ARG;
+  info->n_segments = (int)c->segs.size();
+  info->buffer_len = c->buf_len;
+  info->n_compressed = c->n_compressed;
+  return GEAR_OK;
+}
+
+extern "C" gear_status gear_segment_info_get(const gear_cache* c, int32_t segment, gear_segment_info* info) {
+  if (!c || !info || segment < 0 || segment >= (int)c->segs.size()) return GEAR_ERR_ARG;
+  const SegDesc& s = c->segs[segment];
+  info->n_c = s.n_c; info->rank = s.rank; info->g_k = s.T; info->g_v = c->cc.g_v; info->k_k = s.k_k; info->k_v = c->cc.k_v;
+  return GEAR_OK;
+}
+
+extern "C" gear_status gear_cache_bytes(const gear_cache* c, gear_bytes* out) {
+  if (!c || !out) return GEAR_ERR_ARG;
+  memset(out, 0, sizeof(*out));
+  const long long BH = c->cc.BH, d = kHeadDim;
+  for (const SegDesc& s : c->segs) {
+    out->codes += BH * 2 * (long long)s.n_c * d * c->cc.bits / 8;
+    out->scale_zero += BH * ((long long)s.nblk * d * 4 + (long long)s.n_c * c->cc.ngv * 4);
+    out->outliers += BH * ((long long)s.nblk * d * 2 * s.k_k * 3 + (long long)s.n_c * c->cc.ngv * 2 * c->cc.k_v * 3);
+    out->lowrank_a += BH * 2 * (long long)s.n_c * s.rank * 2;
+    out->lowrank_b += BH * 2 * d * s.rank * 2;
+    out->stored_total += BH * s.bh_stride;
+  }
+  out->buffer = BH * 2 * (long long)c->buf_len * d * 2;
+  out->stored_total += out->buffer;
+  out->alloc_total = (long long)(c->arena_bytes + c->dbg_bytes + c->flush_ws_bytes + c->partial_bytes +
+                                 2 * (size_t)BH * c->cfg.buffer_cap * d * 2 + sizeof(SegDesc) * (size_t)c->table_cap);
+  return GEAR_OK;
+}
+
+extern "C" gear_status gear_last_device_status(gear_cache* c, int32_t* code) {
+  if (!c || !code) return GEAR_ERR_ARG;
+  int v = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess || cudaMemcpy(&v, c->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemset(c->status, 0, 4) != cudaSuccess) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  *code = v;
+  return GEAR_OK;
+}
+
+extern "C" const char* gear_strerror(gear_status s) {
+  switch (s) {
+    case GEAR_OK: return "ok";
+    case GEAR_FLUSHED: return "buffer flushed";
+    case GEAR_ERR_ARG: return "invalid argument";
+    case GEAR_ERR_SHAPE: return "sizes violate the grouping rules";
+    case GEAR_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case GEAR_ERR_CAPACITY: return "capacity exhausted";
+    case GEAR_ERR_ALLOC: return "device allocation failed";
+    case GEAR_ERR_CUDA: return "CUDA runtime error";
+    case GEAR_ERR_TIMEOUT: return "bounded device-side wait gave up";
+    case GEAR_ERR_STATE: return "call not valid in the cache's current state";
+    default: return "unknown status";
+  }
+}

@@ -1,0 +1,671 @@
+// GEAR compression of one segment (Algorithm 1, prefill body / buffer flush):
+//   quant_pack_kernel : Filter_s (Eq. 4), Quant_b(X - S) (Eq. 2, Eq. 5), packing, residual R = X - D^ - S
+//   pi_* kernels      : SVDSolver (Algorithm 2) on every head's residual R_h, batch-wise and head-wise
+// All arithmetic that decides a code is a fixed sequence of binary32 operations
+// (round-to-nearest-even, no fused multiply-add, no fast-math).
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+
+#include "gear_internal.cuh"
+
+namespace gear {
+
+// ---------------------------------------------------------------------------
+// Filter + Quant + pack for one block (T tokens x 128 channels) of K or V.
+// ---------------------------------------------------------------------------
+constexpr int kXPitch = 130;   // halves per row of the fp16 tile in shared memory
+constexpr int kRPitch = 129;   // floats per row of the residual tile
+
+struct TopList {
+  float v[kMaxOutliers];
+  int i[kMaxOutliers];
+};
+
+// (value, index) order used by Filter_s: larger value first (smaller for the
+// bottom list), then lower index.
+template <bool TOP>
+__device__ __forceinline__ bool goes_before(float va, int ia, float vb, int ib) {
+  if (ib < 0) return ia >= 0;
+  if (ia < 0) return false;
+  if (TOP ? (va > vb) : (va < vb)) return true;
+  return va == vb && ia < ib;
+}
+
+template <int KMAX, bool TOP>
+__device__ __forceinline__ void list_insert(TopList& l, int k, float v, int idx) {
+#pragma unroll
+  for (int s = 0; s < KMAX; ++s) {
+    if (s < k && goes_before<TOP>(v, idx, l.v[s], l.i[s])) {
+      float tv = l.v[s]; int ti = l.i[s];
+      l.v[s] = v; l.i[s] = idx;
+      v = tv; idx = ti;
+    }
+  }
+}
+
+template <int KMAX>
+__device__ __forceinline__ bool list_has(const TopList& l, int k, int idx) {
+  bool h = false;
+#pragma unroll
+  for (int s = 0; s < KMAX; ++s) h |= (s < k && l.i[s] == idx);
+  return h;
+}
+
+struct GroupResult {
+  __half scale, zero;
+  float dmax;   // max |x - zero| over the group's outliers
+};
+
+// One quantization group of `len` entries reached through x_at(e); writes the
+// code and residual of every entry through put(e, code, resid) and the sorted
+// outlier list (in-group index ascending) through put_out(slot, idx, value).
+template <int BITS, int KMAX, class XAt, class Put, class PutOut>
+__device__ __forceinline__ GroupResult process_group(int len, int k, XAt x_at, Put put, PutOut put_out) {
+  TopList top, bot;
+#pragma unroll
+  for (int s = 0; s < KMAX; ++s) { top.v[s] = 0.f; top.i[s] = -1; bot.v[s] = 0.f; bot.i[s] = -1; }
+  if (k > 0) {
+    for (int e = 0; e < len; ++e) list_insert<KMAX, true>(top, k, x_at(e), e);
+    for (int e = 0; e < len; ++e)
+      if (!list_has<KMAX>(top, k, e)) list_insert<KMAX, false>(bot, k, x_at(e), e);
+  }
+  float mn = INFINITY, mx = -INFINITY;
+  for (int e = 0; e < len; ++e) {
+    if (k > 0 && (list_has<KMAX>(top, k, e) || list_has<KMAX>(bot, k, e))) continue;
+    const float x = x_at(e);
+    mn = fminf(mn, x);
+    mx = fmaxf(mx, x);
+  }
+  // Eq. 2 on the kept entries: binary32, one rounding per operation.
+  const float levels = (float)((1 << BITS) - 1);
+  const float range = __fsub_rn(mx, mn);
+  const float d32 = __fdiv_rn(range, levels);
+  const __half d16 = __float2half_rn(d32);
+  const float d = __half2float(d16);
+  const float inv = d != 0.f ? __fdiv_rn(1.0f, d) : 0.f;
+  for (int e = 0; e < len; ++e) {
+    const float x = x_at(e);
+    const bool out = k > 0 && (list_has<KMAX>(top, k, e) || list_has<KMAX>(bot, k, e));
+    int code = 0;
+    float resid = 0.f;
+    if (!out) {
+      if (d != 0.f) {
+        const float t = __fmul_rn(__fsub_rn(x, mn), inv);
+        code = (int)fminf(fmaxf(rintf(t), 0.f), levels);
+      }
+      resid = x - fmaf((float)code, d, mn);
+    }
+    put(e, code, resid);
+  }
+  GroupResult r;
+  r.scale = d16;
+  r.zero = __float2half_rn(mn);
+  r.dmax = 0.f;
+  if (k > 0) {
+    // merge the two lists by index: rank of each entry among the 2k
+#pragma unroll
+    for (int a = 0; a < 2 * KMAX; ++a) {
+      const bool from_top = a < KMAX;
+      const int s = from_top ? a : a - KMAX;
+      if (s >= k) continue;
+      const int ia = from_top ? top.i[s] : bot.i[s];
+      const float va = from_top ? top.v[s] : bot.v[s];
+      int rank = 0;
+#pragma unroll
+      for (int b = 0; b < KMAX; ++b) {
+        rank += (b < k && top.i[b] < ia);
+        rank += (b < k && bot.i[b] < ia);
+      }
+      put_out(rank, ia, va);
+      r.dmax = fmaxf(r.dmax, fabsf(va - mn));
+    }
+  }
+  return r;
+}
+
+template <int BITS, int KMAX>
+__global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const SegDesc& sd = p.seg;
+  const int T = sd.T;
+  const int side = blockIdx.z, bhl = blockIdx.y, blk = blockIdx.x, tid = threadIdx.x;
+  __half* xs = reinterpret_cast<__half*>(smem_raw);
+  unsigned char* cs = smem_raw + round_up(T * kXPitch * 2, 16);
+  float* rs = reinterpret_cast<float*>(cs + T * kHeadDim);
+  __shared__ unsigned int dmax_bits;
+  if (tid == 0) dmax_bits = 0u;
+
+  const __half* X = (side == 0 ? p.K : p.V) + ((size_t)bhl * sd.n_c + (size_t)blk * T) * kHeadDim;
+  for (int i = tid; i < T * 16; i += 128) {
+    const int row = i >> 4, c = i & 15;
+    const uint4 v = *reinterpret_cast<const uint4*>(X + row * kHeadDim + c * 8);
+    unsigned int* dst = reinterpret_cast<unsigned int*>(xs + row * kXPitch + c * 8);
+    dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+  }
+  __syncthreads();
+
+  unsigned char* rec = p.arena + sd.seg_base + (size_t)(p.bh0 + bhl) * sd.bh_stride + sd.bfac_bytes +
+                       (size_t)blk * sd.rec_bytes;
+  float my_dmax = 0.f;
+  if (side == 0) {
+    // keys: one group per channel over the T tokens of the block (per-channel grouping)
+    const int j = tid;
+    const int k = sd.k_k;
+    __half* oval = reinterpret_cast<__half*>(rec + sd.off_koval) + j * 2 * k;
+    unsigned char* oidx = rec + sd.off_koidx + j * 2 * k;
+    GroupResult g = process_group<BITS, KMAX>(
+        T, k, [&](int e) { return __half2float(xs[e * kXPitch + j]); },
+        [&](int e, int code, float r) { cs[e * kHeadDim + j] = (unsigned char)code; rs[e * kRPitch + j] = r; },
+        [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
+    reinterpret_cast<__half2*>(rec + sd.off_kscale)[j] = __halves2half2(g.scale, g.zero);
+    my_dmax = g.dmax;
+  } else {
+    // values: one group per token over g_V consecutive channels (per-token grouping)
+    const int k = p.cc.k_v, gv = p.cc.g_v, ngv = p.cc.ngv;
+    for (int gi = tid; gi < T * ngv; gi += 128) {
+      const int tok = gi / ngv, c = gi % ngv;
+      __half* oval = reinterpret_cast<__half*>(rec + sd.off_voval) + gi * 2 * k;
+      unsigned char* oidx = rec + sd.off_voidx + gi * 2 * k;
+      GroupResult g = process_group<BITS, KMAX>(
+          gv, k, [&](int e) { return __half2float(xs[tok * kXPitch + c * gv + e]); },
+          [&](int e, int code, float r) {
+            cs[tok * kHeadDim + c * gv + e] = (unsigned char)code;
+            rs[tok * kRPitch + c * gv + e] = r;
+          },
+          [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
+      reinterpret_cast<__half2*>(rec + sd.off_vscale)[gi] = __halves2half2(g.scale, g.zero);
+      my_dmax = fmaxf(my_dmax, g.dmax);
+    }
+  }
+  atomicMax(&dmax_bits, __float_as_uint(my_dmax));   // non-negative floats order like their bit patterns
+  __syncthreads();
+  if (tid == 0) reinterpret_cast<float*>(rec)[side] = __uint_as_float(dmax_bits);
+
+  // pack the codes into mma-fragment order
+  const int nq = words_per_lane(BITS), hpw = regs_per_word(BITS);
+  const int words_per_slab = 32 * nq;
+  unsigned int* dst = reinterpret_cast<unsigned int*>(rec + (side == 0 ? sd.off_kcodes : sd.off_vcodes));
+  for (int li = tid; li < (T / kSlab) * words_per_slab; li += 128) {
+    const int slab = li / words_per_slab, wl = li % words_per_slab;
+    const int plane = wl >> 7, lane = (wl & 127) >> 2, q = plane * 4 + (wl & 3);
+    unsigned int word = 0;
+    for (int u = 0; u < hpw; ++u)
+      for (int e = 0; e < 2; ++e) {
+        int tok, ch;
+        if (side == 0) code_coord_k(BITS, lane, q, u, e, tok, ch); else code_coord_v(BITS, lane, q, u, e, tok, ch);
+        word |= (unsigned int)cs[(slab * kSlab + tok) * kHeadDim + ch] << (16 * e + BITS * u);
+      }
+    dst[slab * (sd.slab_codes / 4) + wl] = word;
+  }
+  // residual tile -> workspace (only needed when a low-rank part is fitted)
+  if (p.R != nullptr) {
+    float* R = p.R + (((size_t)bhl * 2 + side) * sd.n_c + (size_t)blk * T) * kHeadDim;
+    for (int i = tid; i < T * kHeadDim; i += 128) R[i] = rs[(i >> 7) * kRPitch + (i & 127)];
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Power iteration (Algorithm 2).  A "tile" is one (batch, head, K|V) residual
+// R_h [n_c, 128] in the workspace.  Factor buffers are [128][16] fp32, zero
+// beyond the rank.
+// ---------------------------------------------------------------------------
+constexpr int kChunkRows = 512;
+constexpr int kPassWarps = 8;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Counter-based Gaussian for library-drawn start vectors (splitmix64 + Box-Muller).
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+__global__ void pi_init_kernel(PiArgs p, const float* B0, int bh0, int BH_total_rank_stride,
+                               unsigned long long seed, int segment) {
+  // one thread per (tile, channel, rho); B0 layout [bh][2][128][rank]
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  const int total = p.ntiles * kHeadDim * kMaxRank;
+  if (idx >= total) return;
+  const int rho = idx % kMaxRank, ch = (idx / kMaxRank) % kHeadDim, tile = idx / (kMaxRank * kHeadDim);
+  float v = 0.f;
+  if (rho < p.rank) {
+    const size_t gtile = (size_t)bh0 * 2 + tile;
+    if (B0 != nullptr) {
+      v = B0[(gtile * kHeadDim + ch) * p.rank + rho];
+    } else {
+      const unsigned long long h = mix64(seed ^ mix64(((unsigned long long)segment << 40) ^ (gtile * 4096ull + ch * 16 + rho)));
+      const float u1 = ((float)(unsigned int)(h >> 40) + 1.0f) * (1.0f / 16777217.0f);
+      const float u2 = (float)(unsigned int)((h >> 8) & 0xFFFFFFu) * (1.0f / 16777216.0f);
+      v = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
+    }
+  }
+  p.Bcur[idx] = v;
+  (void)BH_total_rank_stride;
+}
+
+// mode 0: a = R b ; partial of R^T a                         (loops before the last)
+// mode 1: a = R b -> A0 ; partial Gram a^T a                  (last loop, first product)
+// mode 2: a = A0 W (W = R1^-1 R2^-1) -> stored A ; partial of R^T a   (last loop, second product)
+template <int RP, int MODE>
+__global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
+  __shared__ float red[kHeadDim * RP];            // cross-warp sum, accumulated warp by warp
+  __shared__ float arow[kPassWarps][kMaxRank];     // mode 1: the current row of A, one per warp
+  __shared__ float Wm[kMaxRank * kMaxRank];
+  const int tile = blockIdx.y, chunk = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row0 = chunk * kChunkRows;
+  const int row1 = min(p.n_c, row0 + kChunkRows);
+  const float* R = p.R + (size_t)tile * p.n_c * kHeadDim;
+  float* A0 = p.A0 + (size_t)tile * p.n_c * kMaxRank;
+
+  float b[4][RP];
+  if (MODE != 2) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+      for (int r = 0; r < RP; ++r) b[j][r] = p.Bcur[((size_t)tile * kHeadDim + lane * 4 + j) * kMaxRank + r];
+  } else {
+    for (int i = threadIdx.x; i < kMaxRank * kMaxRank; i += blockDim.x) Wm[i] = p.W[(size_t)tile * 256 + i];
+    __syncthreads();
+  }
+  float acc[4][RP];       // mode 0 / 2: this lane's 4 channels of R^T a
+  float gram[8];          // mode 1: this lane's 8 Gram entries (pairs lane*8 .. lane*8+7 of RP*RP)
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+#pragma unroll
+    for (int r = 0; r < RP; ++r) acc[j][r] = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) gram[i] = 0.f;
+
+  for (int row = row0 + warp; row < row1; row += kPassWarps) {
+    const float4 x4 = *reinterpret_cast<const float4*>(R + (size_t)row * kHeadDim + lane * 4);
+    const float x[4] = {x4.x, x4.y, x4.z, x4.w};
+    float a[RP];
+    if (MODE != 2) {
+#pragma unroll
+      for (int r = 0; r < RP; ++r) {
+        float s = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) s = fmaf(x[j], b[j][r], s);
+        a[r] = warp_sum(s);
+      }
+    } else {
+      float a0[RP];
+#pragma unroll
+      for (int r = 0; r < RP; ++r) a0[r] = A0[(size_t)row * kMaxRank + r];
+#pragma unroll
+      for (int r = 0; r < RP; ++r) {
+        float s = 0.f;
+#pragma unroll
+        for (int q = 0; q < RP; ++q) s = fmaf(a0[q], Wm[q * kMaxRank + r], s);
+        a[r] = s;
+      }
+    }
+    if (MODE == 1) {
+      __syncwarp();
+      if (lane == 0) {
+#pragma unroll
+        for (int r = 0; r < RP; ++r) arow[warp][r] = a[r];
+      }
+      __syncwarp();
+      if (lane < RP) A0[(size_t)row * kMaxRank + lane] = arow[warp][lane];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int pr = lane * 8 + i;
+        if (pr < RP * RP) gram[i] = fmaf(arow[warp][pr / RP], arow[warp][pr % RP], gram[i]);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int r = 0; r < RP; ++r) acc[j][r] = fmaf(x[j], a[r], acc[j][r]);
+      if (MODE == 2) {
+        // store the final A row: fp16 in fragment order inside the record, fp32 copy on request
+        float mine = 0.f;
+#pragma unroll
+        for (int r = 0; r < RP; ++r) if (r == lane) mine = a[r];
+        if (lane < p.seg.r_pad) {
+          const SegDesc& sd = p.seg;
+          const int bhl = tile >> 1, side = tile & 1;
+          const int blk = row / sd.T, tib = row % sd.T, slab = tib / kSlab, ts = tib % kSlab;
+          unsigned char* rec = p.arena + sd.seg_base + (size_t)(p.bh0 + bhl) * sd.bh_stride + sd.bfac_bytes +
+                               (size_t)blk * sd.rec_bytes;
+          const float val = lane < sd.rank ? mine : 0.f;
+          if (side == 0)
+            reinterpret_cast<__half*>(rec + sd.off_ak + slab * sd.slab_a)[ts * sd.r_pad + lane] = __float2half_rn(val);
+          else
+            reinterpret_cast<__half*>(rec + sd.off_av + slab * sd.slab_a)[lane * kSlab + ts] = __float2half_rn(val);
+          if (p.dbgA != nullptr && lane < sd.rank)
+            p.dbgA[(((size_t)(p.bh0 + bhl) * 2 + side) * sd.n_c + row) * sd.rank + lane] = val;
+        }
+      }
+    }
+  }
+  // combine the warps of this block in a fixed order, write the chunk's partial
+  for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x) red[i] = 0.f;
+  __syncthreads();
+  for (int w = 0; w < kPassWarps; ++w) {
+    if (warp == w) {
+      if (MODE == 1) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) red[lane * 8 + i] += gram[i];
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+          for (int r = 0; r < RP; ++r) red[(lane * 4 + j) * RP + r] += acc[j][r];
+      }
+    }
+    __syncthreads();
+  }
+  if (MODE == 1) {
+    for (int i = threadIdx.x; i < RP * RP; i += blockDim.x)
+      p.Gp[((size_t)tile * p.nchunk + chunk) * 256 + (i / RP) * kMaxRank + i % RP] = red[i];
+  } else {
+    for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x)
+      p.Bp[(((size_t)tile * p.nchunk + chunk) * kHeadDim + i / RP) * kMaxRank + i % RP] = red[i];
+  }
+}
+
+// Sum the chunk partials of R^T a into the factor buffer (fixed order).  With
+// `orth`, orthonormalise its columns (modified Gram-Schmidt, two sweeps per
+// column) -- the QR of B at the top of Algorithm 2's last loop.  With `store`,
+// write the final B as fp16 ([r_pad][128] for keys, [128][r_pad] for values).
+__global__ void __launch_bounds__(kHeadDim) pi_reduce_b_kernel(PiArgs p, int orth, int store) {
+  __shared__ float wsum[4];
+  const int tile = blockIdx.x, j = threadIdx.x, lane = j & 31, warp = j >> 5;
+  float b[kMaxRank];
+#pragma unroll
+  for (int r = 0; r < kMaxRank; ++r) {
+    float s = 0.f;
+    if (r < p.rank)
+      for (int c = 0; c < p.nchunk; ++c) s += p.Bp[(((size_t)tile * p.nchunk + c) * kHeadDim + j) * kMaxRank + r];
+    b[r] = s;
+  }
+  auto block_sum = [&](float v) {
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) wsum[warp] = v;
+    __syncthreads();
+    return (wsum[0] + wsum[1]) + (wsum[2] + wsum[3]);
+  };
+  if (orth) {
+#pragma unroll
+    for (int c = 0; c < kMaxRank; ++c) {
+      if (c < p.rank) {                      // uniform over the block
+#pragma unroll
+        for (int sweep = 0; sweep < 2; ++sweep) {
+#pragma unroll
+          for (int q = 0; q < kMaxRank; ++q) {
+            if (q < c) {
+              const float d = block_sum(b[q] * b[c]);
+              b[c] = fmaf(-d, b[q], b[c]);
+            }
+          }
+        }
+        const float nrm2 = block_sum(b[c] * b[c]);
+        b[c] = nrm2 > 0.f ? b[c] * rsqrtf(nrm2) : 0.f;
+        // one Newton step on the normalisation keeps the column norm at 1 to rounding
+        const float n2 = block_sum(b[c] * b[c]);
+        if (n2 > 0.f) b[c] *= (1.5f - 0.5f * n2);
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < kMaxRank; ++r) p.Bcur[((size_t)tile * kHeadDim + j) * kMaxRank + r] = b[r];
+  if (store) {
+    const SegDesc& sd = p.seg;
+    const int bhl = tile >> 1, side = tile & 1;
+    __half* bf = reinterpret_cast<__half*>(p.arena + sd.seg_base + (size_t)(p.bh0 + bhl) * sd.bh_stride);
+#pragma unroll
+    for (int r = 0; r < kMaxRank; ++r) {
+      if (r < sd.r_pad) {
+        const __half v = __float2half_rn(r < sd.rank ? b[r] : 0.f);
+        if (side == 0) bf[r * kHeadDim + j] = v;
+        else bf[sd.r_pad * kHeadDim + j * sd.r_pad + r] = v;
+        if (p.dbgB != nullptr && r < sd.rank)
+          p.dbgB[(((size_t)(p.bh0 + bhl) * 2 + side) * kHeadDim + j) * sd.rank + r] = b[r];
+      }
+    }
+  }
+}
+
+// Gram matrix of the current A (sum of chunk partials), its Cholesky factor
+// U (G = U^T U) and U^-1.  first = 1: W <- U^-1.  first = 0: W <- W U^-1.
+// A column whose pivot vanishes (rank-deficient residual) is zeroed.
+__global__ void __launch_bounds__(32) pi_chol_kernel(PiArgs p, int first) {
+  __shared__ float G[kMaxRank][kMaxRank + 1], U[kMaxRank][kMaxRank + 1], Ui[kMaxRank][kMaxRank + 1],
+      Wo[kMaxRank][kMaxRank + 1];
+  const int tile = blockIdx.x, lane = threadIdx.x, r = p.rank;
+  for (int i = lane; i < 256; i += 32) {
+    float s = 0.f;
+    for (int c = 0; c < p.nchunk; ++c) s += p.Gp[((size_t)tile * p.nchunk + c) * 256 + i];
+    G[i / kMaxRank][i % kMaxRank] = s;
+    U[i / kMaxRank][i % kMaxRank] = 0.f;
+    Ui[i / kMaxRank][i % kMaxRank] = 0.f;
+    Wo[i / kMaxRank][i % kMaxRank] = first ? 0.f : p.W[(size_t)tile * 256 + i];
+  }
+  __syncwarp();
+  if (lane == 0) {
+    float tr = 0.f;
+    for (int i = 0; i < r; ++i) tr += G[i][i];
+    const float tiny = tr * 1e-12f;
+    for (int j = 0; j < r; ++j) {          // upper-triangular U, row by row
+      float d = G[j][j];
+      for (int k = 0; k < j; ++k) d -= U[k][j] * U[k][j];
+      const bool ok = d > tiny && d > 0.f;
+      const float ujj = ok ? sqrtf(d) : 0.f;
+      U[j][j] = ujj;
+      for (int i = j + 1; i < r; ++i) {
+        float s = G[j][i];
+        for (int k = 0; k < j; ++k) s -= U[k][j] * U[k][i];
+        U[j][i] = ok ? s / ujj : 0.f;
+      }
+    }
+    for (int c = 0; c < r; ++c) {          // U^-1 by back substitution, column by column
+      for (int i = c; i >= 0; --i) {
+        if (U[i][i] == 0.f) { Ui[i][c] = 0.f; continue; }
+        float s = (i == c) ? 1.f : 0.f;
+        for (int k = i + 1; k <= c; ++k) s -= U[i][k] * Ui[k][c];
+        Ui[i][c] = s / U[i][i];
+      }
+      if (U[c][c] == 0.f) for (int i = 0; i <= c; ++i) Ui[i][c] = 0.f;
+    }
+  }
+  __syncwarp();
+  for (int i = lane; i < 256; i += 32) {
+    const int a = i / kMaxRank, b = i % kMaxRank;
+    float v = 0.f;
+    if (a < r && b < r) {
+      if (first) v = Ui[a][b];
+      else for (int k = 0; k < r; ++k) v = fmaf(Wo[a][k], Ui[k][b], v);
+    }
+    p.W[(size_t)tile * 256 + i] = v;
+  }
+}
+
+// Gram partials of A0 W (second round of CholeskyQR): one thread per row.
+__global__ void __launch_bounds__(256) pi_gram2_kernel(PiArgs p) {
+  __shared__ float Wm[kMaxRank * kMaxRank];
+  __shared__ float rows[8][32][kMaxRank + 1];
+  __shared__ float red[8][256];
+  const int tile = blockIdx.y, chunk = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int i = threadIdx.x; i < 256; i += blockDim.x) Wm[i] = p.W[(size_t)tile * 256 + i];
+  __syncthreads();
+  const int r = p.rank;
+  const int row0 = chunk * kChunkRows, row1 = min(p.n_c, row0 + kChunkRows);
+  const float* A0 = p.A0 + (size_t)tile * p.n_c * kMaxRank;
+  float g[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) g[i] = 0.f;
+  for (int base = row0 + warp * 32; base < row1; base += 8 * 32) {
+    const int row = base + lane;
+    float a0[kMaxRank];
+#pragma unroll
+    for (int q = 0; q < kMaxRank; ++q) a0[q] = (row < row1 && q < r) ? A0[(size_t)row * kMaxRank + q] : 0.f;
+#pragma unroll
+    for (int c = 0; c < kMaxRank; ++c) {
+      float s = 0.f;
+#pragma unroll
+      for (int q = 0; q < kMaxRank; ++q) s = fmaf(a0[q], Wm[q * kMaxRank + c], s);
+      rows[warp][lane][c] = s;
+    }
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int pr = lane * 8 + i, u = pr / kMaxRank, v = pr % kMaxRank;
+      float s = g[i];
+      for (int t = 0; t < 32; ++t) s = fmaf(rows[warp][t][u], rows[warp][t][v], s);
+      g[i] = s;
+    }
+    __syncwarp();
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) red[warp][lane * 8 + i] = g[i];
+  __syncthreads();
+  for (int i = threadIdx.x; i < 256; i += blockDim.x) {
+    float s = 0.f;
+    for (int w = 0; w < 8; ++w) s += red[w][i];
+    p.Gp[((size_t)tile * p.nchunk + chunk) * 256 + i] = s;
+  }
+}
+
+// Segment with rank 0: nothing to fit, but the A sections of the records do not exist either.
+// Segment descriptor table entry, written by the device so that no host copy is needed.
+__global__ void write_desc_kernel(SegDesc* table, int index, SegDesc d) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) table[index] = d;
+}
+
+__global__ void append_kernel(__half* buf_k, __half* buf_v, const __half* k_new, const __half* v_new,
+                              int BH, int n_b, int slot) {
+  // one 16-byte chunk per thread: BH * 16 chunks per side
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= BH * 16 * 2) return;
+  const int side = i / (BH * 16), r = i % (BH * 16), bh = r >> 4, c = r & 15;
+  const uint4 v = reinterpret_cast<const uint4*>(side == 0 ? k_new : v_new)[bh * 16 + c];
+  reinterpret_cast<uint4*>(side == 0 ? buf_k : buf_v)[((size_t)bh * n_b + slot) * 16 + c] = v;
+}
+
+// ---------------------------------------------------------------------------
+// host side: launch sequence for a range of (batch, head) pairs
+// ---------------------------------------------------------------------------
+template <int BITS>
+static cudaError_t launch_quant(const CompressArgs& a, int nbh, int kmax_needed, cudaStream_t st) {
+  const int T = a.seg.T;
+  const size_t smem = round_up(T * kXPitch * 2, 16) + (size_t)T * kHeadDim + (size_t)T * kRPitch * 4;
+  dim3 grid(a.seg.nblk, nbh, 2);
+#define GEAR_LAUNCH_Q(KM)                                                                                   \
+  {                                                                                                         \
+    cudaError_t e = cudaFuncSetAttribute(quant_pack_kernel<BITS, KM>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                         (int)smem);                                                       \
+    if (e != cudaSuccess) return e;                                                                         \
+    quant_pack_kernel<BITS, KM><<<grid, 128, smem, st>>>(a);                                                \
+  }
+  if (kmax_needed <= 1) GEAR_LAUNCH_Q(1)
+  else if (kmax_needed <= 2) GEAR_LAUNCH_Q(2)
+  else if (kmax_needed <= 4) GEAR_LAUNCH_Q(4)
+  else GEAR_LAUNCH_Q(8)
+#undef GEAR_LAUNCH_Q
+  return cudaGetLastError();
+}
+
+template <int MODE>
+static void launch_pass(const PiArgs& p, cudaStream_t st) {
+  dim3 grid(p.nchunk, p.ntiles);
+  const int rp = p.rank <= 4 ? 4 : (p.rank <= 8 ? 8 : 16);
+  if (rp == 4) pi_pass_kernel<4, MODE><<<grid, kPassWarps * 32, 0, st>>>(p);
+  else if (rp == 8) pi_pass_kernel<8, MODE><<<grid, kPassWarps * 32, 0, st>>>(p);
+  else pi_pass_kernel<16, MODE><<<grid, kPassWarps * 32, 0, st>>>(p);
+}
+
+size_t compress_workspace_bytes(int nbh, int n_c, int rank) {
+  if (rank == 0) return 256;
+  const size_t ntiles = (size_t)nbh * 2;
+  const size_t nchunk = (n_c + kChunkRows - 1) / kChunkRows;
+  size_t b = 0;
+  b += ntiles * n_c * kHeadDim * 4;               // R
+  b += ntiles * kHeadDim * kMaxRank * 4;          // Bcur
+  b += ntiles * nchunk * kHeadDim * kMaxRank * 4; // Bp
+  b += ntiles * n_c * kMaxRank * 4;               // A0
+  b += ntiles * nchunk * 256 * 4;                 // Gp
+  b += ntiles * 256 * 4;                          // W
+  return b + 1024;
+}
+
+cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned char* ws, cudaStream_t st) {
+  const SegDesc& sd = job.seg;
+  const size_t ntiles = (size_t)nbh * 2;
+  const int nchunk = (sd.n_c + kChunkRows - 1) / kChunkRows;
+  float* wsf = reinterpret_cast<float*>(ws);
+  PiArgs pa;
+  pa.seg = sd; pa.arena = job.arena; pa.bh0 = bh0; pa.ntiles = (int)ntiles; pa.n_c = sd.n_c; pa.rank = sd.rank;
+  pa.nchunk = nchunk;
+  pa.R = nullptr; pa.Bcur = nullptr; pa.Bp = nullptr; pa.A0 = nullptr; pa.Gp = nullptr; pa.W = nullptr;
+  pa.dbgA = job.dbgA; pa.dbgB = job.dbgB;
+  if (sd.rank > 0) {
+    pa.R = wsf;       wsf += ntiles * sd.n_c * kHeadDim;
+    pa.Bcur = wsf;    wsf += ntiles * kHeadDim * kMaxRank;
+    pa.Bp = wsf;      wsf += ntiles * nchunk * kHeadDim * kMaxRank;
+    pa.A0 = wsf;      wsf += ntiles * sd.n_c * kMaxRank;
+    pa.Gp = wsf;      wsf += ntiles * nchunk * 256;
+    pa.W = wsf;
+  }
+  CompressArgs ca;
+  ca.seg = sd; ca.cc = job.cc; ca.arena = job.arena; ca.bh0 = bh0;
+  ca.K = job.K + (size_t)bh0 * sd.n_c * kHeadDim;
+  ca.V = job.V + (size_t)bh0 * sd.n_c * kHeadDim;
+  ca.R = pa.R;
+  const int kneed = sd.k_k > job.cc.k_v ? sd.k_k : job.cc.k_v;
+  cudaError_t e = job.cc.bits == 2 ? launch_quant<2>(ca, nbh, kneed, st) : launch_quant<4>(ca, nbh, kneed, st);
+  if (e != cudaSuccess) return e;
+  if (sd.rank == 0) return cudaSuccess;
+
+  const int tot = (int)ntiles * kHeadDim * kMaxRank;
+  const float* b0 = job.B0 ? job.B0 : nullptr;
+  pi_init_kernel<<<(tot + 255) / 256, 256, 0, st>>>(pa, b0, bh0, 0, job.seed, job.segment_index);
+  for (int l = 0; l < job.iters; ++l) {
+    const bool last = l == job.iters - 1;
+    if (!last) {
+      launch_pass<0>(pa, st);                                   // A = R B ; B = R^T A
+      // the loop after this one is the last: its QR of B is folded into the reduction
+      pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(pa, (l + 1 == job.iters - 1) ? 1 : 0, 0);
+    } else {
+      if (job.iters == 1) {                                     // single loop: orthonormalise the start itself
+        PiArgs q = pa; q.nchunk = 0;
+        // Bp unused with zero chunks: re-use the reduce kernel on Bcur through a one-chunk view
+        cudaMemcpyAsync(pa.Bp, pa.Bcur, ntiles * kHeadDim * kMaxRank * 4, cudaMemcpyDeviceToDevice, st);
+        q.nchunk = 1;
+        pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(q, 1, 0);
+      }
+      launch_pass<1>(pa, st);                                   // A = R B, Gram of A
+      pi_chol_kernel<<<(int)ntiles, 32, 0, st>>>(pa, 1);        // A <- Q(A) by CholeskyQR, twice
+      pi_gram2_kernel<<<dim3(nchunk, (int)ntiles), 256, 0, st>>>(pa);
+      pi_chol_kernel<<<(int)ntiles, 32, 0, st>>>(pa, 0);
+      launch_pass<2>(pa, st);                                   // store A ; B = R^T A
+      pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(pa, 0, 1);
+    }
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_write_desc(SegDesc* table, int index, const SegDesc& d, cudaStream_t st) {
+  write_desc_kernel<<<1, 32, 0, st>>>(table, index, d);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_append(void* buf_k, void* buf_v, const void* k_new, const void* v_new, int BH, int n_b, int slot,
+                          cudaStream_t st) {
+  const int n = BH * 16 * 2;
+  append_kernel<<<(n + 255) / 256, 256, 0, st>>>((__half*)buf_k, (__half*)buf_v, (const __half*)k_new,
+                                                 (const __half*)v_new, BH, n_b, slot);
+  return cudaGetLastError();
+}
+
+}  // namespace gear
