@@ -126,7 +126,8 @@ def test_many_small_segments_and_state_errors(pair_factory):
         G.gear_append_buffer(p.cache, tok, tok)
     assert e.value.status == G.GEAR_ERR_CAPACITY
     with pytest.raises(G.GearError) as e:
-        G.gear_decode_attn(p.cache, tok[:, :, 1:], tok.float())      # misaligned query pointer
+        flat = torch.zeros(2 * 128 + 8, dtype=torch.float16, device="cuda")
+        G.gear_decode_attn(p.cache, flat[1:], tok.float())           # misaligned query pointer
     assert e.value.status == G.GEAR_ERR_ALIGN
 
 
