@@ -201,6 +201,9 @@ gear_status gear_last_device_status(gear_cache* cache, int32_t* code);
 
 const char* gear_strerror(gear_status s);
 
+/* Number of kernels this library has launched in this process so far (all caches). */
+uint64_t gear_kernel_launches(void);
+
 #ifdef __cplusplus
 }
 #endif

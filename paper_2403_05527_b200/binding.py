@@ -72,6 +72,7 @@ _SIGNATURES = {
     "gear_cache_bytes": (C.c_int32, [C.c_void_p, C.POINTER(GearBytes)]),
     "gear_last_device_status": (C.c_int32, [C.c_void_p, C.POINTER(C.c_int32)]),
     "gear_strerror": (C.c_char_p, [C.c_int32]),
+    "gear_kernel_launches": (C.c_uint64, []),
 }
 
 
@@ -198,6 +199,10 @@ def gear_last_device_status(cache) -> int:
     code = C.c_int32()
     _check(lib().gear_last_device_status(cache, C.byref(code)), "gear_last_device_status")
     return code.value
+
+
+def gear_kernel_launches() -> int:
+    return int(lib().gear_kernel_launches())
 
 
 def gear_export(cache, segment: int, what: str, batch: int, n_kv_heads: int):

@@ -4,6 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <new>
 #include <vector>
 
@@ -14,6 +15,10 @@ namespace gear {
 int decode_occupancy(int bits, int G, int warps_per_cta, size_t smem);
 }
 using namespace gear;
+
+static std::atomic<unsigned long long> g_launches{0};
+void gear::count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+extern "C" uint64_t gear_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 struct gear_cache {
   gear_config cfg;

@@ -625,7 +625,10 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
   const int kneed = sd.k_k > job.cc.k_v ? sd.k_k : job.cc.k_v;
   cudaError_t e = job.cc.bits == 2 ? launch_quant<2>(ca, nbh, kneed, st) : launch_quant<4>(ca, nbh, kneed, st);
   if (e != cudaSuccess) return e;
+  count_launches(1);
   if (sd.rank == 0) return cudaSuccess;
+  // init + per early loop (pass, reduce) + last loop (pass, chol, gram, chol, pass, reduce)
+  count_launches(1 + 2 * (job.iters - 1) + 6 + (job.iters == 1 ? 1 : 0));
 
   const int tot = (int)ntiles * kHeadDim * kMaxRank;
   const float* b0 = job.B0 ? job.B0 : nullptr;
@@ -657,6 +660,7 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
 
 cudaError_t launch_write_desc(SegDesc* table, int index, const SegDesc& d, cudaStream_t st) {
   write_desc_kernel<<<1, 32, 0, st>>>(table, index, d);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -665,6 +669,7 @@ cudaError_t launch_append(void* buf_k, void* buf_v, const void* k_new, const voi
   const int n = BH * 16 * 2;
   append_kernel<<<(n + 255) / 256, 256, 0, st>>>((__half*)buf_k, (__half*)buf_v, (const __half*)k_new,
                                                  (const __half*)v_new, BH, n_b, slot);
+  count_launches(1);
   return cudaGetLastError();
 }
 

@@ -857,6 +857,7 @@ cudaError_t launch_decode(const DecodeArgs& a, int warps_per_cta, int grid, size
   if (a.cc.bits == 2) { if (G <= 4) GEAR_DEC(2, 1) else GEAR_DEC(2, 2) }
   else { if (G <= 4) GEAR_DEC(4, 1) else GEAR_DEC(4, 2) }
 #undef GEAR_DEC
+  count_launches(1);
   return cudaGetLastError();
 }
 

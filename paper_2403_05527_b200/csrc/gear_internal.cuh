@@ -9,6 +9,9 @@
 
 namespace gear {
 
+// process-wide count of kernels this library launched (read through gear_kernel_launches)
+void count_launches(int n);
+
 struct CompressArgs {
   SegDesc seg;
   CacheConst cc;
