@@ -11,9 +11,6 @@
 #include "../../include/gear.h"
 #include "gear_internal.cuh"
 
-namespace gear {
-int decode_occupancy(int bits, int G, int warps_per_cta, size_t smem);
-}
 using namespace gear;
 
 static std::atomic<unsigned long long> g_launches{0};
@@ -31,6 +28,7 @@ struct gear_cache {
   unsigned char* arena; size_t arena_bytes; size_t arena_used;
   float* dbg; size_t dbg_bytes; size_t dbg_used;        // fp32 factor copies (GEAR_FLAG_KEEP_FP32_FACTORS)
   SegDesc* table_dev; int table_cap;
+  int* blk2seg; int blk_cap;                             // segment index of every compressed block
   void* buf_k; void* buf_v;                              // [BH][n_b][128] fp16
   unsigned char* flush_ws; size_t flush_ws_bytes;
   float* partial; size_t partial_bytes; int max_parts;
@@ -43,8 +41,8 @@ struct gear_cache {
   long long n_compressed;
   int n_blocks_c;
   // cached launch plan of the decode kernel (depends on the segments' shapes)
-  int plan_key, plan_warps, plan_grid, plan_stage, plan_warp_smem, plan_max_T, plan_max_rpad;
-  size_t plan_smem;
+  int plan_key, plan_occ;
+  DecodeArgs plan;
 };
 
 static int outlier_count(float s_pct, int len) {
@@ -90,7 +88,7 @@ static SegDesc shape_segment(const gear_cache* c, int n_c, int rank) {
 
 extern "C" void gear_free(gear_cache* c) {
   if (!c) return;
-  cudaFree(c->arena); cudaFree(c->dbg); cudaFree(c->table_dev); cudaFree(c->buf_k); cudaFree(c->buf_v);
+  cudaFree(c->arena); cudaFree(c->dbg); cudaFree(c->table_dev); cudaFree(c->blk2seg); cudaFree(c->buf_k); cudaFree(c->buf_v);
   cudaFree(c->flush_ws); cudaFree(c->partial); cudaFree(c->tickets); cudaFree(c->status);
   cudaFree(c->stage_k); cudaFree(c->stage_v); cudaFree(c->stage_q); cudaFree(c->stage_out); cudaFree(c->stage_b0);
   delete c;
@@ -112,7 +110,7 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   gear_cache* c = new (std::nothrow) gear_cache();
   if (!c) return GEAR_ERR_ALLOC;
   c->cfg = *cfg;
-  c->arena = nullptr; c->dbg = nullptr; c->table_dev = nullptr; c->buf_k = c->buf_v = nullptr; c->flush_ws = nullptr;
+  c->arena = nullptr; c->dbg = nullptr; c->table_dev = nullptr; c->blk2seg = nullptr; c->buf_k = c->buf_v = nullptr; c->flush_ws = nullptr;
   c->partial = nullptr; c->tickets = nullptr; c->status = nullptr;
   c->stage_k = c->stage_v = c->stage_q = nullptr; c->stage_out = nullptr; c->stage_b0 = nullptr;
   c->cc.bits = cfg->bits;
@@ -144,6 +142,8 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   GEAR_TRY_ALLOC(c->arena, c->arena_bytes);
   c->table_cap = (int)(cfg->max_tokens / 16 + 8);
   GEAR_TRY_ALLOC(c->table_dev, sizeof(SegDesc) * (size_t)c->table_cap);
+  c->blk_cap = (int)(cfg->max_tokens / 16 + 8);
+  GEAR_TRY_ALLOC(c->blk2seg, sizeof(int) * (size_t)c->blk_cap);
   GEAR_TRY_ALLOC(c->buf_k, BH * n_b * kHeadDim * 2);
   GEAR_TRY_ALLOC(c->buf_v, BH * n_b * kHeadDim * 2);
   c->flush_ws_bytes = compress_workspace_bytes((int)BH, n_b, cfg->rank_flush);
@@ -158,7 +158,7 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   const int hp = c->G <= 4 ? 4 : 8;
   const int passes = (c->G + hp - 1) / hp;
   const size_t units = BH * passes;
-  const size_t nw_max = (size_t)c->sm_count * 16;
+  const size_t nw_max = (size_t)c->sm_count * 32;        // one warp per CTA, at most 32 CTAs per SM
   c->max_parts = (int)(nw_max / units + 3);
   c->partial_bytes = units * c->max_parts * (size_t)hp * 130 * 4;
   GEAR_TRY_ALLOC(c->partial, c->partial_bytes);
@@ -183,6 +183,7 @@ static gear_status compress_segment(gear_cache* c, const void* K, const void* V,
   if ((int)c->segs.size() >= c->table_cap) return GEAR_ERR_CAPACITY;
   if (c->n_compressed + n > c->cfg.max_tokens) return GEAR_ERR_CAPACITY;
   SegDesc sd = shape_segment(c, n, rank);
+  if (c->n_blocks_c + sd.nblk > c->blk_cap) return GEAR_ERR_CAPACITY;
   if (sd.k_k > kMaxOutliers || (sd.k_k > 0 && 2 * sd.k_k >= sd.T)) return GEAR_ERR_SHAPE;
   const size_t need = align_up((size_t)sd.bh_stride, 16) * c->cc.BH;
   sd.bh_stride = (long long)align_up((size_t)sd.bh_stride, 16);
@@ -225,7 +226,7 @@ static gear_status compress_segment(gear_cache* c, const void* K, const void* V,
     cudaFreeAsync(ws, st);
   }
   if (e != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
-  e = launch_write_desc(c->table_dev, (int)c->segs.size(), sd, st);
+  e = launch_write_desc(c->table_dev, c->blk2seg, (int)c->segs.size(), sd, st);
   if (e != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
   c->segs.push_back(sd);
   c->dbgA_off.push_back(offA); c->dbgB_off.push_back(offB);
@@ -284,27 +285,19 @@ extern "C" gear_status gear_append_buffer(gear_cache* c, const void* k_new, cons
 }
 
 static gear_status plan_decode(gear_cache* c) {
-  const int key = (int)c->segs.size() * 4096 + c->buf_len;
+  const int key = (int)c->segs.size();
   if (c->plan_key == key) return GEAR_OK;
-  int max_rec = 0, max_bfac = 0, max_T = 16, max_rpad = 0;
+  int max_k = 0, max_v = 0, max_bfac = 0, max_T = 16;
   for (const SegDesc& s : c->segs) {
-    if (s.rec_bytes > max_rec) max_rec = s.rec_bytes;
+    if (s.off_vpart > max_k) max_k = s.off_vpart;
+    if (s.rec_bytes - s.off_vpart > max_v) max_v = s.rec_bytes - s.off_vpart;
     if (s.bfac_bytes > max_bfac) max_bfac = s.bfac_bytes;
     if (s.T > max_T) max_T = s.T;
-    if (s.r_pad > max_rpad) max_rpad = s.r_pad;
   }
-  const int hp = c->G <= 4 ? 4 : 8;
-  int stage = 0, wsm = 0;
-  decode_smem_plan(c->cc.bits, max_rec, max_bfac, max_T, max_rpad, hp, &stage, &wsm);
-  int warps = 4;
-  while (warps > 1 && (size_t)warps * wsm > 220 * 1024) warps >>= 1;
-  const size_t smem = (size_t)warps * wsm;
-  if (smem > 227 * 1024) return GEAR_ERR_SHAPE;
-  int occ = decode_occupancy(c->cc.bits, c->G, warps, smem);
+  if (!decode_plan(c->cc.bits, c->G, c->cc.ngv, max_k, max_v, max_bfac, max_T, 227 * 1024, &c->plan)) return GEAR_ERR_SHAPE;
+  const int occ = decode_occupancy(c->cc.bits, c->G, c->cc.ngv, (size_t)c->plan.ws.total);
   if (occ < 1) return GEAR_ERR_CUDA;
-  if (occ * warps > 16) occ = 16 / warps;
-  c->plan_warps = warps; c->plan_grid = c->sm_count * occ; c->plan_stage = stage; c->plan_warp_smem = wsm;
-  c->plan_max_T = max_T; c->plan_max_rpad = max_rpad; c->plan_smem = smem;
+  c->plan_occ = occ;
   c->plan_key = key;
   return GEAR_OK;
 }
@@ -315,16 +308,20 @@ extern "C" gear_status gear_decode_attn(gear_cache* c, const void* q, float* out
   if (c->n_compressed == 0 && c->buf_len == 0) return GEAR_ERR_STATE;
   gear_status s = plan_decode(c);
   if (s != GEAR_OK) return s;
-  DecodeArgs a;
-  a.arena = c->arena; a.table = c->table_dev;
+  DecodeArgs a = c->plan;
+  a.arena = c->arena; a.table = c->table_dev; a.blk2seg = c->blk2seg;
   a.buf_k = (const __half*)c->buf_k; a.buf_v = (const __half*)c->buf_v;
   a.q = (const __half*)q; a.out = out; a.partial = c->partial; a.tickets = c->tickets; a.status = c->status;
-  a.cc = c->cc; a.nseg = (int)c->segs.size(); a.n_blocks_c = c->n_blocks_c; a.buf_len = c->buf_len;
+  a.cc = c->cc; a.n_blocks_c = c->n_blocks_c; a.buf_len = c->buf_len;
   a.n_kv_heads = c->cfg.n_kv_heads; a.group_heads = c->G; a.max_parts = c->max_parts;
-  a.stage_bytes = c->plan_stage; a.warp_smem = c->plan_warp_smem; a.max_T = c->plan_max_T; a.max_rpad = c->plan_max_rpad;
   const float sc = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)kHeadDim);
   a.scale_log2 = sc * 1.4426950408889634f;
-  if (launch_decode(a, c->plan_warps, c->plan_grid, c->plan_smem, (cudaStream_t)stream) != cudaSuccess) {
+  // one warp per CTA; never more warps than blocks of work
+  const int hp = c->G <= 4 ? 4 : 8;
+  const long long work = (long long)c->cc.BH * ((c->G + hp - 1) / hp) * (c->n_blocks_c + (c->buf_len + 15) / 16);
+  long long grid = (long long)c->sm_count * c->plan_occ;
+  if (grid > work) grid = work;
+  if (launch_decode(a, (int)grid, (cudaStream_t)stream) != cudaSuccess) {
     cudaGetLastError();
     return GEAR_ERR_CUDA;
   }

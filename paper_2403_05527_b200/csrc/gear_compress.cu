@@ -539,8 +539,9 @@ __global__ void __launch_bounds__(256) pi_gram2_kernel(PiArgs p) {
 
 // Segment with rank 0: nothing to fit, but the A sections of the records do not exist either.
 // Segment descriptor table entry, written by the device so that no host copy is needed.
-__global__ void write_desc_kernel(SegDesc* table, int index, SegDesc d) {
-  if (threadIdx.x == 0 && blockIdx.x == 0) table[index] = d;
+__global__ void write_desc_kernel(SegDesc* table, int* blk2seg, int index, SegDesc d) {
+  if (threadIdx.x == 0) table[index] = d;
+  for (int b = threadIdx.x; b < d.nblk; b += blockDim.x) blk2seg[d.blk_start + b] = index;
 }
 
 __global__ void append_kernel(__half* buf_k, __half* buf_v, const __half* k_new, const __half* v_new,
@@ -658,8 +659,8 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
   return cudaGetLastError();
 }
 
-cudaError_t launch_write_desc(SegDesc* table, int index, const SegDesc& d, cudaStream_t st) {
-  write_desc_kernel<<<1, 32, 0, st>>>(table, index, d);
+cudaError_t launch_write_desc(SegDesc* table, int* blk2seg, int index, const SegDesc& d, cudaStream_t st) {
+  write_desc_kernel<<<1, 256, 0, st>>>(table, blk2seg, index, d);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -7,9 +7,8 @@
 #include "gear_internal.cuh"
 
 namespace gear {
-int decode_occupancy(int bits, int G, int warps_per_cta, size_t smem);
 
-static const int kFp16MaxWarps = 148 * 16 * 2;
+static const int kFp16MaxWarps = 148 * 32 * 2;
 
 size_t fp16_attn_scratch(int batch, int n_q_heads) {
   // tickets + status, then partials: one per (unit, warp touching it); units <= batch * n_q_heads
@@ -27,30 +26,28 @@ cudaError_t launch_fp16_attn(const void* K, const void* V, const void* q, float*
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  int stage = 0, wsm = 0;
-  decode_smem_plan(2, 0, 0, 16, 0, hp, &stage, &wsm);
-  const int warps = 4;
-  const size_t smem = (size_t)warps * wsm;
-  int occ = decode_occupancy(2, G, warps, smem);
-  if (occ < 1) return cudaErrorInvalidConfiguration;
-  if (occ * warps > 16) occ = 16 / warps;
-  const int grid = sms * occ;
-  unsigned char* s = reinterpret_cast<unsigned char*>(scratch);
   DecodeArgs a;
-  a.arena = nullptr; a.table = nullptr;
+  if (!decode_plan(2, G, 1, 0, 0, 0, 16, 227 * 1024, &a)) return cudaErrorInvalidConfiguration;
+  const int occ = decode_occupancy(2, G, 1, (size_t)a.ws.total);
+  if (occ < 1) return cudaErrorInvalidConfiguration;
+  long long grid = (long long)sms * occ;
+  const long long work = (long long)units * ((n + 15) / 16);
+  if (grid > work) grid = work;
+  if (grid > kFp16MaxWarps) grid = kFp16MaxWarps;
+  unsigned char* s = reinterpret_cast<unsigned char*>(scratch);
+  a.arena = nullptr; a.table = nullptr; a.blk2seg = nullptr;
   a.buf_k = (const __half*)K; a.buf_v = (const __half*)V; a.q = (const __half*)q; a.out = out;
   a.status = reinterpret_cast<int*>(s);
   a.tickets = reinterpret_cast<int*>(s + 256);
   a.partial = reinterpret_cast<float*>(s + 256 + ((units * 4 + 255) / 256) * 256);
   a.cc.bits = 2; a.cc.g_v = kHeadDim; a.cc.ngv = 1; a.cc.k_v = 0; a.cc.BH = batch * n_kv_heads; a.cc.n_b = (int)n_alloc;
-  a.nseg = 0; a.n_blocks_c = 0; a.buf_len = (int)n;
+  a.n_blocks_c = 0; a.buf_len = (int)n;
   a.n_kv_heads = n_kv_heads; a.group_heads = G;
-  a.max_parts = (int)((size_t)grid * warps / units + 3);
-  a.stage_bytes = stage; a.warp_smem = wsm; a.max_T = 16; a.max_rpad = 0;
+  a.max_parts = (int)((size_t)grid / units + 3);
   a.scale_log2 = scale * 1.4426950408889634f;
   cudaError_t e = cudaMemsetAsync(s, 0, 256 + units * 4, st);
   if (e != cudaSuccess) return e;
-  return launch_decode(a, warps, grid, smem, st);
+  return launch_decode(a, (int)grid, st);
 }
 
 }  // namespace gear

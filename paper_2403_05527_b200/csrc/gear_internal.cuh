@@ -52,36 +52,44 @@ struct CompressJob {
 
 size_t compress_workspace_bytes(int nbh, int n_c, int rank);
 cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned char* ws, cudaStream_t st);
-cudaError_t launch_write_desc(SegDesc* table, int index, const SegDesc& d, cudaStream_t st);
+cudaError_t launch_write_desc(SegDesc* table, int* blk2seg, int index, const SegDesc& d, cudaStream_t st);
 cudaError_t launch_append(void* buf_k, void* buf_v, const void* k_new, const void* v_new, int BH, int n_b, int slot,
                           cudaStream_t st);
 
 // decode attention over the compressed cache
+constexpr int kMaxStages = 4;
+struct WarpSmem {      // byte offsets of a warp's (= a CTA's) shared-memory regions
+  int ring, sdp, sdc, qf, qs, frag, corr_k, ps, corr_v, ocorr, wl, misc, total;
+};
 struct DecodeArgs {
   const unsigned char* arena;
   const SegDesc* table;
+  const int* blk2seg;         // [n_blocks_c] segment index of every compressed block
   const __half* buf_k;        // [BH][n_b][128]
   const __half* buf_v;
   const __half* q;            // [B][Hq][128]
   float* out;                 // [B][Hq][128]
-  float* partial;             // [BH][max_parts][G][130]
-  int* tickets;               // [BH * head passes]
+  float* partial;             // [units][max_parts][HP][130]
+  int* tickets;               // [units]
   int* status;
   CacheConst cc;
-  int nseg;
   int n_blocks_c;             // compressed blocks per (batch, head)
   int buf_len;                // tokens in the fp16 buffer
   int n_kv_heads, group_heads;   // H, G = Hq / H
   int max_parts;
+  int nstage;                 // ring stages (<= kMaxStages)
   int stage_bytes;            // bytes of one ring stage
-  int warp_smem;              // bytes of shared memory per warp
+  int bregion;                // bytes at the front of a stage reserved for one B factor
   int max_T;                  // largest block length over the segments
-  int max_rpad;
+  int hpa;                    // query heads per pass that get shared-memory rows
+  WarpSmem ws;
   float scale_log2;           // softmax scale * log2(e)
 };
-cudaError_t launch_decode(const DecodeArgs& a, int warps_per_cta, int grid, size_t smem, cudaStream_t st);
-void decode_smem_plan(int bits, int max_rec, int max_bfac, int max_T, int max_rpad, int heads_per_pass,
-                      int* stage_bytes, int* warp_smem);
+cudaError_t launch_decode(const DecodeArgs& a, int grid, cudaStream_t st);
+// Shared-memory plan of one warp; returns false if no stage count fits.  heads = G (query heads per kv head).
+bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int max_bfac, int max_T, size_t smem_budget,
+                 DecodeArgs* a);
+int decode_occupancy(int bits, int heads, int ngv, size_t smem);
 
 // fp16-cache attention
 cudaError_t launch_fp16_attn(const void* K, const void* V, const void* q, float* out, int batch, int n_q_heads,

@@ -8,19 +8,22 @@
 //     [ B factors ][ record of block 0 ][ record of block 1 ] ...
 // so that the decode kernel fetches a block (and, for block 0, the factors in
 // front of it) with one bulk copy.  A record holds, section by section:
+// key part (everything the score pass needs), then value part:
 //     header     16 B : fp32 max |x - zero| over the block's key / value outliers
 //     kscale     128 x (scale fp16, zero fp16)                 one pair per channel
 //     koval      128 x 2k_K fp16   outlier values, per channel, in-group index ascending
 //     koidx      128 x 2k_K u8     their token index inside the block
 //     kcodes     T/16 slabs x 16*128*b/8 bytes, in mma-fragment order (see code_coord_k)
-//     vcodes     same size, (see code_coord_v)
 //     ak         T/16 slabs x [16 tokens][r_pad] fp16          rows of A_K
+//   -- off_vpart --
+//     vcodes     same size as kcodes (see code_coord_v)
 //     av         T/16 slabs x [r_pad][16 tokens] fp16          rows of A_V, transposed per slab
 //     vscale     T x (d_H/g_V) x (scale fp16, zero fp16)
 //     voval      T x (d_H/g_V) x 2k_V fp16
 //     voidx      T x (d_H/g_V) x 2k_V u8   channel index inside the group
-// Every section starts on a 16-byte boundary.  The B factors are
-//     [r_pad][128] fp16 (B_K transposed)  then  [128][r_pad] fp16 (B_V).
+// Every section starts on a 16-byte boundary, so the decode kernel can fetch the
+// key part and the value part of a block with one bulk copy each.  The B factors
+// are  [r_pad][128] fp16 (B_K transposed)  then  [128][r_pad] fp16 (B_V).
 #pragma once
 #include <stdint.h>
 
@@ -50,7 +53,7 @@ struct SegDesc {
       off_vscale, off_voval, off_voidx;
   int slab_codes;        // bytes of codes per slab and side
   int slab_a;            // bytes of A rows per slab and side
-  int pad_;
+  int off_vpart;         // start of the value part inside a record (= bytes of the key part)
 };
 
 // Cache-wide constants the kernels need.
@@ -82,15 +85,15 @@ __host__ __device__ inline void layout_segment(SegDesc& s, const CacheConst& c) 
   s.off_koval = o;   o += kHeadDim * 2 * s.k_k * 2;
   s.off_koidx = o;   o += round_up(kHeadDim * 2 * s.k_k, 16);
   s.off_kcodes = o;  o += nslab * s.slab_codes;
-  s.off_vcodes = o;  o += nslab * s.slab_codes;
   s.off_ak = o;      o += round_up(nslab * s.slab_a, 16);
+  s.off_vpart = o;
+  s.off_vcodes = o;  o += nslab * s.slab_codes;
   s.off_av = o;      o += round_up(nslab * s.slab_a, 16);
   s.off_vscale = o;  o += s.T * c.ngv * 4;
   s.off_voval = o;   o += round_up(s.T * c.ngv * 2 * c.k_v * 2, 16);
   s.off_voidx = o;   o += round_up(s.T * c.ngv * 2 * c.k_v, 16);
   s.rec_bytes = o;
   s.bh_stride = (long long)s.bfac_bytes + (long long)s.nblk * s.rec_bytes;
-  s.pad_ = 0;
 }
 
 // ---------------------------------------------------------------------------
