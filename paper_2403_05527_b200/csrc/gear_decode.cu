@@ -31,8 +31,6 @@ namespace gear {
 constexpr int kBufPitch = 272;                  // bytes per fp16 row of a buffer slab in shared memory
 constexpr int kBufItem = kSlab * kBufPitch;     // one slab of key rows or of value rows
 constexpr int kSpinLimit = 4000000;
-constexpr int kChunkSlabs = 4;                  // slabs whose scores are held in registers at once
-constexpr int kChunkTok = kChunkSlabs * kSlab;
 constexpr int kFragStride = 72;                 // 32-bit words per fragment row set (64 + padding against bank conflicts)
 
 static_assert(sizeof(SegDesc) <= 128 && sizeof(SegDesc) % 4 == 0, "descriptor copy assumes <= 32 words");
@@ -136,45 +134,48 @@ __device__ __forceinline__ int clamp60(int e) { return max(-60, min(60, e)); }
 bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int max_bfac, int max_T, size_t smem_budget,
                  DecodeArgs* a) {
   (void)bits;
-  const int NT = heads <= 4 ? 1 : 2, HP = 4 * NT;
-  const int hpa = heads < HP ? heads : HP;
+  const int HP = heads == 1 ? 1 : (heads <= 4 ? 4 : 8), NT = HP > 4 ? 2 : 1;
   const int bregion = round_up(max_bfac / 2, 128);
   int part = max_kpart > max_vpart ? max_kpart : max_vpart;
   int stage = bregion + part;
   if (stage < kBufItem) stage = kBufItem;
   stage = round_up(stage, 128);
   if (max_T < kSlab) max_T = kSlab;
-  const int frag_rows = 8 > kChunkSlabs * (ngv + 1) ? 8 : kChunkSlabs * (ngv + 1);
+  const int nslab = max_T / kSlab;
+  const int frag_rows = 8 > nslab * (ngv + 1) ? 8 : nslab * (ngv + 1);
   for (int ns = kMaxStages; ns >= 2; --ns) {
     WarpSmem w;
     int o = 0;
     w.ring = o;    o += ns * stage;
     w.sdp = o;     o += 128;
     w.sdc = o;     o += 128;
-    w.qf = o;      o += hpa * kHeadDim * 4;
-    w.qs = o;      o += hpa * kHeadDim * 2;
+    w.qf = o;      o += HP * kHeadDim * 4;
+    w.qs = o;      o += HP * kHeadDim * 2;
     w.frag = o;    o += NT * frag_rows * kFragStride * 4;
-    w.corr_k = o;  o += hpa * max_T * 4;
-    w.ps = o;      o += hpa * kChunkTok * 4;
-    w.corr_v = o;  o += hpa * kHeadDim * 4;
-    w.ocorr = o;   o += hpa * kHeadDim * 4;
-    w.wl = o;      o += kMaxRank * HP * 4;
-    w.misc = o;    o += 4 * HP * 4;
+    w.corr_k = o;  o += HP * max_T * 4;
+    w.ps = o;      o += HP * max_T * 4;
+    w.corr_v = o;  o += HP * kHeadDim * 4;
+    w.ocorr = o;   o += HP * kHeadDim * 4;
+    w.wl = o;      o += kMaxRank * 8 * 4;
+    w.misc = o;    o += 64;
     w.total = round_up(o, 128);
     // prefer three stages with more resident warps over four stages with fewer
-    if (ns == kMaxStages && (size_t)w.total * 10 > smem_budget) continue;
+    if (ns == kMaxStages && (size_t)(w.total + 1024) * 10 > smem_budget) continue;
     if ((size_t)w.total > smem_budget) continue;
-    a->nstage = ns; a->stage_bytes = stage; a->bregion = bregion; a->max_T = max_T; a->hpa = hpa; a->ws = w;
+    a->nstage = ns; a->stage_bytes = stage; a->bregion = bregion; a->max_T = max_T; a->hpa = HP; a->ws = w;
     return true;
   }
   return false;
 }
 
 // ------------------------------------------------------------------ the kernel
-template <int BITS, int NT, int NGV>
-__global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const __grid_constant__ DecodeArgs a) {
-  constexpr int HP = 4 * NT;                      // query heads per pass
+// HEADS = query heads handled per pass: 1 (multi-head attention), 4 or 8 (grouped queries; a pass may hold fewer).
+template <int BITS, int HEADS, int NGV>
+__global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(const __grid_constant__ DecodeArgs a) {
+  constexpr int HP = HEADS;
+  constexpr int NT = HEADS > 4 ? 2 : 1;           // 8-column tiles of the B operand
   constexpr int GV = kHeadDim / NGV;              // channels per value group
+  constexpr int SLABW = kSlab * kHeadDim * BITS / 8 / 16;   // uint4 per slab of codes
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ __align__(8) uint64_t bar[kMaxStages];
 
@@ -186,125 +187,130 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
   unsigned char* ring = smem + a.ws.ring;
   SegDesc* sdp = reinterpret_cast<SegDesc*>(smem + a.ws.sdp);
   SegDesc* sdc = reinterpret_cast<SegDesc*>(smem + a.ws.sdc);
-  float* qf = reinterpret_cast<float*>(smem + a.ws.qf);          // [hpa][128] q * scale * log2(e)
-  __half* qs = reinterpret_cast<__half*>(smem + a.ws.qs);        // [hpa][128] q
+  float* qf = reinterpret_cast<float*>(smem + a.ws.qf);          // [HP][128] q * scale * log2(e)
+  __half* qs = reinterpret_cast<__half*>(smem + a.ws.qs);        // [HP][128] q
   uint32_t* frag = reinterpret_cast<uint32_t*>(smem + a.ws.frag);
-  int* corr_k = reinterpret_cast<int*>(smem + a.ws.corr_k);      // [hpa][maxT]
-  float* ps = reinterpret_cast<float*>(smem + a.ws.ps);          // [hpa][64]
-  int* corr_v = reinterpret_cast<int*>(smem + a.ws.corr_v);      // [hpa][128]
-  float* ocorr = reinterpret_cast<float*>(smem + a.ws.ocorr);    // [hpa][128]
-  float* wl = reinterpret_cast<float*>(smem + a.ws.wl);          // [16][HP]
+  int* corr_k = reinterpret_cast<int*>(smem + a.ws.corr_k);      // [HP][maxT]
+  float* ps = reinterpret_cast<float*>(smem + a.ws.ps);          // [HP][maxT] scores, then probabilities
+  int* corr_v = reinterpret_cast<int*>(smem + a.ws.corr_v);      // [HP][128]
+  float* ocorr = reinterpret_cast<float*>(smem + a.ws.ocorr);    // [HP][128]
+  float* wl = reinterpret_cast<float*>(smem + a.ws.wl);          // [16][8]
   int* qexp_s = reinterpret_cast<int*>(smem + a.ws.misc);        // [HP]
-  float* alpha_s = reinterpret_cast<float*>(smem + a.ws.misc) + HP;
-
-  // value-phase fragments share the region of the key-phase ones
-  uint32_t* fragV = frag;                                        // [NT][NGV][4 slabs] rows of kFragStride words
-  uint32_t* fragP = frag + NT * NGV * kChunkSlabs * kFragStride; // [NT][4 slabs]
 
   if (lane == 0)
     for (int s = 0; s < NS; ++s) mbar_init(&bar[s], 1);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   for (int i = lane; i < (a.ws.corr_k - a.ws.frag) / 4; i += 32) frag[i] = 0u;
-  for (int i = lane; i < a.hpa * maxT; i += 32) corr_k[i] = 0;
-  for (int i = lane; i < a.hpa * kHeadDim; i += 32) corr_v[i] = 0;
+  for (int i = lane; i < HP * maxT; i += 32) corr_k[i] = 0;
+  for (int i = lane; i < HP * kHeadDim; i += 32) corr_v[i] = 0;
   __syncwarp();
 
   // ---- this warp's range of the flat (unit, block) space; unit = (batch, kv head, head pass)
   const int nbuf_blocks = (a.buf_len + kSlab - 1) / kSlab;
   const int NB = a.n_blocks_c + nbuf_blocks;
-  const long long F = (long long)a.cc.BH * passes * NB;
-  const long long NW = gridDim.x, gw = blockIdx.x;
-  const long long f0 = gw * F / NW, f1 = (gw + 1) * F / NW;
-  if (f0 >= f1) return;                      // the host launches no more warps than blocks
+  int n_left, u, blk_lo;                        // blocks left for this warp, current unit, first block in it
+  {
+    const long long F = (long long)a.cc.BH * passes * NB;
+    const long long NW = gridDim.x, gw = blockIdx.x;
+    const long long f0 = gw * F / NW, f1 = (gw + 1) * F / NW;
+    if (f0 >= f1) return;                       // the host launches no more warps than blocks
+    n_left = (int)(f1 - f0);
+    u = (int)(f0 / NB);
+    blk_lo = (int)(f0 - (long long)u * NB);
+  }
 
-  // ---- producer: two items per block (key part, value part), issued in order into ring stage n_issued % NS
-  long long p_f = f0;
-  int p_unit = (int)(f0 / NB);
-  int p_blk = (int)(f0 - (long long)p_unit * NB);
-  int p_share_lo = p_blk, p_half = 0, n_issued = 0, p_seg_lo = 0, p_seg_hi = 0;
   auto load_desc = [&](SegDesc* dst, int blk) {
     const int* src = reinterpret_cast<const int*>(a.table + a.blk2seg[blk]);
     __syncwarp();
     if (lane < (int)(sizeof(SegDesc) / 4)) reinterpret_cast<int*>(dst)[lane] = src[lane];
     __syncwarp();
   };
+
+  // ---- producer: two items per block (key part, value part), issued in order into the ring
+  int p_left = n_left, p_blk = blk_lo, p_share_lo = blk_lo, p_half = 0, p_stage = 0;
+  int p_bh = u / passes, p_pass = u - p_bh * passes;
+  int p_seg_lo = 0, p_seg_hi = 0, p_kbytes = 0, p_vbytes = 0, p_hb = 0;
+  const unsigned char* p_segb = nullptr;        // B factors of the producer's (segment, batch, head)
+  const unsigned char* p_rec = nullptr;         // record of block p_blk
+  int n_inflight = 0;
   auto issue = [&]() {
-    if (p_f >= f1) return;
-    const int s = n_issued % NS;
-    unsigned char* dst = ring + (size_t)s * a.stage_bytes;
+    if (p_left == 0) return;
+    unsigned char* dst = ring + p_stage * a.stage_bytes;
+    uint64_t* b = &bar[p_stage];
     if (p_blk < a.n_blocks_c) {
-      if (p_blk < p_seg_lo || p_blk >= p_seg_hi) {
+      if (p_blk >= p_seg_hi) {                  // new segment (or new unit): refresh the cached descriptor
         load_desc(sdp, p_blk);
         p_seg_lo = sdp->blk_start;
         p_seg_hi = p_seg_lo + sdp->nblk;
+        p_kbytes = sdp->off_vpart;
+        p_vbytes = sdp->rec_bytes - p_kbytes;
+        p_hb = sdp->bfac_bytes >> 1;
+        p_segb = a.arena + sdp->seg_base + (size_t)p_bh * sdp->bh_stride;
+        p_rec = p_segb + 2 * p_hb + (size_t)(p_blk - p_seg_lo) * (p_kbytes + p_vbytes);
       }
       if (lane == 0) {
-        const int bl = p_blk - p_seg_lo;
-        const int bh = p_unit / passes;
-        const int hb = sdp->bfac_bytes >> 1;
-        const unsigned char* src_b = a.arena + sdp->seg_base + (size_t)bh * sdp->bh_stride;
-        const unsigned char* src_r = src_b + sdp->bfac_bytes + (size_t)bl * sdp->rec_bytes;
         if (p_half == 0) {
-          const bool wb = hb > 0 && (bl == 0 || p_blk == p_share_lo);
-          mbar_expect_tx(&bar[s], sdp->off_vpart + (wb ? hb : 0));
-          if (wb) bulk_g2s(dst, src_b, hb, &bar[s]);
-          bulk_g2s(dst + a.bregion, src_r, sdp->off_vpart, &bar[s]);
+          const bool wb = p_hb > 0 && (p_blk == p_seg_lo || p_blk == p_share_lo);
+          mbar_expect_tx(b, p_kbytes + (wb ? p_hb : 0));
+          if (wb) bulk_g2s(dst, p_segb, p_hb, b);
+          bulk_g2s(dst + a.bregion, p_rec, p_kbytes, b);
         } else {
-          const bool wb = hb > 0 && (bl == p_seg_hi - p_seg_lo - 1 || p_f == f1 - 1);
-          const int vbytes = sdp->rec_bytes - sdp->off_vpart;
-          mbar_expect_tx(&bar[s], vbytes + (wb ? hb : 0));
-          if (wb) bulk_g2s(dst, src_b + hb, hb, &bar[s]);
-          bulk_g2s(dst + a.bregion, src_r + sdp->off_vpart, vbytes, &bar[s]);
+          const bool wb = p_hb > 0 && (p_blk == p_seg_hi - 1 || p_left == 1);
+          mbar_expect_tx(b, p_vbytes + (wb ? p_hb : 0));
+          if (wb) bulk_g2s(dst, p_segb + p_hb, p_hb, b);
+          bulk_g2s(dst + a.bregion, p_rec + p_kbytes, p_vbytes, b);
         }
       }
     } else if (lane == 0) {
       const int j = p_blk - a.n_blocks_c;
       const int rows = min(kSlab, a.buf_len - j * kSlab);
-      const int bh = p_unit / passes;
-      const __half* src = (p_half == 0 ? a.buf_k : a.buf_v) + ((size_t)bh * a.cc.n_b + (size_t)j * kSlab) * kHeadDim;
-      mbar_expect_tx(&bar[s], rows * 256);
-      for (int r = 0; r < rows; ++r) bulk_g2s(dst + r * kBufPitch, src + r * kHeadDim, 256, &bar[s]);
+      const __half* src = (p_half == 0 ? a.buf_k : a.buf_v) + ((size_t)p_bh * a.cc.n_b + (size_t)j * kSlab) * kHeadDim;
+      mbar_expect_tx(b, rows * 256);
+      for (int r = 0; r < rows; ++r) bulk_g2s(dst + r * kBufPitch, src + r * kHeadDim, 256, b);
     }
-    ++n_issued;
+    ++n_inflight;
+    if (++p_stage == NS) p_stage = 0;
     if (p_half == 0) {
       p_half = 1;
     } else {
-      p_half = 0; ++p_f; ++p_blk;
-      if (p_blk == NB) { p_blk = 0; ++p_unit; p_share_lo = 0; }
+      p_half = 0; --p_left; ++p_blk;
+      p_rec += p_kbytes + p_vbytes;
+      if (p_blk == NB) {
+        p_blk = 0; p_share_lo = 0; p_seg_hi = 0;
+        if (++p_pass == passes) { p_pass = 0; ++p_bh; }
+      }
     }
   };
   for (int s = 0; s < NS; ++s) issue();
 
-  int n_released = 0, item_k = 0, c_seg_lo = 0, c_seg_hi = 0;     // item_k: index of the current block's key item
+  int c_stage = 0, c_par = 0, c_seg_lo = 0, c_seg_hi = 0;
   bool alive = true;
-  // wait for item `idx`; returns its stage
-  auto acquire = [&](int idx) -> unsigned char* {
-    const int s = idx % NS;
-    if (!mbar_wait(&bar[s], (uint32_t)((idx / NS) & 1), a.status)) { alive = false; return nullptr; }
-    return ring + (size_t)s * a.stage_bytes;
+  // wait for the next item (items are consumed in order); returns its stage
+  auto acquire = [&]() -> unsigned char* {
+    unsigned char* st = ring + c_stage * a.stage_bytes;
+    if (!mbar_wait(&bar[c_stage], (uint32_t)c_par, a.status)) alive = false;
+    if (++c_stage == NS) { c_stage = 0; c_par ^= 1; }
+    --n_inflight;
+    return st;
   };
-  auto release = [&]() {       // the oldest item is consumed (items are released in order): refill its stage
+  auto release = [&]() {       // the oldest item is consumed: refill its stage
     __syncwarp();
-    ++n_released;
     issue();
   };
 
   // ---- loop over the units this warp touches
-  long long f = f0;
-  while (f < f1 && alive) {
-    const int u = (int)(f / NB);
-    const int blk_lo = (int)(f - (long long)u * NB);
-    const int blk_hi = (int)min((long long)NB, blk_lo + (f1 - f));
+  while (n_left > 0 && alive) {
+    const int blk_hi = min(NB, blk_lo + n_left);
     const int bh = u / passes, pass = u - bh * passes;
-    const int HPu = min(HP, G - pass * HP);
+    const int HPu = HEADS == 1 ? 1 : min(HP, G - pass * HP);
     const int hq0 = bh * G + pass * HP;                 // first query head of this pass
 
     // unit state
-    float O[8][NT][4], U[NT][4], m_run[NT], l_run[NT], cm[HP][NGV];
+    float O[8][NT][4], U[NT][4], m_run[HP], l_run[HP], cm[HP][NGV];
     uint32_t bw[NT][2];                                  // low-rank key term: B operand (q B_K) of the current segment
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      m_run[nt] = -INFINITY; l_run[nt] = 0.f; bw[nt][0] = bw[nt][1] = 0u;
+      bw[nt][0] = bw[nt][1] = 0u;
 #pragma unroll
       for (int i = 0; i < 4; ++i) U[nt][i] = 0.f;
 #pragma unroll
@@ -313,9 +319,11 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
         for (int i = 0; i < 4; ++i) O[mt][nt][i] = 0.f;
     }
 #pragma unroll
-    for (int h = 0; h < HP; ++h)
+    for (int h = 0; h < HP; ++h) {
+      m_run[h] = -INFINITY; l_run[h] = 0.f;
 #pragma unroll
       for (int g = 0; g < NGV; ++g) cm[h][g] = 0.f;
+    }
     bool u_pending = false;
 
     // query rows of this pass -> shared (fp16 as given, and fp32 times scale * log2 e); exponent of max |q|
@@ -338,28 +346,30 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
     }
     __syncwarp();
 
-    for (int blk = blk_lo; blk < blk_hi && alive; ++blk) {
+#pragma unroll 1
+    for (int blk = blk_lo; blk < blk_hi; ++blk) {
       const bool is_buf = blk >= a.n_blocks_c;
       // ---------------- block geometry
-      int nslab = 1, r_pad = 0, k2k = 0, valid_tokens = kSlab, slab_a = 0;
+      int T = kSlab, r_pad = 0, k2k = 0, valid_tokens = kSlab;
       bool with_bk = false, with_bv = false;
       if (!is_buf) {
-        if (blk < c_seg_lo || blk >= c_seg_hi) {
+        if (blk >= c_seg_hi || blk < c_seg_lo) {
           load_desc(sdc, blk);
           c_seg_lo = sdc->blk_start;
           c_seg_hi = c_seg_lo + sdc->nblk;
         }
-        const int bl = blk - c_seg_lo;
-        nslab = sdc->T / kSlab; r_pad = sdc->r_pad; k2k = 2 * sdc->k_k; slab_a = sdc->slab_a;
-        valid_tokens = sdc->T;
-        with_bk = r_pad > 0 && (bl == 0 || blk == blk_lo);
-        with_bv = r_pad > 0 && (bl == c_seg_hi - c_seg_lo - 1 || blk == blk_hi - 1);
+        T = sdc->T; r_pad = sdc->r_pad; k2k = 2 * sdc->k_k;
+        valid_tokens = T;
+        with_bk = r_pad > 0 && (blk == c_seg_lo || blk == blk_lo);
+        with_bv = r_pad > 0 && (blk == c_seg_hi - 1 || blk == blk_hi - 1);
       } else {
         valid_tokens = min(kSlab, a.buf_len - (blk - a.n_blocks_c) * kSlab);
       }
+      const int nslab = T / kSlab;
+      const int slab_a = 2 * kSlab * r_pad;
 
       // ================================================================ key item
-      unsigned char* stK = acquire(item_k);
+      unsigned char* stK = acquire();
       if (!alive) break;
       const unsigned char* kp = stK + a.bregion;
       float dmax_v = 0.f;
@@ -376,7 +386,7 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
           for (int i = 0; i < 4; ++i) wacc[nt][i] = 0.f;
-#pragma unroll
+#pragma unroll 2
         for (int kc = 0; kc < 8; ++kc) {
           uint32_t af[4] = {0u, 0u, 0u, 0u};
           if (gid < r_pad) {
@@ -402,16 +412,16 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
         __syncwarp();
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {       // D[rho][col 2t] = w[rho][head t + 4nt]
-          wl[gid * HP + t + 4 * nt] = wacc[nt][0] * a.scale_log2;
-          wl[(gid + 8) * HP + t + 4 * nt] = wacc[nt][2] * a.scale_log2;
+          wl[gid * 8 + t + 4 * nt] = wacc[nt][0] * a.scale_log2;
+          wl[(gid + 8) * 8 + t + 4 * nt] = wacc[nt][2] * a.scale_log2;
         }
         __syncwarp();
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           const int h = (gid >> 1) + 4 * nt;
           uint32_t hi0, lo0, hi1, lo1;
-          split_hi_lo(wl[(2 * t) * HP + h], wl[(2 * t + 1) * HP + h], hi0, lo0);
-          split_hi_lo(wl[(2 * t + 8) * HP + h], wl[(2 * t + 9) * HP + h], hi1, lo1);
+          split_hi_lo(wl[(2 * t) * 8 + h], wl[(2 * t + 1) * 8 + h], hi0, lo0);
+          split_hi_lo(wl[(2 * t + 8) * 8 + h], wl[(2 * t + 9) * 8 + h], hi1, lo1);
           bw[nt][0] = (gid & 1) ? lo0 : hi0;
           bw[nt][1] = (gid & 1) ? lo1 : hi1;
         }
@@ -496,120 +506,135 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
           const uint2 v = *reinterpret_cast<const uint2*>(frag + (nt * 8 + kc) * kFragStride + lane * 2);
           bq[nt][kc][0] = v.x; bq[nt][kc][1] = v.y;
         }
-      __syncwarp();                                  // the fragment region is rewritten in the value phase
 
-      unsigned char* stV = nullptr;
-      const int nchunk = (nslab + kChunkSlabs - 1) / kChunkSlabs;
-      for (int c = 0; c < nchunk && alive; ++c) {
-        const int ns = min(kChunkSlabs, nslab - c * kChunkSlabs);
-        // ---------------- key scores of up to four slabs, kept in registers
-        float sc[NT][kChunkSlabs][2];
+      // ---------------- key scores, slab by slab; scores go to shared memory
+      {
+        const uint4* cw = reinterpret_cast<const uint4*>(kp + (is_buf ? 0 : sdc->off_kcodes)) + lane;
+        const __half* ak = reinterpret_cast<const __half*>(kp + (is_buf ? 0 : sdc->off_ak));
+        float Si[NT];
 #pragma unroll
-        for (int s = 0; s < kChunkSlabs; ++s) {
+        for (int nt = 0; nt < NT; ++nt) Si[nt] = pow2i(-own_sexp[nt]);
+#pragma unroll 1
+        for (int slab = 0; slab < nslab; ++slab) {
+          float acc[2][NT][4];
 #pragma unroll
-          for (int nt = 0; nt < NT; ++nt) sc[nt][s][0] = sc[nt][s][1] = -INFINITY;
-          if (s < ns) {
-            const int slab = c * kChunkSlabs + s;
-            float acc[NT][4];
+          for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-              for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
-            uint4 w0 = make_uint4(0u, 0u, 0u, 0u), w1 = w0;
+              for (int i = 0; i < 4; ++i) acc[hf][nt][i] = 0.f;
+          uint4 w0 = make_uint4(0u, 0u, 0u, 0u), w1 = w0;
+          if (!is_buf) {
+            w0 = cw[slab * SLABW];
+            if (BITS == 4) w1 = cw[slab * SLABW + 32];
+          }
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {            // channel chunks 4 hf .. 4 hf + 3
+            uint32_t af[4][4];
             if (!is_buf) {
-              const uint4* cw = reinterpret_cast<const uint4*>(kp + sdc->off_kcodes + slab * sdc->slab_codes);
-              w0 = cw[lane];
-              if (BITS == 4) w1 = cw[32 + lane];
-            }
+              if (BITS == 2) {
+                uint32_t r[8];
+                unpack_word<2>(hf == 0 ? w0.x : w0.y, r);
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {            // channel chunks 4 hf .. 4 hf + 3
-              uint32_t af[4][4];
-              if (!is_buf) {
-                if (BITS == 2) {
-                  uint32_t r[8];
-                  unpack_word<2>(hf == 0 ? w0.x : w0.y, r);
+                for (int u2 = 0; u2 < 8; ++u2) af[u2 >> 1][(u2 & 1) * 2] = r[u2];
+                unpack_word<2>(hf == 0 ? w0.z : w0.w, r);
 #pragma unroll
-                  for (int u2 = 0; u2 < 8; ++u2) af[u2 >> 1][(u2 & 1) * 2] = r[u2];
-                  unpack_word<2>(hf == 0 ? w0.z : w0.w, r);
-#pragma unroll
-                  for (int u2 = 0; u2 < 8; ++u2) af[u2 >> 1][(u2 & 1) * 2 + 1] = r[u2];
-                } else {
-#pragma unroll
-                  for (int th = 0; th < 2; ++th) {
-                    const uint4 w = th == 0 ? w0 : w1;
-                    uint32_t r[4];
-                    unpack_word<4>(hf == 0 ? w.x : w.z, r);
-#pragma unroll
-                    for (int u2 = 0; u2 < 4; ++u2) af[u2 >> 1][(u2 & 1) * 2 + th] = r[u2];
-                    unpack_word<4>(hf == 0 ? w.y : w.w, r);
-#pragma unroll
-                    for (int u2 = 0; u2 < 4; ++u2) af[2 + (u2 >> 1)][(u2 & 1) * 2 + th] = r[u2];
-                  }
-                }
+                for (int u2 = 0; u2 < 8; ++u2) af[u2 >> 1][(u2 & 1) * 2 + 1] = r[u2];
               } else {
 #pragma unroll
-                for (int k4 = 0; k4 < 4; ++k4)
-                  ldmatrix_x4(af[k4], stK + ((lane & 7) + 8 * ((lane >> 3) & 1)) * kBufPitch +
-                                          (16 * (4 * hf + k4) + 8 * (lane >> 4)) * 2);
+                for (int th = 0; th < 2; ++th) {
+                  const uint4 w = th == 0 ? w0 : w1;
+                  uint32_t r[4];
+                  unpack_word<4>(hf == 0 ? w.x : w.z, r);
+#pragma unroll
+                  for (int u2 = 0; u2 < 4; ++u2) af[u2 >> 1][(u2 & 1) * 2 + th] = r[u2];
+                  unpack_word<4>(hf == 0 ? w.y : w.w, r);
+#pragma unroll
+                  for (int u2 = 0; u2 < 4; ++u2) af[2 + (u2 >> 1)][(u2 & 1) * 2 + th] = r[u2];
+                }
               }
+            } else {
 #pragma unroll
               for (int k4 = 0; k4 < 4; ++k4)
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) mma16816(acc[nt], af[k4], bq[nt][4 * hf + k4][0], bq[nt][4 * hf + k4][1]);
-            }
-            if (r_pad > 0) {                          // low-rank key term: A_K rows times w
-              const __half* ak = reinterpret_cast<const __half*>(kp + sdc->off_ak + slab * slab_a);
-              uint32_t aa[4] = {0u, 0u, 0u, 0u};
-              if (2 * t < r_pad) {
-                aa[0] = *reinterpret_cast<const uint32_t*>(ak + gid * r_pad + 2 * t);
-                aa[1] = *reinterpret_cast<const uint32_t*>(ak + (gid + 8) * r_pad + 2 * t);
-              }
-              if (2 * t + 8 < r_pad) {
-                aa[2] = *reinterpret_cast<const uint32_t*>(ak + gid * r_pad + 2 * t + 8);
-                aa[3] = *reinterpret_cast<const uint32_t*>(ak + (gid + 8) * r_pad + 2 * t + 8);
-              }
-#pragma unroll
-              for (int nt = 0; nt < NT; ++nt) mma16816(acc[nt], aa, bw[nt][0], bw[nt][1]);
+                ldmatrix_x4(af[k4], stK + ((lane & 7) + 8 * ((lane >> 3) & 1)) * kBufPitch +
+                                        (16 * (4 * hf + k4) + 8 * (lane >> 4)) * 2);
             }
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-              const int h = t + 4 * nt;
-              const float Si = pow2i(-own_sexp[nt]);
+            for (int k4 = 0; k4 < 4; ++k4)
+#pragma unroll
+              for (int nt = 0; nt < NT; ++nt)
+                mma16816(acc[hf][nt], af[k4], bq[nt][4 * hf + k4][0], bq[nt][4 * hf + k4][1]);
+          }
+          if (r_pad > 0) {                          // low-rank key term: A_K rows times w
+            const __half* aks = ak + slab * (slab_a / 2);
+            uint32_t aa[4] = {0u, 0u, 0u, 0u};
+            if (2 * t < r_pad) {
+              aa[0] = *reinterpret_cast<const uint32_t*>(aks + gid * r_pad + 2 * t);
+              aa[1] = *reinterpret_cast<const uint32_t*>(aks + (gid + 8) * r_pad + 2 * t);
+            }
+            if (2 * t + 8 < r_pad) {
+              aa[2] = *reinterpret_cast<const uint32_t*>(aks + gid * r_pad + 2 * t + 8);
+              aa[3] = *reinterpret_cast<const uint32_t*>(aks + (gid + 8) * r_pad + 2 * t + 8);
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) mma16816(acc[1][nt], aa, bw[nt][0], bw[nt][1]);
+          }
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            const int h = t + 4 * nt;
+            if (h < HPu) {
 #pragma unroll
               for (int half = 0; half < 2; ++half) {
                 const int tok = slab * kSlab + gid + 8 * half;          // token inside the block
-                float v = acc[nt][2 * half] + acc[nt][2 * half + 1] + ch_own[nt];
-                if (k2k > 0 && h < HPu) {
-                  v = fmaf((float)corr_k[h * maxT + tok], Si, v);
+                float v = (acc[0][nt][2 * half] + acc[0][nt][2 * half + 1]) +
+                          (acc[1][nt][2 * half] + acc[1][nt][2 * half + 1]) + ch_own[nt];
+                if (k2k > 0) {
+                  v = fmaf((float)corr_k[h * maxT + tok], Si[nt], v);
                   corr_k[h * maxT + tok] = 0;
                 }
-                sc[nt][s][half] = (tok < valid_tokens && h < HPu) ? v : -INFINITY;
+                ps[h * maxT + tok] = tok < valid_tokens ? v : -INFINITY;
               }
             }
           }
         }
-        if (c == nchunk - 1) release();               // the key item is consumed
+      }
+      release();                                      // the key item is consumed
 
-        // ---------------- online softmax over the chunk: one rescale at most
+      // ---------------- online softmax over the block: one rescale at most
+      {
+        float alpha[HP];
         bool grew = false;
-        float m_new[NT];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          float mx = -INFINITY;
+        for (int h = 0; h < HP; ++h) {
+          alpha[h] = 1.f;
+          if (h < HPu) {
+            float* row = ps + h * maxT;
+            float mx = -INFINITY;
+            for (int tk = lane; tk < T; tk += 32) mx = fmaxf(mx, row[tk]);
 #pragma unroll
-          for (int s = 0; s < kChunkSlabs; ++s) mx = fmaxf(mx, fmaxf(sc[nt][s][0], sc[nt][s][1]));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-          m_new[nt] = fmaxf(m_run[nt], mx);
-          grew |= m_new[nt] > m_run[nt];
+            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            const float m_new = fmaxf(m_run[h], mx);       // finite: every block holds a valid token
+            if (m_new > m_run[h]) {
+              alpha[h] = exp2f(m_run[h] - m_new);
+              grew = true;
+              m_run[h] = m_new;
+            }
+            float l = 0.f;
+            for (int tk = lane; tk < T; tk += 32) {
+              const float p = exp2f(row[tk] - m_new);       // exp2(-inf) = 0 for masked tokens
+              l += p;
+              row[tk] = p;
+            }
+            l_run[h] = fmaf(l_run[h], alpha[h], l);
+          }
         }
-        if (__any_sync(0xffffffffu, grew)) {
+        if (grew) {                                      // warp-uniform: m_run is the same in every lane
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
-            const float al = (m_new[nt] == -INFINITY) ? 1.f : exp2f(m_run[nt] - m_new[nt]);
-            if (gid == 0) alpha_s[t + 4 * nt] = al;
-            l_run[nt] *= al;
+            float al = alpha[4 * nt];
+#pragma unroll
+            for (int hh = 1; hh < 4; ++hh)
+              if (4 * nt + hh < HP && t == hh) al = alpha[4 * nt + hh];
 #pragma unroll
             for (int i = 0; i < 4; ++i) U[nt][i] *= al;
 #pragma unroll
@@ -617,115 +642,97 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
 #pragma unroll
               for (int i = 0; i < 4; ++i) O[mt][nt][i] *= al;
           }
-          __syncwarp();
 #pragma unroll
           for (int h = 0; h < HP; ++h) {
             if (h < HPu) {
-              const float al = alpha_s[h];
 #pragma unroll
-              for (int g = 0; g < NGV; ++g) cm[h][g] *= al;
+              for (int g = 0; g < NGV; ++g) cm[h][g] *= alpha[h];
               float4* oc = reinterpret_cast<float4*>(ocorr + h * kHeadDim + lane * 4);
               float4 v = *oc;
-              v.x *= al; v.y *= al; v.z *= al; v.w *= al;
+              v.x *= alpha[h]; v.y *= alpha[h]; v.z *= alpha[h]; v.w *= alpha[h];
               *oc = v;
             }
           }
-          __syncwarp();
         }
+      }
+      __syncwarp();
+
+      // ================================================================ value item
+      unsigned char* stV = acquire();
+      if (!alive) break;
+      const unsigned char* vp = stV + a.bregion;          // value part of the record
+      const int o_av = is_buf ? 0 : sdc->off_av - sdc->off_vpart;
+      const int o_vsz = is_buf ? 0 : sdc->off_vscale - sdc->off_vpart;
+      uint32_t* fragV = frag;                                         // [NT][NGV][nslab] rows of kFragStride words
+      uint32_t* fragP = frag + NT * NGV * nslab * kFragStride;        // [NT][nslab]
+      if (is_buf && valid_tokens < kSlab) {
+        // rows past the end of the buffer hold stale bytes: clear them (0 * garbage must stay 0)
+        for (int i = lane; i < (kSlab - valid_tokens) * (kBufPitch / 16); i += 32) {
+          const int r = valid_tokens + i / (kBufPitch / 16), cc = i % (kBufPitch / 16);
+          reinterpret_cast<uint4*>(stV + r * kBufPitch)[cc] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_async_smem();
+      }
+
+      // ---------------- B operands of the value products: p * scale (per token and group) and p, split hi / lo;
+      //                  the zero-point term goes to the fp32 side sums cm
+      for (int pr = lane; pr < T / 2; pr += 32) {      // this lane's token pairs
+        const int s = pr >> 3, pi = pr & 7, tw = pi & 3, rg = pi >> 2;
+        const int tp = 2 * pr;
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          m_run[nt] = m_new[nt];
-          const int h = t + 4 * nt;
+        for (int h = 0; h < HP; ++h) {
+          if (h < HPu) {
+            const float2 pp = *reinterpret_cast<const float2*>(ps + h * maxT + tp);
+            const int col = 2 * (h & 3);
+            uint32_t hi, lo;
+            if (r_pad > 0 || is_buf) {
+              split_hi_lo(pp.x, pp.y, hi, lo);
+              uint32_t* bp = fragP + ((h >> 2) * nslab + s) * kFragStride + rg;
+              bp[(col * 4 + tw) * 2] = hi;
+              bp[((col + 1) * 4 + tw) * 2] = lo;
+            }
+            if (!is_buf) {
+              const __half2* vsz = reinterpret_cast<const __half2*>(vp + o_vsz) + tp * NGV;
 #pragma unroll
-          for (int s = 0; s < kChunkSlabs; ++s) {
-            if (s < ns) {
-#pragma unroll
-              for (int half = 0; half < 2; ++half) {
-                const float p = exp2f(sc[nt][s][half] - m_new[nt]);     // exp2(-inf) = 0 for masked tokens
-                l_run[nt] += p;
-                if (h < HPu) ps[h * kChunkTok + s * kSlab + gid + 8 * half] = p;
+              for (int g = 0; g < NGV; ++g) {
+                const __half2 z0 = vsz[g], z1 = vsz[NGV + g];
+                split_hi_lo(pp.x * __low2float(z0), pp.y * __low2float(z1), hi, lo);
+                uint32_t* bv = fragV + (((h >> 2) * NGV + g) * nslab + s) * kFragStride + rg;
+                bv[(col * 4 + tw) * 2] = hi;
+                bv[((col + 1) * 4 + tw) * 2] = lo;
+                cm[h][g] = fmaf(pp.x, __high2float(z0), fmaf(pp.y, __high2float(z1), cm[h][g]));
               }
             }
           }
         }
-        __syncwarp();
+      }
+      __syncwarp();
 
-        // ================================================================ value item
-        if (stV == nullptr) {
-          stV = acquire(item_k + 1);
-          if (!alive) break;
-          if (is_buf && valid_tokens < kSlab) {
-            // rows past the end of the buffer hold stale bytes: clear them (0 * garbage must stay 0)
-            for (int i = lane; i < (kSlab - valid_tokens) * (kBufPitch / 16); i += 32) {
-              const int r = valid_tokens + i / (kBufPitch / 16), cc = i % (kBufPitch / 16);
-              reinterpret_cast<uint4*>(stV + r * kBufPitch)[cc] = make_uint4(0u, 0u, 0u, 0u);
-            }
-            fence_async_smem();
-            __syncwarp();
-          }
-        }
-        const unsigned char* vp = stV + a.bregion - (is_buf ? 0 : sdc->off_vpart);   // record base seen from the value part
-        const int tok0c = c * kChunkTok;                                               // first token of the chunk
-
-        // ---------------- B operands of the value products: p * scale (per token and group) and p, split hi / lo;
-        //                  the zero-point term goes to the fp32 side sums cm
-        {
-          const int s = lane >> 3, pi = lane & 7;        // this lane's token pair of the chunk
-          const int tp = s * kSlab + 2 * pi;
-          const int tw = (pi & 3), rg = pi >> 2;
-          if (s < ns) {
-#pragma unroll
-            for (int h = 0; h < HP; ++h) {
-              if (h < HPu) {
-                const float2 pp = *reinterpret_cast<const float2*>(ps + h * kChunkTok + tp);
-                const int col = 2 * (h & 3);
-                uint32_t hi, lo;
-                if (r_pad > 0 || is_buf) {
-                  split_hi_lo(pp.x, pp.y, hi, lo);
-                  uint32_t* bp = fragP + ((h >> 2) * kChunkSlabs + s) * kFragStride + rg;
-                  bp[(col * 4 + tw) * 2] = hi;
-                  bp[((col + 1) * 4 + tw) * 2] = lo;
-                }
-                if (!is_buf) {
-                  const __half2* vsz = reinterpret_cast<const __half2*>(vp + sdc->off_vscale) + (size_t)(tok0c + tp) * NGV;
-#pragma unroll
-                  for (int g = 0; g < NGV; ++g) {
-                    const __half2 z0 = vsz[g], z1 = vsz[NGV + g];
-                    split_hi_lo(pp.x * __low2float(z0), pp.y * __low2float(z1), hi, lo);
-                    uint32_t* bv = fragV + (((h >> 2) * NGV + g) * kChunkSlabs + s) * kFragStride + rg;
-                    bv[(col * 4 + tw) * 2] = hi;
-                    bv[((col + 1) * 4 + tw) * 2] = lo;
-                    cm[h][g] = fmaf(pp.x, __high2float(z0), fmaf(pp.y, __high2float(z1), cm[h][g]));
-                  }
-                }
-              }
-            }
-          }
-        }
-        __syncwarp();
-
-        // ---------------- values: out += sum_tok (p * scale) * code on the tensor cores, low rank on the side
+      // ---------------- values: out += sum_tok (p * scale) * code on the tensor cores, low rank on the side
+      {
+        const uint4* cw = reinterpret_cast<const uint4*>(vp) + lane;
+        const __half* avb = reinterpret_cast<const __half*>(vp + o_av);
 #pragma unroll 1
-        for (int s = 0; s < ns; ++s) {
-          const int slab = c * kChunkSlabs + s;
+        for (int slab = 0; slab < nslab; ++slab) {
           uint32_t bp[NT][2];
+          if (r_pad > 0 || is_buf) {
 #pragma unroll
-          for (int nt = 0; nt < NT; ++nt) {
-            const uint2 v = *reinterpret_cast<const uint2*>(fragP + (nt * kChunkSlabs + s) * kFragStride + lane * 2);
-            bp[nt][0] = v.x; bp[nt][1] = v.y;
+            for (int nt = 0; nt < NT; ++nt) {
+              const uint2 v = *reinterpret_cast<const uint2*>(fragP + (nt * nslab + slab) * kFragStride + lane * 2);
+              bp[nt][0] = v.x; bp[nt][1] = v.y;
+            }
           }
           if (!is_buf) {
-            const uint4* cw = reinterpret_cast<const uint4*>(vp + sdc->off_vcodes + slab * sdc->slab_codes);
             uint32_t bv[NT][NGV][2];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
               for (int g = 0; g < NGV; ++g) {
-                const uint2 v = *reinterpret_cast<const uint2*>(fragV + ((nt * NGV + g) * kChunkSlabs + s) * kFragStride + lane * 2);
+                const uint2 v = *reinterpret_cast<const uint2*>(fragV + ((nt * NGV + g) * nslab + slab) * kFragStride + lane * 2);
                 bv[nt][g][0] = v.x; bv[nt][g][1] = v.y;
               }
             if (BITS == 2) {
-              const uint4 w = cw[lane];
+              const uint4 w = cw[slab * SLABW];
               const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
               for (int q4 = 0; q4 < 4; ++q4) {
@@ -742,7 +749,7 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
             } else {
 #pragma unroll
               for (int pl = 0; pl < 2; ++pl) {
-                const uint4 w = cw[pl * 32 + lane];
+                const uint4 w = cw[slab * SLABW + pl * 32];
                 const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
@@ -755,7 +762,7 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
               }
             }
             if (r_pad > 0) {                          // low-rank value term, first product: U = A_V^T p
-              const __half* avs = reinterpret_cast<const __half*>(vp + sdc->off_av + slab * slab_a);
+              const __half* avs = avb + slab * (slab_a / 2);
               uint32_t aa[4] = {0u, 0u, 0u, 0u};
               if (gid < r_pad) {
                 aa[0] = *reinterpret_cast<const uint32_t*>(avs + gid * kSlab + 2 * t);
@@ -767,7 +774,6 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
               }
 #pragma unroll
               for (int nt = 0; nt < NT; ++nt) mma16816(U[nt], aa, bp[nt][0], bp[nt][1]);
-              u_pending = true;
             }
           } else {
 #pragma unroll
@@ -779,68 +785,68 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
             }
           }
         }
+        if (!is_buf && r_pad > 0) u_pending = true;
+      }
 
-        // ---------------- sparse value term: p[tok] * (x - zero[tok, g]) scattered to the outlier's channel
-        if (!is_buf && a.cc.k_v > 0) {
-          const int k2v = 2 * a.cc.k_v;
-          const int sexp = clamp60(21 - float_exponent(dmax_v));
-          const float S = pow2i(sexp), Si = pow2i(-sexp);
-          const __half2* vsz = reinterpret_cast<const __half2*>(vp + sdc->off_vscale);
-          for (int tk = lane; tk < ns * kSlab; tk += 32) {
-            const int tb = tok0c + tk;
-            float pS[HP];
+      // ---------------- sparse value term: p[tok] * (x - zero[tok, g]) scattered to the outlier's channel
+      if (!is_buf && a.cc.k_v > 0) {
+        const int k2v = 2 * a.cc.k_v;
+        const int sexp = clamp60(21 - float_exponent(dmax_v));
+        const float S = pow2i(sexp), Si = pow2i(-sexp);
+        const __half2* vsz = reinterpret_cast<const __half2*>(vp + o_vsz);
+        const unsigned char* voval = vp + (sdc->off_voval - sdc->off_vpart);
+        const unsigned char* voidx = vp + (sdc->off_voidx - sdc->off_vpart);
+        for (int tk = lane; tk < T; tk += 32) {
+          float pS[HP];
 #pragma unroll
-            for (int h = 0; h < HP; ++h) pS[h] = h < HPu ? ps[h * kChunkTok + tk] * S : 0.f;
-            auto v_entry = [&](int g, float val, int idx) {
-              const float d = val - __high2float(vsz[tb * NGV + g]);
-              const int ch = g * GV + idx;
+          for (int h = 0; h < HP; ++h) pS[h] = h < HPu ? ps[h * maxT + tk] * S : 0.f;
+          auto v_entry = [&](int g, float val, int idx) {
+            const float d = val - __high2float(vsz[tk * NGV + g]);
+            const int ch = g * GV + idx;
 #pragma unroll
-              for (int h = 0; h < HP; ++h)
-                if (h < HPu) atomicAdd(&corr_v[h * kHeadDim + ch], __float2int_rn(pS[h] * d));
-            };
-            if (NGV * k2v == 4) {
-              const uint2 ov = reinterpret_cast<const uint2*>(vp + sdc->off_voval)[tb];
-              const uint32_t oi = reinterpret_cast<const uint32_t*>(vp + sdc->off_voidx)[tb];
-              v_entry(0, __low2float(u32_as_h2(ov.x)), oi & 0xFFu);
-              v_entry(NGV == 2 ? 0 : (NGV == 4 ? 1 : 0), __high2float(u32_as_h2(ov.x)), (oi >> 8) & 0xFFu);
-              v_entry(NGV == 2 ? 1 : (NGV == 4 ? 2 : 0), __low2float(u32_as_h2(ov.y)), (oi >> 16) & 0xFFu);
-              v_entry(NGV == 2 ? 1 : (NGV == 4 ? 3 : 0), __high2float(u32_as_h2(ov.y)), oi >> 24);
-            } else {
-              const __half* ov = reinterpret_cast<const __half*>(vp + sdc->off_voval) + (size_t)tb * NGV * k2v;
-              const unsigned char* oi = vp + sdc->off_voidx + (size_t)tb * NGV * k2v;
+            for (int h = 0; h < HP; ++h)
+              if (h < HPu) atomicAdd(&corr_v[h * kHeadDim + ch], __float2int_rn(pS[h] * d));
+          };
+          if (NGV * k2v == 4) {
+            const uint2 ov = reinterpret_cast<const uint2*>(voval)[tk];
+            const uint32_t oi = reinterpret_cast<const uint32_t*>(voidx)[tk];
+            v_entry(0, __low2float(u32_as_h2(ov.x)), oi & 0xFFu);
+            v_entry(0, __high2float(u32_as_h2(ov.x)), (oi >> 8) & 0xFFu);
+            v_entry(NGV == 2 ? 1 : 0, __low2float(u32_as_h2(ov.y)), (oi >> 16) & 0xFFu);
+            v_entry(NGV == 2 ? 1 : 0, __high2float(u32_as_h2(ov.y)), oi >> 24);
+          } else {
+            const __half* ov = reinterpret_cast<const __half*>(voval) + (size_t)tk * NGV * k2v;
+            const unsigned char* oi = voidx + (size_t)tk * NGV * k2v;
 #pragma unroll
-              for (int g = 0; g < NGV; ++g)
-                for (int e = 0; e < k2v; ++e) v_entry(g, __half2float(ov[g * k2v + e]), oi[g * k2v + e]);
-            }
-          }
-          __syncwarp();
-#pragma unroll
-          for (int h = 0; h < HP; ++h) {
-            if (h < HPu) {
-              int4* cv = reinterpret_cast<int4*>(corr_v + h * kHeadDim) + lane;
-              float4* oc = reinterpret_cast<float4*>(ocorr + h * kHeadDim) + lane;
-              const int4 v = *cv;
-              *cv = make_int4(0, 0, 0, 0);
-              float4 o = *oc;
-              o.x = fmaf((float)v.x, Si, o.x);
-              o.y = fmaf((float)v.y, Si, o.y);
-              o.z = fmaf((float)v.z, Si, o.z);
-              o.w = fmaf((float)v.w, Si, o.w);
-              *oc = o;
-            }
+            for (int g = 0; g < NGV; ++g)
+              for (int e = 0; e < k2v; ++e) v_entry(g, __half2float(ov[g * k2v + e]), oi[g * k2v + e]);
           }
         }
-        __syncwarp();                                 // ps and the fragments are rewritten by the next chunk
+        __syncwarp();
+#pragma unroll
+        for (int h = 0; h < HP; ++h) {
+          if (h < HPu) {
+            int4* cv = reinterpret_cast<int4*>(corr_v + h * kHeadDim) + lane;
+            float4* oc = reinterpret_cast<float4*>(ocorr + h * kHeadDim) + lane;
+            const int4 v = *cv;
+            *cv = make_int4(0, 0, 0, 0);
+            float4 o = *oc;
+            o.x = fmaf((float)v.x, Si, o.x);
+            o.y = fmaf((float)v.y, Si, o.y);
+            o.z = fmaf((float)v.z, Si, o.z);
+            o.w = fmaf((float)v.w, Si, o.w);
+            *oc = o;
+          }
+        }
       }
-      if (!alive) break;
 
       // ---------------- end of a segment (or of this warp's share of it): out += B_V U
       if (with_bv && u_pending) {
         __syncwarp();
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          wl[gid * HP + t + 4 * nt] = U[nt][0] + U[nt][1];
-          wl[(gid + 8) * HP + t + 4 * nt] = U[nt][2] + U[nt][3];
+          wl[gid * 8 + t + 4 * nt] = U[nt][0] + U[nt][1];
+          wl[(gid + 8) * 8 + t + 4 * nt] = U[nt][2] + U[nt][3];
 #pragma unroll
           for (int i = 0; i < 4; ++i) U[nt][i] = 0.f;
         }
@@ -850,8 +856,8 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
         for (int nt = 0; nt < NT; ++nt) {
           const int h = (gid >> 1) + 4 * nt;
           uint32_t hi0, lo0, hi1, lo1;
-          split_hi_lo(wl[(2 * t) * HP + h], wl[(2 * t + 1) * HP + h], hi0, lo0);
-          split_hi_lo(wl[(2 * t + 8) * HP + h], wl[(2 * t + 9) * HP + h], hi1, lo1);
+          split_hi_lo(wl[(2 * t) * 8 + h], wl[(2 * t + 1) * 8 + h], hi0, lo0);
+          split_hi_lo(wl[(2 * t + 8) * 8 + h], wl[(2 * t + 9) * 8 + h], hi1, lo1);
           bu[nt][0] = (gid & 1) ? lo0 : hi0;
           bu[nt][1] = (gid & 1) ? lo1 : hi1;
         }
@@ -874,30 +880,30 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
         u_pending = false;
       }
       release();                                      // the value item is consumed
-      item_k += 2;
     }
     if (!alive) break;
 
     // ---------------- partial result of this unit: (m, l, o) per head
+    const long long F = (long long)a.cc.BH * passes * NB, NW = gridDim.x;
     const long long bflat = (long long)u * NB, eflat = bflat + NB;
     const long long w_first = ((bflat + 1) * NW + F - 1) / F - 1;
     const long long w_last = (eflat * NW + F - 1) / F - 1;
     const int n_parts = (int)(w_last - w_first + 1);
-    const int slot = (int)(gw - w_first);
+    const int slot = (int)(blockIdx.x - w_first);
     float* part_base = a.partial + ((size_t)u * a.max_parts + slot) * (HP * 130);
-    float cm_own[NT][NGV];
+    float cm_own[NT][NGV], m_own[NT], l_own[NT];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      float l = l_run[nt];
-      l += __shfl_xor_sync(0xffffffffu, l, 4);
-      l += __shfl_xor_sync(0xffffffffu, l, 8);
-      l += __shfl_xor_sync(0xffffffffu, l, 16);
-      l_run[nt] = l;
+      m_own[nt] = 0.f; l_own[nt] = 0.f;
 #pragma unroll
       for (int g = 0; g < NGV; ++g) cm_own[nt][g] = 0.f;
     }
 #pragma unroll
-    for (int h = 0; h < HP; ++h)
+    for (int h = 0; h < HP; ++h) {
+      float l = l_run[h];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+      if ((h & 3) == t) { m_own[h >> 2] = m_run[h]; l_own[h >> 2] = l; }
 #pragma unroll
       for (int g = 0; g < NGV; ++g) {
         float c = cm[h][g];
@@ -905,6 +911,7 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
         for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
         if ((h & 3) == t) cm_own[h >> 2][g] = c;
       }
+    }
     __syncwarp();
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -918,7 +925,7 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
             const int ch = 16 * mt + gid + 8 * half;
             dst[ch] = O[mt][nt][2 * half] + O[mt][nt][2 * half + 1] + ocorr[h * kHeadDim + ch] + cm_own[nt][(mt * 16) / GV];
           }
-        if (gid == 0) { dst[128] = m_run[nt]; dst[129] = l_run[nt]; }
+        if (gid == 0) { dst[128] = m_own[nt]; dst[129] = l_own[nt]; }
       }
     }
     __threadfence();
@@ -950,13 +957,15 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
       }
       if (lane == 0) a.tickets[u] = 0;
     }
-    f += blk_hi - blk_lo;
+    n_left -= blk_hi - blk_lo;
+    blk_lo = 0;
+    ++u;
   }
   // a warp that gave up still has copies in flight: let them land (bounded) before leaving
   if (!alive) {
-    for (int i = n_released; i < n_issued; ++i) {
-      const int s = i % NS;
-      for (int k = 0; k < kSpinLimit && !mbar_try(&bar[s], (uint32_t)((i / NS) & 1)); ++k) {}
+    for (int i = 0; i < n_inflight; ++i) {
+      for (int k = 0; k < kSpinLimit && !mbar_try(&bar[c_stage], (uint32_t)c_par); ++k) {}
+      if (++c_stage == NS) { c_stage = 0; c_par ^= 1; }
     }
   }
 }
@@ -964,13 +973,13 @@ __global__ void __launch_bounds__(32, NT == 1 ? 10 : 5) gear_decode_kernel(const
 // ------------------------------------------------------------------ host side
 template <class Fn>
 static bool with_decode_kernel(int bits, int heads, int ngv, Fn fn) {
-  const int nt = heads <= 4 ? 1 : 2;
+  const int hp = heads == 1 ? 1 : (heads <= 4 ? 4 : 8);
 #define GEAR_DEC_CASE(B, N, V) \
-  if (bits == B && nt == N && ngv == V) { fn(gear_decode_kernel<B, N, V>); return true; }
-  GEAR_DEC_CASE(2, 1, 1) GEAR_DEC_CASE(2, 1, 2) GEAR_DEC_CASE(2, 1, 4) GEAR_DEC_CASE(2, 1, 8)
-  GEAR_DEC_CASE(2, 2, 1) GEAR_DEC_CASE(2, 2, 2) GEAR_DEC_CASE(2, 2, 4) GEAR_DEC_CASE(2, 2, 8)
-  GEAR_DEC_CASE(4, 1, 1) GEAR_DEC_CASE(4, 1, 2) GEAR_DEC_CASE(4, 1, 4) GEAR_DEC_CASE(4, 1, 8)
-  GEAR_DEC_CASE(4, 2, 1) GEAR_DEC_CASE(4, 2, 2) GEAR_DEC_CASE(4, 2, 4) GEAR_DEC_CASE(4, 2, 8)
+  if (bits == B && hp == N && ngv == V) { fn(gear_decode_kernel<B, N, V>); return true; }
+#define GEAR_DEC_HEADS(B, V) GEAR_DEC_CASE(B, 1, V) GEAR_DEC_CASE(B, 4, V) GEAR_DEC_CASE(B, 8, V)
+  GEAR_DEC_HEADS(2, 1) GEAR_DEC_HEADS(2, 2) GEAR_DEC_HEADS(2, 4) GEAR_DEC_HEADS(2, 8)
+  GEAR_DEC_HEADS(4, 1) GEAR_DEC_HEADS(4, 2) GEAR_DEC_HEADS(4, 4) GEAR_DEC_HEADS(4, 8)
+#undef GEAR_DEC_HEADS
 #undef GEAR_DEC_CASE
   return false;
 }
