@@ -24,6 +24,8 @@
 #include <cuda_runtime.h>
 #include <math.h>
 
+#include <type_traits>
+
 #include "gear_internal.cuh"
 
 namespace gear {
@@ -60,6 +62,7 @@ __device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
 }
 // Bounded wait: gives up after kSpinLimit polls and reports through `status`.
 __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, int* status) {
+#pragma unroll 1
   for (int i = 0; i < kSpinLimit; ++i)
     if (mbar_try(b, parity)) return true;
   atomicExch(status, -7 /* GEAR_ERR_TIMEOUT */);
@@ -92,29 +95,32 @@ __device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_c
 
 // (x & mask) | 0x6400 puts each masked field into the mantissa of 1024.0; one
 // half2 fma with exact constants brings it back to the integer code.
-__device__ __forceinline__ uint32_t field_to_h2(uint32_t x, uint32_t mask, float inv_step, float offs) {
-  const __half2 h = u32_as_h2(lop3_and_or(x, mask, 0x64006400u));
-  return h2_as_u32(__hfma2(h, __float2half2_rn(inv_step), __float2half2_rn(offs)));
+// `mul`, `add`: half2 bit patterns of the constants.
+__device__ __forceinline__ uint32_t field_to_h2(uint32_t x, uint32_t mask, uint32_t mul, uint32_t add) {
+  uint32_t r;
+  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(lop3_and_or(x, mask, 0x64006400u)), "r"(mul), "r"(add));
+  return r;
 }
 // One 32-bit word of codes -> its fragment registers r[0 .. 16/BITS).
 template <int BITS>
 __device__ __forceinline__ void unpack_word(uint32_t x, uint32_t* r) {
   if (BITS == 2) {
+    // (1, -1024), (1/4, -256), (1/16, -64), (1/64, -16), (1/256, -4) as half2
     const uint32_t y = x >> 10;
-    r[0] = field_to_h2(x, 0x00030003u, 1.0f, -1024.0f);
-    r[1] = field_to_h2(x, 0x000C000Cu, 0.25f, -256.0f);
-    r[2] = field_to_h2(x, 0x00300030u, 0.0625f, -64.0f);
-    r[3] = field_to_h2(x, 0x00C000C0u, 0.015625f, -16.0f);
-    r[4] = field_to_h2(x, 0x03000300u, 0.00390625f, -4.0f);
-    r[5] = field_to_h2(y, 0x00030003u, 1.0f, -1024.0f);
-    r[6] = field_to_h2(y, 0x000C000Cu, 0.25f, -256.0f);
-    r[7] = field_to_h2(y, 0x00300030u, 0.0625f, -64.0f);
+    r[0] = field_to_h2(x, 0x00030003u, 0x3C003C00u, 0xE400E400u);
+    r[1] = field_to_h2(x, 0x000C000Cu, 0x34003400u, 0xDC00DC00u);
+    r[2] = field_to_h2(x, 0x00300030u, 0x2C002C00u, 0xD400D400u);
+    r[3] = field_to_h2(x, 0x00C000C0u, 0x24002400u, 0xCC00CC00u);
+    r[4] = field_to_h2(x, 0x03000300u, 0x1C001C00u, 0xC400C400u);
+    r[5] = field_to_h2(y, 0x00030003u, 0x3C003C00u, 0xE400E400u);
+    r[6] = field_to_h2(y, 0x000C000Cu, 0x34003400u, 0xDC00DC00u);
+    r[7] = field_to_h2(y, 0x00300030u, 0x2C002C00u, 0xD400D400u);
   } else {
     const uint32_t y = x >> 8;
-    r[0] = field_to_h2(x, 0x000F000Fu, 1.0f, -1024.0f);
-    r[1] = field_to_h2(x, 0x00F000F0u, 0.0625f, -64.0f);
-    r[2] = field_to_h2(y, 0x000F000Fu, 1.0f, -1024.0f);
-    r[3] = field_to_h2(y, 0x00F000F0u, 0.0625f, -64.0f);
+    r[0] = field_to_h2(x, 0x000F000Fu, 0x3C003C00u, 0xE400E400u);
+    r[1] = field_to_h2(x, 0x00F000F0u, 0x2C002C00u, 0xD400D400u);
+    r[2] = field_to_h2(y, 0x000F000Fu, 0x3C003C00u, 0xE400E400u);
+    r[3] = field_to_h2(y, 0x00F000F0u, 0x2C002C00u, 0xD400D400u);
   }
 }
 
@@ -493,6 +499,7 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
             const unsigned char* oi = kp + sdc->off_koidx + lane * 4 * k2k;
 #pragma unroll
             for (int j = 0; j < 4; ++j)
+#pragma unroll 1
               for (int e = 0; e < k2k; ++e) k_entry(j, __half2float(ov[j * k2k + e]), oi[j * k2k + e]);
           }
         }
@@ -509,94 +516,103 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
 
       // ---------------- key scores, slab by slab; scores go to shared memory
       {
-        const uint4* cw = reinterpret_cast<const uint4*>(kp + (is_buf ? 0 : sdc->off_kcodes)) + lane;
-        const __half* ak = reinterpret_cast<const __half*>(kp + (is_buf ? 0 : sdc->off_ak));
         float Si[NT];
+        int psoff[NT];                                  // this lane's first score slot (head t + 4 nt, token gid)
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) Si[nt] = pow2i(-own_sexp[nt]);
+        for (int nt = 0; nt < NT; ++nt) { Si[nt] = pow2i(-own_sexp[nt]); psoff[nt] = (t + 4 * nt) * maxT + gid; }
+        const bool pa0 = 2 * t < r_pad, pa1 = 2 * t + 8 < r_pad;
+        const bool has_ko = k2k > 0;
+        auto k_slabs = [&](auto buf_tag) {
+          constexpr bool kBuf = decltype(buf_tag)::value;
+          const uint4* cwp = reinterpret_cast<const uint4*>(kp + (kBuf ? 0 : sdc->off_kcodes)) + lane;
+          const __half* akp = reinterpret_cast<const __half*>(kp + (kBuf ? 0 : sdc->off_ak)) + gid * r_pad + 2 * t;
+          const int ak8 = 8 * r_pad, ak_step = kSlab * r_pad;
+          int tok0 = 0;
 #pragma unroll 1
-        for (int slab = 0; slab < nslab; ++slab) {
-          float acc[2][NT][4];
+          for (int slab = 0; slab < nslab; ++slab) {
+            float acc[2][NT][4];
 #pragma unroll
-          for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-              for (int i = 0; i < 4; ++i) acc[hf][nt][i] = 0.f;
-          uint4 w0 = make_uint4(0u, 0u, 0u, 0u), w1 = w0;
-          if (!is_buf) {
-            w0 = cw[slab * SLABW];
-            if (BITS == 4) w1 = cw[slab * SLABW + 32];
-          }
-#pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {            // channel chunks 4 hf .. 4 hf + 3
-            uint32_t af[4][4];
-            if (!is_buf) {
-              if (BITS == 2) {
-                uint32_t r[8];
-                unpack_word<2>(hf == 0 ? w0.x : w0.y, r);
-#pragma unroll
-                for (int u2 = 0; u2 < 8; ++u2) af[u2 >> 1][(u2 & 1) * 2] = r[u2];
-                unpack_word<2>(hf == 0 ? w0.z : w0.w, r);
-#pragma unroll
-                for (int u2 = 0; u2 < 8; ++u2) af[u2 >> 1][(u2 & 1) * 2 + 1] = r[u2];
-              } else {
-#pragma unroll
-                for (int th = 0; th < 2; ++th) {
-                  const uint4 w = th == 0 ? w0 : w1;
-                  uint32_t r[4];
-                  unpack_word<4>(hf == 0 ? w.x : w.z, r);
-#pragma unroll
-                  for (int u2 = 0; u2 < 4; ++u2) af[u2 >> 1][(u2 & 1) * 2 + th] = r[u2];
-                  unpack_word<4>(hf == 0 ? w.y : w.w, r);
-#pragma unroll
-                  for (int u2 = 0; u2 < 4; ++u2) af[2 + (u2 >> 1)][(u2 & 1) * 2 + th] = r[u2];
-                }
-              }
-            } else {
-#pragma unroll
-              for (int k4 = 0; k4 < 4; ++k4)
-                ldmatrix_x4(af[k4], stK + ((lane & 7) + 8 * ((lane >> 3) & 1)) * kBufPitch +
-                                        (16 * (4 * hf + k4) + 8 * (lane >> 4)) * 2);
-            }
-#pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4)
+            for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
               for (int nt = 0; nt < NT; ++nt)
-                mma16816(acc[hf][nt], af[k4], bq[nt][4 * hf + k4][0], bq[nt][4 * hf + k4][1]);
-          }
-          if (r_pad > 0) {                          // low-rank key term: A_K rows times w
-            const __half* aks = ak + slab * (slab_a / 2);
-            uint32_t aa[4] = {0u, 0u, 0u, 0u};
-            if (2 * t < r_pad) {
-              aa[0] = *reinterpret_cast<const uint32_t*>(aks + gid * r_pad + 2 * t);
-              aa[1] = *reinterpret_cast<const uint32_t*>(aks + (gid + 8) * r_pad + 2 * t);
-            }
-            if (2 * t + 8 < r_pad) {
-              aa[2] = *reinterpret_cast<const uint32_t*>(aks + gid * r_pad + 2 * t + 8);
-              aa[3] = *reinterpret_cast<const uint32_t*>(aks + (gid + 8) * r_pad + 2 * t + 8);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[hf][nt][i] = 0.f;
+            uint4 w0 = make_uint4(0u, 0u, 0u, 0u), w1 = w0;
+            if (!kBuf) {
+              w0 = cwp[0];
+              if (BITS == 4) w1 = cwp[32];
+              cwp += SLABW;
             }
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) mma16816(acc[1][nt], aa, bw[nt][0], bw[nt][1]);
-          }
+            for (int hf = 0; hf < 2; ++hf) {            // channel chunks 4 hf .. 4 hf + 3
+              uint32_t af[4][4];
+              if (!kBuf) {
+                if (BITS == 2) {
+                  uint32_t r[8];
+                  unpack_word<2>(hf == 0 ? w0.x : w0.y, r);
 #pragma unroll
-          for (int nt = 0; nt < NT; ++nt) {
-            const int h = t + 4 * nt;
-            if (h < HPu) {
+                  for (int u2 = 0; u2 < 8; ++u2) af[u2 >> 1][(u2 & 1) * 2] = r[u2];
+                  unpack_word<2>(hf == 0 ? w0.z : w0.w, r);
 #pragma unroll
-              for (int half = 0; half < 2; ++half) {
-                const int tok = slab * kSlab + gid + 8 * half;          // token inside the block
-                float v = (acc[0][nt][2 * half] + acc[0][nt][2 * half + 1]) +
-                          (acc[1][nt][2 * half] + acc[1][nt][2 * half + 1]) + ch_own[nt];
-                if (k2k > 0) {
-                  v = fmaf((float)corr_k[h * maxT + tok], Si[nt], v);
-                  corr_k[h * maxT + tok] = 0;
+                  for (int u2 = 0; u2 < 8; ++u2) af[u2 >> 1][(u2 & 1) * 2 + 1] = r[u2];
+                } else {
+#pragma unroll
+                  for (int th = 0; th < 2; ++th) {
+                    const uint4 w = th == 0 ? w0 : w1;
+                    uint32_t r[4];
+                    unpack_word<4>(hf == 0 ? w.x : w.z, r);
+#pragma unroll
+                    for (int u2 = 0; u2 < 4; ++u2) af[u2 >> 1][(u2 & 1) * 2 + th] = r[u2];
+                    unpack_word<4>(hf == 0 ? w.y : w.w, r);
+#pragma unroll
+                    for (int u2 = 0; u2 < 4; ++u2) af[2 + (u2 >> 1)][(u2 & 1) * 2 + th] = r[u2];
+                  }
                 }
-                ps[h * maxT + tok] = tok < valid_tokens ? v : -INFINITY;
+              } else {
+#pragma unroll
+                for (int k4 = 0; k4 < 4; ++k4)
+                  ldmatrix_x4(af[k4], stK + ((lane & 7) + 8 * ((lane >> 3) & 1)) * kBufPitch +
+                                          (16 * (4 * hf + k4) + 8 * (lane >> 4)) * 2);
+              }
+#pragma unroll
+              for (int k4 = 0; k4 < 4; ++k4)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+                  mma16816(acc[hf][nt], af[k4], bq[nt][4 * hf + k4][0], bq[nt][4 * hf + k4][1]);
+            }
+            if (!kBuf) {                                // low-rank key term: A_K rows times w (zero rows when r = 0)
+              uint32_t aa[4] = {0u, 0u, 0u, 0u};
+              if (pa0) {
+                aa[0] = *reinterpret_cast<const uint32_t*>(akp);
+                aa[1] = *reinterpret_cast<const uint32_t*>(akp + ak8);
+              }
+              if (pa1) {
+                aa[2] = *reinterpret_cast<const uint32_t*>(akp + 8);
+                aa[3] = *reinterpret_cast<const uint32_t*>(akp + ak8 + 8);
+              }
+              akp += ak_step;
+#pragma unroll
+              for (int nt = 0; nt < NT; ++nt) mma16816(acc[1][nt], aa, bw[nt][0], bw[nt][1]);
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              if (t + 4 * nt < HPu) {
+                float v0 = (acc[0][nt][0] + acc[0][nt][1]) + (acc[1][nt][0] + acc[1][nt][1]) + ch_own[nt];
+                float v1 = (acc[0][nt][2] + acc[0][nt][3]) + (acc[1][nt][2] + acc[1][nt][3]) + ch_own[nt];
+                if (!kBuf && has_ko) {
+                  int* ck = corr_k + psoff[nt] + tok0;
+                  v0 = fmaf((float)ck[0], Si[nt], v0);
+                  v1 = fmaf((float)ck[8], Si[nt], v1);
+                  ck[0] = 0; ck[8] = 0;
+                }
+                float* pr = ps + psoff[nt] + tok0;
+                pr[0] = v0; pr[8] = v1;
               }
             }
+            tok0 += kSlab;
           }
-        }
+        };
+        if (is_buf) k_slabs(std::true_type{}); else k_slabs(std::false_type{});
       }
       release();                                      // the key item is consumed
 
@@ -610,7 +626,8 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
           if (h < HPu) {
             float* row = ps + h * maxT;
             float mx = -INFINITY;
-            for (int tk = lane; tk < T; tk += 32) mx = fmaxf(mx, row[tk]);
+#pragma unroll 1
+            for (int tk = lane; tk < valid_tokens; tk += 32) mx = fmaxf(mx, row[tk]);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             const float m_new = fmaxf(m_run[h], mx);       // finite: every block holds a valid token
@@ -620,8 +637,9 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
               m_run[h] = m_new;
             }
             float l = 0.f;
+#pragma unroll 1
             for (int tk = lane; tk < T; tk += 32) {
-              const float p = exp2f(row[tk] - m_new);       // exp2(-inf) = 0 for masked tokens
+              const float p = tk < valid_tokens ? exp2f(row[tk] - m_new) : 0.f;   // tokens past the end of the buffer
               l += p;
               row[tk] = p;
             }
@@ -676,6 +694,7 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
 
       // ---------------- B operands of the value products: p * scale (per token and group) and p, split hi / lo;
       //                  the zero-point term goes to the fp32 side sums cm
+#pragma unroll 1
       for (int pr = lane; pr < T / 2; pr += 32) {      // this lane's token pairs
         const int s = pr >> 3, pi = pr & 7, tw = pi & 3, rg = pi >> 2;
         const int tp = 2 * pr;
@@ -685,7 +704,7 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
             const float2 pp = *reinterpret_cast<const float2*>(ps + h * maxT + tp);
             const int col = 2 * (h & 3);
             uint32_t hi, lo;
-            if (r_pad > 0 || is_buf) {
+            {
               split_hi_lo(pp.x, pp.y, hi, lo);
               uint32_t* bp = fragP + ((h >> 2) * nslab + s) * kFragStride + rg;
               bp[(col * 4 + tw) * 2] = hi;
@@ -710,81 +729,89 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
 
       // ---------------- values: out += sum_tok (p * scale) * code on the tensor cores, low rank on the side
       {
-        const uint4* cw = reinterpret_cast<const uint4*>(vp) + lane;
-        const __half* avb = reinterpret_cast<const __half*>(vp + o_av);
+        const bool pv0 = gid < r_pad, pv1 = gid + 8 < r_pad;
+        auto v_slabs = [&](auto buf_tag) {
+          constexpr bool kBuf = decltype(buf_tag)::value;
+          const uint4* cwp = reinterpret_cast<const uint4*>(vp) + lane;
+          const __half* avp = reinterpret_cast<const __half*>(vp + o_av) + gid * kSlab + 2 * t;
+          const uint32_t* fvp = fragV + lane * 2;
+          const uint32_t* fpp = fragP + lane * 2;
+          const int fstep = nslab * kFragStride, av_step = kSlab * r_pad;
 #pragma unroll 1
-        for (int slab = 0; slab < nslab; ++slab) {
-          uint32_t bp[NT][2];
-          if (r_pad > 0 || is_buf) {
+          for (int slab = 0; slab < nslab; ++slab) {
+            uint32_t bp[NT][2];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-              const uint2 v = *reinterpret_cast<const uint2*>(fragP + (nt * nslab + slab) * kFragStride + lane * 2);
+              const uint2 v = *reinterpret_cast<const uint2*>(fpp + nt * fstep);
               bp[nt][0] = v.x; bp[nt][1] = v.y;
             }
-          }
-          if (!is_buf) {
-            uint32_t bv[NT][NGV][2];
+            fpp += kFragStride;
+            if (!kBuf) {
+              uint32_t bv[NT][NGV][2];
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
+              for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-              for (int g = 0; g < NGV; ++g) {
-                const uint2 v = *reinterpret_cast<const uint2*>(fragV + ((nt * NGV + g) * nslab + slab) * kFragStride + lane * 2);
-                bv[nt][g][0] = v.x; bv[nt][g][1] = v.y;
-              }
-            if (BITS == 2) {
-              const uint4 w = cw[slab * SLABW];
-              const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-              for (int q4 = 0; q4 < 4; ++q4) {
-                uint32_t r[8];
-                unpack_word<2>(wv[q4], r);
-#pragma unroll
-                for (int m2 = 0; m2 < 2; ++m2) {
-                  const int mt = 2 * q4 + m2, g = (mt * 16) / GV;
-                  const uint32_t av[4] = {r[4 * m2], r[4 * m2 + 1], r[4 * m2 + 2], r[4 * m2 + 3]};
-#pragma unroll
-                  for (int nt = 0; nt < NT; ++nt) mma16816(O[mt][nt], av, bv[nt][g][0], bv[nt][g][1]);
+                for (int g = 0; g < NGV; ++g) {
+                  const uint2 v = *reinterpret_cast<const uint2*>(fvp + (nt * NGV + g) * fstep);
+                  bv[nt][g][0] = v.x; bv[nt][g][1] = v.y;
                 }
-              }
-            } else {
-#pragma unroll
-              for (int pl = 0; pl < 2; ++pl) {
-                const uint4 w = cw[slab * SLABW + pl * 32];
+              fvp += kFragStride;
+              if (BITS == 2) {
+                const uint4 w = cwp[0];
                 const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
-                  const int mt = 4 * pl + q4, g = (mt * 16) / GV;
-                  uint32_t av[4];
-                  unpack_word<4>(wv[q4], av);
+                  uint32_t r[8];
+                  unpack_word<2>(wv[q4], r);
 #pragma unroll
-                  for (int nt = 0; nt < NT; ++nt) mma16816(O[mt][nt], av, bv[nt][g][0], bv[nt][g][1]);
+                  for (int m2 = 0; m2 < 2; ++m2) {
+                    const int mt = 2 * q4 + m2, g = (mt * 16) / GV;
+                    const uint32_t av[4] = {r[4 * m2], r[4 * m2 + 1], r[4 * m2 + 2], r[4 * m2 + 3]};
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) mma16816(O[mt][nt], av, bv[nt][g][0], bv[nt][g][1]);
+                  }
+                }
+              } else {
+#pragma unroll
+                for (int pl = 0; pl < 2; ++pl) {
+                  const uint4 w = cwp[pl * 32];
+                  const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                  for (int q4 = 0; q4 < 4; ++q4) {
+                    const int mt = 4 * pl + q4, g = (mt * 16) / GV;
+                    uint32_t av[4];
+                    unpack_word<4>(wv[q4], av);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) mma16816(O[mt][nt], av, bv[nt][g][0], bv[nt][g][1]);
+                  }
                 }
               }
-            }
-            if (r_pad > 0) {                          // low-rank value term, first product: U = A_V^T p
-              const __half* avs = avb + slab * (slab_a / 2);
+              cwp += SLABW;
+              // low-rank value term, first product: U = A_V^T p (zero rows when r = 0)
               uint32_t aa[4] = {0u, 0u, 0u, 0u};
-              if (gid < r_pad) {
-                aa[0] = *reinterpret_cast<const uint32_t*>(avs + gid * kSlab + 2 * t);
-                aa[2] = *reinterpret_cast<const uint32_t*>(avs + gid * kSlab + 2 * t + 8);
+              if (pv0) {
+                aa[0] = *reinterpret_cast<const uint32_t*>(avp);
+                aa[2] = *reinterpret_cast<const uint32_t*>(avp + 8);
               }
-              if (gid + 8 < r_pad) {
-                aa[1] = *reinterpret_cast<const uint32_t*>(avs + (gid + 8) * kSlab + 2 * t);
-                aa[3] = *reinterpret_cast<const uint32_t*>(avs + (gid + 8) * kSlab + 2 * t + 8);
+              if (pv1) {
+                aa[1] = *reinterpret_cast<const uint32_t*>(avp + 8 * kSlab);
+                aa[3] = *reinterpret_cast<const uint32_t*>(avp + 8 * kSlab + 8);
               }
+              avp += av_step;
 #pragma unroll
               for (int nt = 0; nt < NT; ++nt) mma16816(U[nt], aa, bp[nt][0], bp[nt][1]);
-            }
-          } else {
+            } else {
 #pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-              uint32_t av[4];
-              ldmatrix_x4_trans(av, stV + ((lane & 7) + 8 * (lane >> 4)) * kBufPitch + (16 * mt + 8 * ((lane >> 3) & 1)) * 2);
+              for (int mt = 0; mt < 8; ++mt) {
+                uint32_t av[4];
+                ldmatrix_x4_trans(av, stV + ((lane & 7) + 8 * (lane >> 4)) * kBufPitch + (16 * mt + 8 * ((lane >> 3) & 1)) * 2);
 #pragma unroll
-              for (int nt = 0; nt < NT; ++nt) mma16816(O[mt][nt], av, bp[nt][0], bp[nt][1]);
+                for (int nt = 0; nt < NT; ++nt) mma16816(O[mt][nt], av, bp[nt][0], bp[nt][1]);
+              }
             }
           }
-        }
+        };
+        if (is_buf) v_slabs(std::true_type{}); else v_slabs(std::false_type{});
         if (!is_buf && r_pad > 0) u_pending = true;
       }
 
@@ -796,6 +823,7 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
         const __half2* vsz = reinterpret_cast<const __half2*>(vp + o_vsz);
         const unsigned char* voval = vp + (sdc->off_voval - sdc->off_vpart);
         const unsigned char* voidx = vp + (sdc->off_voidx - sdc->off_vpart);
+#pragma unroll 1
         for (int tk = lane; tk < T; tk += 32) {
           float pS[HP];
 #pragma unroll
@@ -819,6 +847,7 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
             const unsigned char* oi = voidx + (size_t)tk * NGV * k2v;
 #pragma unroll
             for (int g = 0; g < NGV; ++g)
+#pragma unroll 1
               for (int e = 0; e < k2v; ++e) v_entry(g, __half2float(ov[g * k2v + e]), oi[g * k2v + e]);
           }
         }
