@@ -33,7 +33,10 @@ namespace gear {
 constexpr int kBufPitch = 272;                  // bytes per fp16 row of a buffer slab in shared memory
 constexpr int kBufItem = kSlab * kBufPitch;     // one slab of key rows or of value rows
 constexpr int kSpinLimit = 4000000;
-constexpr int kFragStride = 72;                 // 32-bit words per fragment row set (64 + padding against bank conflicts)
+// 32-bit words per B-fragment row set.  A row set holds, for every column that carries a query head (hi, lo) and
+// every lane column t, two registers; with one head only two of the eight columns exist and the lanes of the other
+// columns read those (their results are never used).  Padded against bank conflicts.
+__host__ __device__ constexpr int frag_row_words(int hp) { return hp == 1 ? 24 : 72; }
 
 static_assert(sizeof(SegDesc) <= 128 && sizeof(SegDesc) % 4 == 0, "descriptor copy assumes <= 32 words");
 
@@ -141,34 +144,39 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
                  DecodeArgs* a) {
   (void)bits;
   const int HP = heads == 1 ? 1 : (heads <= 4 ? 4 : 8), NT = HP > 4 ? 2 : 1;
-  const int bregion = round_up(max_bfac / 2, 128);
+  const int frs = frag_row_words(HP);
+  const int bregion = round_up(max_bfac / 2, 16);
   int part = max_kpart > max_vpart ? max_kpart : max_vpart;
   int stage = bregion + part;
   if (stage < kBufItem) stage = kBufItem;
-  stage = round_up(stage, 128);
+  stage = round_up(stage, 16);
   if (max_T < kSlab) max_T = kSlab;
   const int nslab = max_T / kSlab;
   const int frag_rows = 8 > nslab * (ngv + 1) ? 8 : nslab * (ngv + 1);
-  for (int ns = kMaxStages; ns >= 2; --ns) {
-    WarpSmem w;
-    int o = 0;
-    w.ring = o;    o += ns * stage;
-    w.sdp = o;     o += 128;
-    w.sdc = o;     o += 128;
-    w.qf = o;      o += HP * kHeadDim * 4;
-    w.qs = o;      o += HP * kHeadDim * 2;
-    w.frag = o;    o += NT * frag_rows * kFragStride * 4;
-    w.corr_k = o;  o += HP * max_T * 4;
-    w.ps = o;      o += HP * max_T * 4;
-    w.corr_v = o;  o += HP * kHeadDim * 4;
-    w.ocorr = o;   o += HP * kHeadDim * 4;
-    w.wl = o;      o += kMaxRank * 8 * 4;
-    w.misc = o;    o += 64;
-    w.total = round_up(o, 128);
-    // prefer three stages with more resident warps over four stages with fewer
-    if (ns == kMaxStages && (size_t)(w.total + 1024) * 10 > smem_budget) continue;
-    if ((size_t)w.total > smem_budget) continue;
-    a->nstage = ns; a->stage_bytes = stage; a->bregion = bregion; a->max_T = max_T; a->hpa = HP; a->ws = w;
+  WarpSmem w;
+  int o = 0;
+  w.sdp = 0;
+  w.sdc = o;     o += 128;
+  w.qf = o;      o += HP * kHeadDim * 4;
+  w.qs = o;      o += HP * kHeadDim * 2;
+  w.frag = o;    o += round_up(NT * frag_rows * frs * 4, 16);
+  w.corr_k = o;  o += HP * max_T * 4;
+  w.ps = o;      o += HP * max_T * 4;
+  w.corr_v = o;  o += HP * kHeadDim * 4;
+  w.ocorr = o;   o += HP * kHeadDim * 4;
+  w.wl = o;      o += kMaxRank * 8 * 4;
+  w.misc = o;    o += 64;
+  w.ring = round_up(o, 16);
+  // most resident warps (in steps of four: one per scheduler) whose ring still holds two stages; then as many
+  // stages as fit
+  const int reg_limit = HP == 1 ? 16 : (HP == 4 ? 12 : 6);
+  for (int warps = reg_limit; warps >= 1; warps -= (warps > 4 ? 4 : 1)) {
+    const long long per = (long long)smem_budget / warps - 1024;     // the system reserves 1 KB per CTA
+    long long ns = (per - w.ring) / stage;
+    if (ns < 2) continue;
+    if (ns > kMaxStages) ns = kMaxStages;
+    w.total = w.ring + (int)ns * stage;
+    a->nstage = (int)ns; a->stage_bytes = stage; a->bregion = bregion; a->max_T = max_T; a->hpa = HP; a->ws = w;
     return true;
   }
   return false;
@@ -177,11 +185,13 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
 // ------------------------------------------------------------------ the kernel
 // HEADS = query heads handled per pass: 1 (multi-head attention), 4 or 8 (grouped queries; a pass may hold fewer).
 template <int BITS, int HEADS, int NGV>
-__global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(const __grid_constant__ DecodeArgs a) {
+__global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) gear_decode_kernel(const __grid_constant__ DecodeArgs a) {
   constexpr int HP = HEADS;
   constexpr int NT = HEADS > 4 ? 2 : 1;           // 8-column tiles of the B operand
   constexpr int GV = kHeadDim / NGV;              // channels per value group
   constexpr int SLABW = kSlab * kHeadDim * BITS / 8 / 16;   // uint4 per slab of codes
+  constexpr int kFragStride = frag_row_words(HP);
+  constexpr int CMASK = HP == 1 ? 1 : 7;          // fragment columns that exist, as a mask on the lane's column
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ __align__(8) uint64_t bar[kMaxStages];
 
@@ -191,7 +201,6 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
   const int maxT = a.max_T;
   const int NS = a.nstage;
   unsigned char* ring = smem + a.ws.ring;
-  SegDesc* sdp = reinterpret_cast<SegDesc*>(smem + a.ws.sdp);
   SegDesc* sdc = reinterpret_cast<SegDesc*>(smem + a.ws.sdc);
   float* qf = reinterpret_cast<float*>(smem + a.ws.qf);          // [HP][128] q * scale * log2(e)
   __half* qs = reinterpret_cast<__half*>(smem + a.ws.qs);        // [HP][128] q
@@ -244,14 +253,14 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
     unsigned char* dst = ring + p_stage * a.stage_bytes;
     uint64_t* b = &bar[p_stage];
     if (p_blk < a.n_blocks_c) {
-      if (p_blk >= p_seg_hi) {                  // new segment (or new unit): refresh the cached descriptor
-        load_desc(sdp, p_blk);
-        p_seg_lo = sdp->blk_start;
-        p_seg_hi = p_seg_lo + sdp->nblk;
-        p_kbytes = sdp->off_vpart;
-        p_vbytes = sdp->rec_bytes - p_kbytes;
-        p_hb = sdp->bfac_bytes >> 1;
-        p_segb = a.arena + sdp->seg_base + (size_t)p_bh * sdp->bh_stride;
+      if (p_blk >= p_seg_hi) {                  // new segment (or new unit): read its descriptor
+        const SegDesc* sd = a.table + a.blk2seg[p_blk];
+        p_seg_lo = sd->blk_start;
+        p_seg_hi = p_seg_lo + sd->nblk;
+        p_kbytes = sd->off_vpart;
+        p_vbytes = sd->rec_bytes - p_kbytes;
+        p_hb = sd->bfac_bytes >> 1;
+        p_segb = a.arena + sd->seg_base + (size_t)p_bh * sd->bh_stride;
         p_rec = p_segb + 2 * p_hb + (size_t)(p_blk - p_seg_lo) * (p_kbytes + p_vbytes);
       }
       if (lane == 0) {
@@ -510,7 +519,7 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int kc = 0; kc < 8; ++kc) {
-          const uint2 v = *reinterpret_cast<const uint2*>(frag + (nt * 8 + kc) * kFragStride + lane * 2);
+          const uint2 v = *reinterpret_cast<const uint2*>(frag + (nt * 8 + kc) * kFragStride + ((gid & CMASK) * 4 + t) * 2);
           bq[nt][kc][0] = v.x; bq[nt][kc][1] = v.y;
         }
 
@@ -734,8 +743,8 @@ __global__ void __launch_bounds__(32, HEADS <= 4 ? 10 : 5) gear_decode_kernel(co
           constexpr bool kBuf = decltype(buf_tag)::value;
           const uint4* cwp = reinterpret_cast<const uint4*>(vp) + lane;
           const __half* avp = reinterpret_cast<const __half*>(vp + o_av) + gid * kSlab + 2 * t;
-          const uint32_t* fvp = fragV + lane * 2;
-          const uint32_t* fpp = fragP + lane * 2;
+          const uint32_t* fvp = fragV + ((gid & CMASK) * 4 + t) * 2;
+          const uint32_t* fpp = fragP + ((gid & CMASK) * 4 + t) * 2;
           const int fstep = nslab * kFragStride, av_step = kSlab * r_pad;
 #pragma unroll 1
           for (int slab = 0; slab < nslab; ++slab) {
