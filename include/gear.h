@@ -140,6 +140,36 @@ gear_status gear_fp16_decode_attn(const void* K, const void* V, const void* q, f
                                   void* scratch, size_t scratch_bytes, void* stream);
 size_t gear_fp16_attn_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim);
 
+/* gear_fp16_decode_attn for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, not a step of the method.)
+ *
+ * Some hosts of this library are not allowed to call cudaMalloc at the point where they need
+ * attention: code running inside a framework that owns the whole device heap, a plug-in that is
+ * handed buffers but no allocator, or a latency-critical loop in which an allocation (which may
+ * synchronise the device) is not acceptable.  For them the scratch memory that
+ * gear_fp16_decode_attn takes from the caller lives in a fixed array of
+ * GEAR_STATIC_SCRATCH_BYTES inside the library's device image: every GPU that loads the
+ * library holds that much memory until the process exits.  The call allocates and frees
+ * nothing, on the device or through any library.
+ *
+ * Arguments and result are those of gear_fp16_decode_attn (K, V, q, out are device pointers,
+ * 16-byte aligned, borrowed for the duration of the enqueued work) without the scratch pair.
+ *   - batch * n_q_heads must not exceed GEAR_STATIC_MAX_QUERY_HEADS; larger problems, or any
+ *     problem whose bookkeeping does not fit the array, return GEAR_ERR_CAPACITY and launch
+ *     nothing.  Within the limit the launch may use fewer CTAs than gear_fp16_decode_attn
+ *     would, so that its partial results fit; the output is the same up to rounding order.
+ *   - The first call on a device looks up the array's device address (once per device, with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and the array keeps what the last call left
+ *     in it; each call clears the part that must start at zero on `stream` before its kernel.
+ *     Two calls whose GPU work can overlap (different streams without an ordering between
+ *     them, or several host threads) race on the array: order them. */
+#define GEAR_STATIC_SCRATCH_BYTES (4u << 20)
+#define GEAR_STATIC_MAX_QUERY_HEADS 256
+gear_status gear_fp16_decode_attn_static(const void* K, const void* V, const void* q, float* out,
+                                         int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                         int64_t n, int64_t n_alloc, float softmax_scale, void* stream);
+
 /* ---- test / accounting helpers (not on the timed path; gear_export synchronises) ---- */
 
 enum {                       /* `what` of gear_export; K_ / V_ select the side                      */

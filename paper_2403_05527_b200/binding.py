@@ -66,6 +66,8 @@ _SIGNATURES = {
                                           C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_float, C.c_void_p,
                                           C.c_size_t, C.c_void_p]),
     "gear_fp16_attn_scratch_bytes": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32]),
+    "gear_fp16_decode_attn_static": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                                 C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_float, C.c_void_p]),
     "gear_export": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]),
     "gear_cache_info": (C.c_int32, [C.c_void_p, C.POINTER(GearInfo)]),
     "gear_segment_info_get": (C.c_int32, [C.c_void_p, C.c_int32, C.POINTER(GearSegmentInfo)]),
@@ -170,6 +172,15 @@ def gear_fp16_decode_attn(K, V, q, out, batch, n_q_heads, n_kv_heads, n, n_alloc
                                               head_dim, n, n_alloc, softmax_scale, _ptr(scratch),
                                               scratch.numel() * scratch.element_size(), _stream(stream)),
                   "gear_fp16_decode_attn")
+
+
+def gear_fp16_decode_attn_static(K, V, q, out, batch, n_q_heads, n_kv_heads, n, n_alloc, softmax_scale=0.0,
+                                 head_dim=128, stream=None) -> int:
+    """gear_fp16_decode_attn without a scratch argument: the library's built-in device array is used, nothing is
+    allocated.  Calls that may overlap on the GPU must be ordered by the caller (they share that array)."""
+    return _check(lib().gear_fp16_decode_attn_static(_ptr(K), _ptr(V), _ptr(q), _ptr(out), batch, n_q_heads, n_kv_heads,
+                                                     head_dim, n, n_alloc, softmax_scale, _stream(stream)),
+                  "gear_fp16_decode_attn_static")
 
 
 def gear_free(cache) -> None:
