@@ -192,6 +192,7 @@ static gear_status compress_segment(gear_cache* c, const void* K, const void* V,
   sd.tok_start = (int)c->n_compressed;
   sd.blk_start = c->n_blocks_c;
   sd.dbg_base = -1;
+  sd.shape_id = static_shape_id(sd, c->cc);
   float* dbgA = nullptr; float* dbgB = nullptr;
   long long offA = -1, offB = -1;
   if (c->dbg && rank > 0) {

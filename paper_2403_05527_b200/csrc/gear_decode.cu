@@ -182,6 +182,61 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
   return false;
 }
 
+// ------------------------------------------------------------------ block shapes
+// The work on a block depends on its shape: tokens T, outliers per key group, padded rank, outliers per value
+// group.  The shapes of the usual configurations are compile-time constants (every offset inside the record becomes
+// an immediate and the slab loops unroll); any other segment runs through the same code with run-time values.
+struct DynShape {                      // values read from the segment descriptor
+  static constexpr bool kDyn = true, kBuf = false;
+  static constexpr int T = 0, k2k = 0, r_pad = 0, k2v = 0, unroll = 1;
+  static constexpr int off_kscale = 0, off_koval = 0, off_koidx = 0, off_kcodes = 0, off_ak = 0, off_av = 0, off_vscale = 0,
+                       off_voval = 0, off_voidx = 0;
+};
+struct BufShape {                      // one slab of fp16 rows of the streaming buffer
+  static constexpr bool kDyn = false, kBuf = true;
+  static constexpr int T = kSlab, k2k = 0, r_pad = 0, k2v = 0, unroll = 1;
+  static constexpr int off_kscale = 0, off_koval = 0, off_koidx = 0, off_kcodes = 0, off_ak = 0, off_av = 0, off_vscale = 0,
+                       off_voval = 0, off_voidx = 0;
+};
+template <int BITS, int NGV, int T_, int KK, int RP, int KV>
+struct StaticShape {                   // mirrors layout_segment(); checked against it on the host (static_shape_id)
+  static constexpr bool kDyn = false, kBuf = false;
+  static constexpr int T = T_, k2k = 2 * KK, r_pad = RP, k2v = 2 * KV, unroll = 4;
+  static constexpr int nslab = T_ / kSlab, slab_codes = kSlab * kHeadDim * BITS / 8;
+  static constexpr int off_kscale = kRecHeader;
+  static constexpr int off_koval = off_kscale + kHeadDim * 4;
+  static constexpr int off_koidx = off_koval + kHeadDim * 2 * KK * 2;
+  static constexpr int off_kcodes = off_koidx + (kHeadDim * 2 * KK + 15) / 16 * 16;
+  static constexpr int off_ak = off_kcodes + nslab * slab_codes;
+  static constexpr int off_vpart = off_ak + (nslab * kSlab * RP * 2 + 15) / 16 * 16;
+  // value part, relative to its start
+  static constexpr int off_av = nslab * slab_codes;
+  static constexpr int off_vscale = off_av + (nslab * kSlab * RP * 2 + 15) / 16 * 16;
+  static constexpr int off_voval = off_vscale + T_ * NGV * 4;
+  static constexpr int off_voidx = off_voval + (T_ * NGV * 2 * KV * 2 + 15) / 16 * 16;
+  static constexpr int rec_bytes = off_vpart + off_voidx + (T_ * NGV * 2 * KV + 15) / 16 * 16;
+  static bool matches(const SegDesc& s, const CacheConst& c) {
+    return c.bits == BITS && c.ngv == NGV && c.k_v == KV && s.T == T_ && s.k_k == KK && s.r_pad == RP &&
+           s.off_kscale == off_kscale && s.off_koval == off_koval && s.off_koidx == off_koidx &&
+           s.off_kcodes == off_kcodes && s.off_ak == off_ak && s.off_vpart == off_vpart &&
+           s.off_vcodes == off_vpart && s.off_av == off_vpart + off_av && s.off_vscale == off_vpart + off_vscale &&
+           s.off_voval == off_vpart + off_voval && s.off_voidx == off_vpart + off_voidx && s.rec_bytes == rec_bytes;
+  }
+};
+// static shapes by id (0 = none).  Two value groups per token (g = 64): ids 1, 2; one group (g = 128): ids 3, 4.
+template <int BITS> using ShapeA1 = StaticShape<BITS, 2, 64, 1, 4, 1>;     // g 64, s <= 3 %, rank 3..4
+template <int BITS> using ShapeA2 = StaticShape<BITS, 2, 64, 1, 8, 1>;     // g 64, rank 5..8
+template <int BITS> using ShapeB1 = StaticShape<BITS, 1, 128, 2, 4, 2>;    // g 128 prefill blocks
+template <int BITS> using ShapeB2 = StaticShape<BITS, 1, 64, 1, 4, 2>;     // g 128, flushed 64-token buffers
+
+int static_shape_id(const SegDesc& s, const CacheConst& c) {
+  if (ShapeA1<2>::matches(s, c) || ShapeA1<4>::matches(s, c)) return 1;
+  if (ShapeA2<2>::matches(s, c) || ShapeA2<4>::matches(s, c)) return 2;
+  if (ShapeB1<2>::matches(s, c) || ShapeB1<4>::matches(s, c)) return 3;
+  if (ShapeB2<2>::matches(s, c) || ShapeB2<4>::matches(s, c)) return 4;
+  return 0;
+}
+
 // ------------------------------------------------------------------ the kernel
 // HEADS = query heads handled per pass: 1 (multi-head attention), 4 or 8 (grouped queries; a pass may hold fewer).
 template <int BITS, int HEADS, int NGV>
@@ -298,7 +353,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
   };
   for (int s = 0; s < NS; ++s) issue();
 
-  int c_stage = 0, c_par = 0, c_seg_lo = 0, c_seg_hi = 0;
+  int c_stage = 0, c_par = 0, c_seg_lo = 0, c_seg_hi = 0, c_shape = 0;
   bool alive = true;
   // wait for the next item (items are consumed in order); returns its stage
   auto acquire = [&]() -> unsigned char* {
@@ -363,29 +418,43 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
 
 #pragma unroll 1
     for (int blk = blk_lo; blk < blk_hi; ++blk) {
-      const bool is_buf = blk >= a.n_blocks_c;
+      const bool buf_blk = blk >= a.n_blocks_c;
+      if (!buf_blk && (blk >= c_seg_hi || blk < c_seg_lo)) {
+        load_desc(sdc, blk);
+        c_seg_lo = sdc->blk_start;
+        c_seg_hi = c_seg_lo + sdc->nblk;
+        c_shape = sdc->shape_id;
+      }
+      auto body = [&](auto shape_tag) {
+      using S = decltype(shape_tag);
+      constexpr bool is_buf = S::kBuf;
       // ---------------- block geometry
-      int T = kSlab, r_pad = 0, k2k = 0, valid_tokens = kSlab;
+      const int T = S::kDyn ? sdc->T : S::T;
+      const int r_pad = S::kDyn ? sdc->r_pad : S::r_pad;
+      const int k2k = S::kDyn ? 2 * sdc->k_k : S::k2k;
+      const int k2v = S::kDyn ? 2 * a.cc.k_v : S::k2v;
+      const int off_kscale = S::kDyn ? sdc->off_kscale : S::off_kscale;
+      const int off_koval = S::kDyn ? sdc->off_koval : S::off_koval;
+      const int off_koidx = S::kDyn ? sdc->off_koidx : S::off_koidx;
+      const int off_kcodes = S::kDyn ? sdc->off_kcodes : S::off_kcodes;
+      const int off_ak = S::kDyn ? sdc->off_ak : S::off_ak;
+      const int o_av = S::kDyn ? sdc->off_av - sdc->off_vpart : S::off_av;
+      const int o_vsz = S::kDyn ? sdc->off_vscale - sdc->off_vpart : S::off_vscale;
+      const int o_voval = S::kDyn ? sdc->off_voval - sdc->off_vpart : S::off_voval;
+      const int o_voidx = S::kDyn ? sdc->off_voidx - sdc->off_vpart : S::off_voidx;
+      int valid_tokens = T;
       bool with_bk = false, with_bv = false;
       if (!is_buf) {
-        if (blk >= c_seg_hi || blk < c_seg_lo) {
-          load_desc(sdc, blk);
-          c_seg_lo = sdc->blk_start;
-          c_seg_hi = c_seg_lo + sdc->nblk;
-        }
-        T = sdc->T; r_pad = sdc->r_pad; k2k = 2 * sdc->k_k;
-        valid_tokens = T;
         with_bk = r_pad > 0 && (blk == c_seg_lo || blk == blk_lo);
         with_bv = r_pad > 0 && (blk == c_seg_hi - 1 || blk == blk_hi - 1);
       } else {
         valid_tokens = min(kSlab, a.buf_len - (blk - a.n_blocks_c) * kSlab);
       }
       const int nslab = T / kSlab;
-      const int slab_a = 2 * kSlab * r_pad;
 
       // ================================================================ key item
       unsigned char* stK = acquire();
-      if (!alive) break;
+      if (!alive) return;
       const unsigned char* kp = stK + a.bregion;
       float dmax_v = 0.f;
       int own_sexp[NT];
@@ -452,7 +521,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
           const float dmax_k = reinterpret_cast<const float*>(kp)[0];
           dmax_v = reinterpret_cast<const float*>(kp)[1];
           ed = float_exponent(dmax_k);
-          const uint4 kz = reinterpret_cast<const uint4*>(kp + sdc->off_kscale)[lane];
+          const uint4 kz = reinterpret_cast<const uint4*>(kp + off_kscale)[lane];
           const uint32_t w4[4] = {kz.x, kz.y, kz.z, kz.w};
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
@@ -494,8 +563,8 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
               if (h < HPu) atomicAdd(&corr_k[h * maxT + idx], __float2int_rn(qS[h][j] * d));
           };
           if (k2k == 2) {
-            const uint4 ov = reinterpret_cast<const uint4*>(kp + sdc->off_koval)[lane];
-            const uint2 oi = reinterpret_cast<const uint2*>(kp + sdc->off_koidx)[lane];
+            const uint4 ov = reinterpret_cast<const uint4*>(kp + off_koval)[lane];
+            const uint2 oi = reinterpret_cast<const uint2*>(kp + off_koidx)[lane];
             const uint32_t o4[4] = {ov.x, ov.y, ov.z, ov.w};
             const uint32_t i2[2] = {oi.x, oi.y};
 #pragma unroll
@@ -504,8 +573,8 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
               k_entry(j, __high2float(u32_as_h2(o4[j])), (i2[j >> 1] >> (16 * (j & 1) + 8)) & 0xFFu);
             }
           } else {
-            const __half* ov = reinterpret_cast<const __half*>(kp + sdc->off_koval) + lane * 4 * k2k;
-            const unsigned char* oi = kp + sdc->off_koidx + lane * 4 * k2k;
+            const __half* ov = reinterpret_cast<const __half*>(kp + off_koval) + lane * 4 * k2k;
+            const unsigned char* oi = kp + off_koidx + lane * 4 * k2k;
 #pragma unroll
             for (int j = 0; j < 4; ++j)
 #pragma unroll 1
@@ -533,11 +602,11 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
         const bool has_ko = k2k > 0;
         auto k_slabs = [&](auto buf_tag) {
           constexpr bool kBuf = decltype(buf_tag)::value;
-          const uint4* cwp = reinterpret_cast<const uint4*>(kp + (kBuf ? 0 : sdc->off_kcodes)) + lane;
-          const __half* akp = reinterpret_cast<const __half*>(kp + (kBuf ? 0 : sdc->off_ak)) + gid * r_pad + 2 * t;
+          const uint4* cwp = reinterpret_cast<const uint4*>(kp + off_kcodes) + lane;
+          const __half* akp = reinterpret_cast<const __half*>(kp + off_ak) + gid * r_pad + 2 * t;
           const int ak8 = 8 * r_pad, ak_step = kSlab * r_pad;
           int tok0 = 0;
-#pragma unroll 1
+#pragma unroll (S::unroll)
           for (int slab = 0; slab < nslab; ++slab) {
             float acc[2][NT][4];
 #pragma unroll
@@ -621,7 +690,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
             tok0 += kSlab;
           }
         };
-        if (is_buf) k_slabs(std::true_type{}); else k_slabs(std::false_type{});
+        k_slabs(std::integral_constant<bool, is_buf>{});
       }
       release();                                      // the key item is consumed
 
@@ -686,10 +755,8 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
 
       // ================================================================ value item
       unsigned char* stV = acquire();
-      if (!alive) break;
+      if (!alive) return;
       const unsigned char* vp = stV + a.bregion;          // value part of the record
-      const int o_av = is_buf ? 0 : sdc->off_av - sdc->off_vpart;
-      const int o_vsz = is_buf ? 0 : sdc->off_vscale - sdc->off_vpart;
       uint32_t* fragV = frag;                                         // [NT][NGV][nslab] rows of kFragStride words
       uint32_t* fragP = frag + NT * NGV * nslab * kFragStride;        // [NT][nslab]
       if (is_buf && valid_tokens < kSlab) {
@@ -746,7 +813,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
           const uint32_t* fvp = fragV + ((gid & CMASK) * 4 + t) * 2;
           const uint32_t* fpp = fragP + ((gid & CMASK) * 4 + t) * 2;
           const int fstep = nslab * kFragStride, av_step = kSlab * r_pad;
-#pragma unroll 1
+#pragma unroll (S::unroll)
           for (int slab = 0; slab < nslab; ++slab) {
             uint32_t bp[NT][2];
 #pragma unroll
@@ -820,18 +887,17 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
             }
           }
         };
-        if (is_buf) v_slabs(std::true_type{}); else v_slabs(std::false_type{});
+        v_slabs(std::integral_constant<bool, is_buf>{});
         if (!is_buf && r_pad > 0) u_pending = true;
       }
 
       // ---------------- sparse value term: p[tok] * (x - zero[tok, g]) scattered to the outlier's channel
-      if (!is_buf && a.cc.k_v > 0) {
-        const int k2v = 2 * a.cc.k_v;
+      if (!is_buf && k2v > 0) {
         const int sexp = clamp60(21 - float_exponent(dmax_v));
         const float S = pow2i(sexp), Si = pow2i(-sexp);
         const __half2* vsz = reinterpret_cast<const __half2*>(vp + o_vsz);
-        const unsigned char* voval = vp + (sdc->off_voval - sdc->off_vpart);
-        const unsigned char* voidx = vp + (sdc->off_voidx - sdc->off_vpart);
+        const unsigned char* voval = vp + o_voval;
+        const unsigned char* voidx = vp + o_voidx;
 #pragma unroll 1
         for (int tk = lane; tk < T; tk += 32) {
           float pS[HP];
@@ -918,6 +984,14 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
         u_pending = false;
       }
       release();                                      // the value item is consumed
+      };
+      if (buf_blk) body(BufShape{});
+      else if (NGV == 2 && c_shape == 1) body(ShapeA1<BITS>{});
+      else if (NGV == 2 && c_shape == 2) body(ShapeA2<BITS>{});
+      else if (NGV == 1 && c_shape == 3) body(ShapeB1<BITS>{});
+      else if (NGV == 1 && c_shape == 4) body(ShapeB2<BITS>{});
+      else body(DynShape{});
+      if (!alive) break;
     }
     if (!alive) break;
 

@@ -90,6 +90,7 @@ cudaError_t launch_decode(const DecodeArgs& a, int grid, cudaStream_t st);
 bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int max_bfac, int max_T, size_t smem_budget,
                  DecodeArgs* a);
 int decode_occupancy(int bits, int heads, int ngv, size_t smem);
+int static_shape_id(const SegDesc& s, const CacheConst& c);
 
 // fp16-cache attention
 cudaError_t launch_fp16_attn(const void* K, const void* V, const void* q, float* out, int batch, int n_q_heads,

@@ -54,6 +54,7 @@ struct SegDesc {
   int slab_codes;        // bytes of codes per slab and side
   int slab_a;            // bytes of A rows per slab and side
   int off_vpart;         // start of the value part inside a record (= bytes of the key part)
+  int shape_id;          // compile-time block shape of the decode kernel that fits this segment, 0 = none
 };
 
 // Cache-wide constants the kernels need.
