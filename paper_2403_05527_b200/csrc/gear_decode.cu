@@ -201,7 +201,7 @@ struct BufShape {                      // one slab of fp16 rows of the streaming
 template <int BITS, int NGV, int T_, int KK, int RP, int KV>
 struct StaticShape {                   // mirrors layout_segment(); checked against it on the host (static_shape_id)
   static constexpr bool kDyn = false, kBuf = false;
-  static constexpr int T = T_, k2k = 2 * KK, r_pad = RP, k2v = 2 * KV, unroll = 4;
+  static constexpr int T = T_, k2k = 2 * KK, r_pad = RP, k2v = 2 * KV, unroll = 2;
   static constexpr int nslab = T_ / kSlab, slab_codes = kSlab * kHeadDim * BITS / 8;
   static constexpr int off_kscale = kRecHeader;
   static constexpr int off_koval = off_kscale + kHeadDim * 4;
@@ -457,10 +457,10 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
       if (!alive) return;
       const unsigned char* kp = stK + a.bregion;
       float dmax_v = 0.f;
-      int own_sexp[NT];
-      float ch_own[NT];
+      int sexp_k[HP];                                 // per head: exponent of the sparse key term's fixed-point scale
+      float c_zero[HP];                               // per head: sum over channels of q * zero-point
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) { own_sexp[nt] = 0; ch_own[nt] = 0.f; }
+      for (int h = 0; h < HP; ++h) { sexp_k[h] = 0; c_zero[h] = 0.f; }
 
       if (with_bk) {
         // w = q B_K through the tensor cores, kept as the B operand of the low-rank key term
@@ -551,7 +551,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
               const int sexp = clamp60(21 - qexp_s[h] - ed);
               const float S = pow2i(sexp);
               qS[h][0] = qv.x * S; qS[h][1] = qv.y * S; qS[h][2] = qv.z * S; qS[h][3] = qv.w * S;
-              if ((h & 3) == t) { ch_own[h >> 2] = c; own_sexp[h >> 2] = sexp; }
+              c_zero[h] = c; sexp_k[h] = sexp;
             }
           }
         }
@@ -594,12 +594,10 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
 
       // ---------------- key scores, slab by slab; scores go to shared memory
       {
-        float Si[NT];
         int psoff[NT];                                  // this lane's first score slot (head t + 4 nt, token gid)
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) { Si[nt] = pow2i(-own_sexp[nt]); psoff[nt] = (t + 4 * nt) * maxT + gid; }
+        for (int nt = 0; nt < NT; ++nt) psoff[nt] = (t + 4 * nt) * maxT + gid;
         const bool pa0 = 2 * t < r_pad, pa1 = 2 * t + 8 < r_pad;
-        const bool has_ko = k2k > 0;
         auto k_slabs = [&](auto buf_tag) {
           constexpr bool kBuf = decltype(buf_tag)::value;
           const uint4* cwp = reinterpret_cast<const uint4*>(kp + off_kcodes) + lane;
@@ -675,14 +673,9 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
               if (t + 4 * nt < HPu) {
-                float v0 = (acc[0][nt][0] + acc[0][nt][1]) + (acc[1][nt][0] + acc[1][nt][1]) + ch_own[nt];
-                float v1 = (acc[0][nt][2] + acc[0][nt][3]) + (acc[1][nt][2] + acc[1][nt][3]) + ch_own[nt];
-                if (!kBuf && has_ko) {
-                  int* ck = corr_k + psoff[nt] + tok0;
-                  v0 = fmaf((float)ck[0], Si[nt], v0);
-                  v1 = fmaf((float)ck[8], Si[nt], v1);
-                  ck[0] = 0; ck[8] = 0;
-                }
+                // raw sums only: the zero-point constant and the sparse term are added in the softmax pass
+                const float v0 = (acc[0][nt][0] + acc[0][nt][1]) + (acc[1][nt][0] + acc[1][nt][1]);
+                const float v1 = (acc[0][nt][2] + acc[0][nt][3]) + (acc[1][nt][2] + acc[1][nt][3]);
                 float* pr = ps + psoff[nt] + tok0;
                 pr[0] = v0; pr[8] = v1;
               }
@@ -703,9 +696,19 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
           alpha[h] = 1.f;
           if (h < HPu) {
             float* row = ps + h * maxT;
+            int* crow = corr_k + h * maxT;
+            const float Sik = pow2i(-sexp_k[h]);
             float mx = -INFINITY;
 #pragma unroll 1
-            for (int tk = lane; tk < valid_tokens; tk += 32) mx = fmaxf(mx, row[tk]);
+            for (int tk = lane; tk < valid_tokens; tk += 32) {
+              float v = row[tk] + c_zero[h];
+              if (!is_buf && k2k > 0) {
+                v = fmaf((float)crow[tk], Sik, v);
+                crow[tk] = 0;
+              }
+              row[tk] = v;
+              mx = fmaxf(mx, v);
+            }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             const float m_new = fmaxf(m_run[h], mx);       // finite: every block holds a valid token
