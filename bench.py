@@ -135,6 +135,23 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------- multi-rank reduction
+def max_over_ranks(value, dist, device):
+    """Largest `value` over all ranks (the job is as slow as its slowest rank); `dist` None means one rank."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world, batch_per_rank, calls_per_rank, seconds):
+    """Every rank attends `batch_per_rank` sequences per call on its own shard of the batch (no exchange between
+    ranks: (batch, head) units are independent), so the job's throughput is the sum over ranks."""
+    return world * batch_per_rank * calls_per_rank / seconds
+
+
 # --------------------------------------------------------------------------- our arm
 def device_kv(torch, w, dev, seed):
     """K, V fp16 [B, H, n, 128] drawn on the device with the distribution of synth.make_kv."""
@@ -243,11 +260,7 @@ def run_ours(args, w):
     t_wall1 = time.time()
     launches = G.gear_kernel_launches() - launches0
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
-    ms_total = s0.elapsed_time(s1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(s0.elapsed_time(s1), dist, dev)
     status = [G.gear_last_device_status(c) for c in caches]
     if any(status):
         raise SystemExit(f"device status word set: {status}")
@@ -255,7 +268,7 @@ def run_ours(args, w):
         raise SystemExit("non-finite attention output")
 
     n_calls = args.steps * nb * L
-    value = world * B * n_calls / (ms_total * 1e-3)
+    value = whole_job_tokens_per_s(world, B, n_calls, ms_total * 1e-3)
     dec_ms = [a.elapsed_time(b) for a, b in events]
     dec_bytes = float(sum(bytes_log))
     achieved = dec_bytes / (sum(dec_ms) * 1e-3) / 1e9
@@ -280,12 +293,8 @@ def run_ours(args, w):
     for _ in range(args.e2e_steps):
         step_e2e()
     barrier()
-    e2e_s = max(time.perf_counter() - t0, 1e-9)
-    if dist is not None:
-        t = torch.tensor([e2e_s], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = world * B * args.e2e_steps * nb * L / e2e_s
+    e2e_s = max_over_ranks(max(time.perf_counter() - t0, 1e-9), dist, dev)
+    e2e_value = whole_job_tokens_per_s(world, B, args.e2e_steps * nb * L, e2e_s)
     h2d = nb * L * (2 * hk_np[0].nbytes + hq_np.nbytes)
     d2h = nb * L * hout_np.nbytes
 
