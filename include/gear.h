@@ -119,6 +119,11 @@ gear_status gear_decode_attn(gear_cache* cache, const void* q, float* out,
 /* Release the cache and everything it owns.  NULL is allowed. */
 void gear_free(gear_cache* cache);
 
+/* gear_compress takes its transient workspace (the residual of the block being compressed, up to 3 GB)
+ * from a stream-ordered pool that the library keeps per device, so that repeated calls do not go back
+ * to the driver.  This call synchronises the current device and returns that memory to the driver. */
+gear_status gear_release_workspace(void);
+
 /* ---- host-buffer variants (copies inside the call; they synchronise `stream`) ---- */
 
 /* gear_append_buffer with k_new, v_new (and B0_flush) in HOST memory. */

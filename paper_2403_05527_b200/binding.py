@@ -60,6 +60,7 @@ _SIGNATURES = {
     "gear_append_buffer": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "gear_decode_attn": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
     "gear_free": (None, [C.c_void_p]),
+    "gear_release_workspace": (C.c_int32, []),
     "gear_append_buffer_host": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "gear_decode_attn_host": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
     "gear_fp16_decode_attn": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
@@ -186,6 +187,10 @@ def gear_fp16_decode_attn_static(K, V, q, out, batch, n_q_heads, n_kv_heads, n, 
 def gear_free(cache) -> None:
     if cache is not None:
         lib().gear_free(cache)
+
+
+def gear_release_workspace() -> int:
+    return _check(lib().gear_release_workspace(), "gear_release_workspace")
 
 
 def gear_cache_info(cache) -> GearInfo:

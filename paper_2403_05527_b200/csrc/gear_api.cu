@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -16,6 +17,42 @@ using namespace gear;
 static std::atomic<unsigned long long> g_launches{0};
 void gear::count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 extern "C" uint64_t gear_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+// Transient workspace of gear_compress comes from one stream-ordered pool per device that keeps its memory between
+// calls (the default pool hands it back to the driver at every synchronisation, which costs milliseconds per call).
+static std::mutex g_pool_mutex;
+static cudaMemPool_t g_pool[64];
+static bool g_pool_ready[64];
+static cudaMemPool_t workspace_pool(int dev) {
+  if (dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_pool_mutex);
+  if (!g_pool_ready[dev]) {
+    cudaMemPoolProps props;
+    memset(&props, 0, sizeof(props));
+    props.allocType = cudaMemAllocationTypePinned;
+    props.handleTypes = cudaMemHandleTypeNone;
+    props.location.type = cudaMemLocationTypeDevice;
+    props.location.id = dev;
+    cudaMemPool_t pool = nullptr;
+    if (cudaMemPoolCreate(&pool, &props) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    unsigned long long keep = ~0ull;
+    cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+    g_pool[dev] = pool;
+    g_pool_ready[dev] = true;
+  }
+  return g_pool[dev];
+}
+
+extern "C" gear_status gear_release_workspace(void) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
+  std::lock_guard<std::mutex> lock(g_pool_mutex);
+  if (dev >= 0 && dev < 64 && g_pool_ready[dev] && cudaMemPoolTrimTo(g_pool[dev], 0) != cudaSuccess) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  return GEAR_OK;
+}
 
 struct gear_cache {
   gear_config cfg;
@@ -208,7 +245,9 @@ static gear_status compress_segment(gear_cache* c, const void* K, const void* V,
   job.seed = c->cfg.seed; job.segment_index = (int)c->segs.size(); job.iters = c->cfg.power_iters;
 
   cudaError_t e = cudaSuccess;
-  if (is_flush) {
+  if (compress_tile_fits(sd.T, sd.n_c)) {
+    e = compress_tile(job, c->cc.BH, st);              // short segment: one launch, residual in shared memory
+  } else if (is_flush) {
     e = compress_range(job, 0, c->cc.BH, c->flush_ws, st);
   } else {
     // bounded transient workspace, (batch, head) pairs processed in ranges
@@ -219,7 +258,11 @@ static gear_status compress_segment(gear_cache* c, const void* K, const void* V,
     if (chunk > c->cc.BH) chunk = c->cc.BH;
     unsigned char* ws = nullptr;
     const size_t ws_bytes = compress_workspace_bytes(chunk, n, rank);
-    if (cudaMallocAsync((void**)&ws, ws_bytes, st) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_ALLOC; }
+    cudaMemPool_t pool = workspace_pool(c->device);
+    if (pool == nullptr || cudaMallocFromPoolAsync((void**)&ws, ws_bytes, pool, st) != cudaSuccess) {
+      cudaGetLastError();
+      return GEAR_ERR_ALLOC;
+    }
     for (int bh0 = 0; bh0 < c->cc.BH && e == cudaSuccess; bh0 += chunk) {
       const int nbh = bh0 + chunk <= c->cc.BH ? chunk : c->cc.BH - bh0;
       e = compress_range(job, bh0, nbh, ws, st);

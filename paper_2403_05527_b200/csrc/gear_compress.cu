@@ -537,6 +537,331 @@ __global__ void __launch_bounds__(256) pi_gram2_kernel(PiArgs p) {
   }
 }
 
+// ---------------------------------------------------------------------------
+// Whole-tile compression for short segments (a flushed buffer, Algorithm 1's
+// decoding phase): one CTA takes one (batch, head, K|V) tile of n_c <= 128
+// tokens through Filter, Quant, residual and all of Algorithm 2 with the
+// residual held in shared memory, so that a flush is one launch instead of a
+// chain of a dozen latency-bound ones.
+// ---------------------------------------------------------------------------
+constexpr int kTileMaxTokens = 128;
+constexpr int kFPitch = kMaxRank + 1;      // floats per row of the factor matrices in shared memory
+
+struct TileArgs {
+  SegDesc seg;
+  CacheConst cc;
+  unsigned char* arena;
+  const __half* K;      // [BH][n_c][128]
+  const __half* V;
+  const float* B0;      // [BH][2][128][rank] or nullptr
+  float* dbgA;
+  float* dbgB;
+  unsigned long long seed;
+  int segment_index;
+  int iters;
+};
+
+__device__ __forceinline__ float block_sum128(float v, float* wsum, int lane, int warp) {
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane == 0) wsum[warp] = v;
+  __syncthreads();
+  return (wsum[0] + wsum[1]) + (wsum[2] + wsum[3]);
+}
+
+// G = U^T U (upper Cholesky factor) and U^-1 for the r x r Gram matrix G; first: W <- U^-1, else W <- W U^-1.
+// A column whose pivot vanishes is zeroed.  Run by one warp; matrices have pitch kFPitch.
+__device__ void chol_update(const float* G, float* U, float* Ui, float* W, int r, int first, int lane) {
+  for (int i = lane; i < kMaxRank * kFPitch; i += 32) { U[i] = 0.f; Ui[i] = 0.f; }
+  __syncwarp();
+  if (lane == 0) {
+    float tr = 0.f;
+    for (int i = 0; i < r; ++i) tr += G[i * kFPitch + i];
+    const float tiny = tr * 1e-12f;
+    for (int j = 0; j < r; ++j) {
+      float d = G[j * kFPitch + j];
+      for (int k = 0; k < j; ++k) d -= U[k * kFPitch + j] * U[k * kFPitch + j];
+      const bool ok = d > tiny && d > 0.f;
+      const float ujj = ok ? sqrtf(d) : 0.f;
+      U[j * kFPitch + j] = ujj;
+      for (int i = j + 1; i < r; ++i) {
+        float sacc = G[j * kFPitch + i];
+        for (int k = 0; k < j; ++k) sacc -= U[k * kFPitch + j] * U[k * kFPitch + i];
+        U[j * kFPitch + i] = ok ? sacc / ujj : 0.f;
+      }
+    }
+    for (int c = 0; c < r; ++c) {
+      for (int i = c; i >= 0; --i) {
+        if (U[i * kFPitch + i] == 0.f) { Ui[i * kFPitch + c] = 0.f; continue; }
+        float sacc = (i == c) ? 1.f : 0.f;
+        for (int k = i + 1; k <= c; ++k) sacc -= U[i * kFPitch + k] * Ui[k * kFPitch + c];
+        Ui[i * kFPitch + c] = sacc / U[i * kFPitch + i];
+      }
+      if (U[c * kFPitch + c] == 0.f) for (int i = 0; i <= c; ++i) Ui[i * kFPitch + c] = 0.f;
+    }
+  }
+  __syncwarp();
+  // W (r x r): each lane owns entries lane, lane + 32, ...; the product needs the old W, so read it all first
+  float wn[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const int i = lane + 32 * e, a = i / kMaxRank, b = i % kMaxRank;
+    float v = 0.f;
+    if (a < r && b < r) {
+      if (first) v = Ui[a * kFPitch + b];
+      else for (int k = 0; k < r; ++k) v = fmaf(W[a * kFPitch + k], Ui[k * kFPitch + b], v);
+    }
+    wn[e] = v;
+  }
+  __syncwarp();
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const int i = lane + 32 * e;
+    W[(i / kMaxRank) * kFPitch + i % kMaxRank] = wn[e];
+  }
+  __syncwarp();
+}
+
+template <int BITS, int KMAX>
+__global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const SegDesc& sd = p.seg;
+  const int T = sd.T, n_c = sd.n_c, r = sd.rank;
+  const int side = blockIdx.y, bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  __half* xs = reinterpret_cast<__half*>(smem_raw);                       // [T][kXPitch]
+  unsigned char* cs = smem_raw + round_up(T * kXPitch * 2, 16);          // [T][128]
+  float* rs = reinterpret_cast<float*>(cs + T * kHeadDim);               // [n_c][kRPitch] residual of the whole tile
+  float* Bm = rs + n_c * kRPitch;                                        // [128][kFPitch]
+  float* Am = Bm + kHeadDim * kFPitch;                                   // [n_c][kFPitch]
+  float* Gm = Am + n_c * kFPitch;                                        // [16][kFPitch]
+  float* Um = Gm + kMaxRank * kFPitch;
+  float* Uim = Um + kMaxRank * kFPitch;
+  float* Wm = Uim + kMaxRank * kFPitch;
+  float* wsum = Wm + kMaxRank * kFPitch;                                 // [4]
+  __shared__ unsigned int dmax_bits;
+
+  const __half* Xt = (side == 0 ? p.K : p.V) + (size_t)bh * n_c * kHeadDim;
+  unsigned char* seg_bh = p.arena + sd.seg_base + (size_t)bh * sd.bh_stride;
+
+  // ---- Filter, Quant, pack, residual: block by block (one key group per channel spans one block)
+  for (int blk = 0; blk < sd.nblk; ++blk) {
+    if (tid == 0) dmax_bits = 0u;
+    const __half* X = Xt + (size_t)blk * T * kHeadDim;
+    for (int i = tid; i < T * 16; i += 128) {
+      const int row = i >> 4, c = i & 15;
+      const uint4 v = *reinterpret_cast<const uint4*>(X + row * kHeadDim + c * 8);
+      unsigned int* dst = reinterpret_cast<unsigned int*>(xs + row * kXPitch + c * 8);
+      dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+    }
+    __syncthreads();
+    unsigned char* rec = seg_bh + sd.bfac_bytes + (size_t)blk * sd.rec_bytes;
+    float* rb = rs + (size_t)blk * T * kRPitch;
+    float my_dmax = 0.f;
+    if (side == 0) {
+      const int j = tid, k = sd.k_k;
+      __half* oval = reinterpret_cast<__half*>(rec + sd.off_koval) + j * 2 * k;
+      unsigned char* oidx = rec + sd.off_koidx + j * 2 * k;
+      GroupResult g = process_group<BITS, KMAX>(
+          T, k, [&](int e) { return __half2float(xs[e * kXPitch + j]); },
+          [&](int e, int code, float res) { cs[e * kHeadDim + j] = (unsigned char)code; rb[e * kRPitch + j] = res; },
+          [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
+      reinterpret_cast<__half2*>(rec + sd.off_kscale)[j] = __halves2half2(g.scale, g.zero);
+      my_dmax = g.dmax;
+    } else {
+      const int k = p.cc.k_v, gv = p.cc.g_v, ngv = p.cc.ngv;
+      for (int gi = tid; gi < T * ngv; gi += 128) {
+        const int tok = gi / ngv, c = gi % ngv;
+        __half* oval = reinterpret_cast<__half*>(rec + sd.off_voval) + gi * 2 * k;
+        unsigned char* oidx = rec + sd.off_voidx + gi * 2 * k;
+        GroupResult g = process_group<BITS, KMAX>(
+            gv, k, [&](int e) { return __half2float(xs[tok * kXPitch + c * gv + e]); },
+            [&](int e, int code, float res) {
+              cs[tok * kHeadDim + c * gv + e] = (unsigned char)code;
+              rb[tok * kRPitch + c * gv + e] = res;
+            },
+            [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
+        reinterpret_cast<__half2*>(rec + sd.off_vscale)[gi] = __halves2half2(g.scale, g.zero);
+        my_dmax = fmaxf(my_dmax, g.dmax);
+      }
+    }
+    atomicMax(&dmax_bits, __float_as_uint(my_dmax));
+    __syncthreads();
+    if (tid == 0) reinterpret_cast<float*>(rec)[side] = __uint_as_float(dmax_bits);
+    const int nq = words_per_lane(BITS), hpw = regs_per_word(BITS);
+    const int words_per_slab = 32 * nq;
+    unsigned int* dst = reinterpret_cast<unsigned int*>(rec + (side == 0 ? sd.off_kcodes : sd.off_vcodes));
+    for (int li = tid; li < (T / kSlab) * words_per_slab; li += 128) {
+      const int slab = li / words_per_slab, wl = li % words_per_slab;
+      const int ln = (wl & 127) >> 2, q = (wl >> 7) * 4 + (wl & 3);      // inverse of word_index()
+      unsigned int word = 0;
+      for (int u = 0; u < hpw; ++u)
+        for (int e = 0; e < 2; ++e) {
+          int tok, ch;
+          if (side == 0) code_coord_k(BITS, ln, q, u, e, tok, ch); else code_coord_v(BITS, ln, q, u, e, tok, ch);
+          word |= (unsigned int)cs[(slab * kSlab + tok) * kHeadDim + ch] << (16 * e + BITS * u);
+        }
+      dst[slab * (sd.slab_codes / 4) + wl] = word;
+    }
+    __syncthreads();
+  }
+  if (r == 0) return;
+
+  // ---- Algorithm 2 on the residual in shared memory.  Thread `tid` owns channel tid of B.
+  const size_t gtile = (size_t)bh * 2 + side;
+  float b[kMaxRank];
+#pragma unroll
+  for (int rho = 0; rho < kMaxRank; ++rho) {
+    float v = 0.f;
+    if (rho < r) {
+      if (p.B0 != nullptr) {
+        v = p.B0[(gtile * kHeadDim + tid) * r + rho];
+      } else {
+        const unsigned long long h =
+            mix64(p.seed ^ mix64(((unsigned long long)p.segment_index << 40) ^ (gtile * 4096ull + tid * 16 + rho)));
+        const float u1 = ((float)(unsigned int)(h >> 40) + 1.0f) * (1.0f / 16777217.0f);
+        const float u2 = (float)(unsigned int)((h >> 8) & 0xFFFFFFu) * (1.0f / 16777216.0f);
+        v = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
+      }
+    }
+    b[rho] = v;
+  }
+  for (int l = 0; l < p.iters; ++l) {
+    const bool last = l == p.iters - 1;
+    if (last) {
+      // B <- Q(B): modified Gram-Schmidt, two sweeps per column, then a Newton step on the norm
+#pragma unroll
+      for (int c = 0; c < kMaxRank; ++c) {
+        if (c < r) {
+#pragma unroll
+          for (int sweep = 0; sweep < 2; ++sweep) {
+#pragma unroll
+            for (int q = 0; q < kMaxRank; ++q) {
+              if (q < c) {
+                const float d = block_sum128(b[q] * b[c], wsum, lane, warp);
+                b[c] = fmaf(-d, b[q], b[c]);
+              }
+            }
+          }
+          const float nrm2 = block_sum128(b[c] * b[c], wsum, lane, warp);
+          b[c] = nrm2 > 0.f ? b[c] * rsqrtf(nrm2) : 0.f;
+          const float n2 = block_sum128(b[c] * b[c], wsum, lane, warp);
+          if (n2 > 0.f) b[c] *= (1.5f - 0.5f * n2);
+        }
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int rho = 0; rho < kMaxRank; ++rho) Bm[tid * kFPitch + rho] = b[rho];
+    __syncthreads();
+    // A = R B: one (row, column) of A per thread and round
+    for (int o = tid; o < n_c * r; o += 128) {
+      const int i = o % n_c, rho = o / n_c;
+      const float* rr = rs + i * kRPitch;
+      float acc = 0.f;
+#pragma unroll 8
+      for (int c = 0; c < kHeadDim; ++c) acc = fmaf(rr[c], Bm[c * kFPitch + rho], acc);
+      Am[i * kFPitch + rho] = acc;
+    }
+    __syncthreads();
+    if (last) {
+      // A <- Q(A) by Cholesky QR, twice: Gram matrix, U^-1 of its Cholesky factor, A <- A U^-1
+      for (int round = 0; round < 2; ++round) {
+        for (int o = tid; o < r * r; o += 128) {
+          const int u = o / r, v = o % r;
+          float acc = 0.f;
+          for (int i = 0; i < n_c; ++i) acc = fmaf(Am[i * kFPitch + u], Am[i * kFPitch + v], acc);
+          Gm[u * kFPitch + v] = acc;
+        }
+        __syncthreads();
+        if (warp == 0) chol_update(Gm, Um, Uim, Wm, r, 1, lane);
+        __syncthreads();
+        for (int i = tid; i < n_c; i += 128) {           // one row per thread
+          float a0[kMaxRank], an[kMaxRank];
+#pragma unroll
+          for (int k = 0; k < kMaxRank; ++k) a0[k] = k < r ? Am[i * kFPitch + k] : 0.f;
+#pragma unroll
+          for (int c = 0; c < kMaxRank; ++c) {
+            float acc = 0.f;
+#pragma unroll
+            for (int k = 0; k < kMaxRank; ++k) acc = fmaf(a0[k], (k < r && c < r) ? Wm[k * kFPitch + c] : 0.f, acc);
+            an[c] = acc;
+          }
+#pragma unroll
+          for (int c = 0; c < kMaxRank; ++c) Am[i * kFPitch + c] = an[c];
+          if (round == 1) {
+            // the final A: fp16 in the records (fragment order), fp32 copy on request
+            const int blk = i / T, tib = i % T, slab = tib / kSlab, ts = tib % kSlab;
+            unsigned char* rec = seg_bh + sd.bfac_bytes + (size_t)blk * sd.rec_bytes;
+#pragma unroll
+            for (int c = 0; c < kMaxRank; ++c) {
+              if (c < sd.r_pad) {
+                const float val = c < r ? an[c] : 0.f;
+                if (side == 0)
+                  reinterpret_cast<__half*>(rec + sd.off_ak + slab * sd.slab_a)[ts * sd.r_pad + c] = __float2half_rn(val);
+                else
+                  reinterpret_cast<__half*>(rec + sd.off_av + slab * sd.slab_a)[c * kSlab + ts] = __float2half_rn(val);
+                if (p.dbgA != nullptr && c < r) p.dbgA[(gtile * n_c + i) * r + c] = val;
+              }
+            }
+          }
+        }
+        __syncthreads();
+      }
+    }
+    // B = R^T A: channel tid
+#pragma unroll
+    for (int rho = 0; rho < kMaxRank; ++rho) b[rho] = 0.f;
+    for (int i = 0; i < n_c; ++i) {
+      const float x = rs[i * kRPitch + tid];
+#pragma unroll
+      for (int rho = 0; rho < kMaxRank; ++rho)
+        if (rho < r) b[rho] = fmaf(x, Am[i * kFPitch + rho], b[rho]);
+    }
+  }
+  // ---- store B: fp16 [r_pad][128] for keys, [128][r_pad] for values
+  __half* bf = reinterpret_cast<__half*>(seg_bh);
+#pragma unroll
+  for (int rho = 0; rho < kMaxRank; ++rho) {
+    if (rho < sd.r_pad) {
+      const __half v = __float2half_rn(rho < r ? b[rho] : 0.f);
+      if (side == 0) bf[rho * kHeadDim + tid] = v;
+      else bf[sd.r_pad * kHeadDim + tid * sd.r_pad + rho] = v;
+      if (p.dbgB != nullptr && rho < r) p.dbgB[(gtile * kHeadDim + tid) * r + rho] = b[rho];
+    }
+  }
+}
+
+static size_t tile_smem_bytes(int T, int n_c) {
+  return round_up(T * kXPitch * 2, 16) + (size_t)T * kHeadDim + (size_t)n_c * kRPitch * 4 +
+         (size_t)(kHeadDim + n_c + 4 * kMaxRank) * kFPitch * 4 + 64;
+}
+
+bool compress_tile_fits(int T, int n_c) { return n_c <= kTileMaxTokens && tile_smem_bytes(T, n_c) <= 200 * 1024; }
+
+cudaError_t compress_tile(const CompressJob& job, int BH, cudaStream_t st) {
+  TileArgs a;
+  a.seg = job.seg; a.cc = job.cc; a.arena = job.arena; a.K = job.K; a.V = job.V; a.B0 = job.B0;
+  a.dbgA = job.dbgA; a.dbgB = job.dbgB; a.seed = job.seed; a.segment_index = job.segment_index; a.iters = job.iters;
+  const size_t smem = tile_smem_bytes(job.seg.T, job.seg.n_c);
+  const int kneed = job.seg.k_k > job.cc.k_v ? job.seg.k_k : job.cc.k_v;
+  dim3 grid(BH, 2);
+  cudaError_t e = cudaSuccess;
+#define GEAR_TILE(B, KM)                                                                                          \
+  {                                                                                                               \
+    e = cudaFuncSetAttribute(compress_tile_kernel<B, KM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+    if (e != cudaSuccess) return e;                                                                               \
+    compress_tile_kernel<B, KM><<<grid, 128, smem, st>>>(a);                                                      \
+  }
+  if (job.cc.bits == 2) {
+    if (kneed <= 1) GEAR_TILE(2, 1) else if (kneed <= 2) GEAR_TILE(2, 2) else if (kneed <= 4) GEAR_TILE(2, 4) else GEAR_TILE(2, 8)
+  } else {
+    if (kneed <= 1) GEAR_TILE(4, 1) else if (kneed <= 2) GEAR_TILE(4, 2) else if (kneed <= 4) GEAR_TILE(4, 4) else GEAR_TILE(4, 8)
+  }
+#undef GEAR_TILE
+  count_launches(1);
+  return cudaGetLastError();
+}
+
 // Segment with rank 0: nothing to fit, but the A sections of the records do not exist either.
 // Segment descriptor table entry, written by the device so that no host copy is needed.
 __global__ void write_desc_kernel(SegDesc* table, int* blk2seg, int index, SegDesc d) {
