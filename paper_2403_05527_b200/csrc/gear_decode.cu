@@ -164,13 +164,13 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
   w.ps = o;      o += HP * max_T * 4;
   w.corr_v = o;  o += HP * kHeadDim * 4;
   w.ocorr = o;   o += HP * kHeadDim * 4;
-  w.wl = o;      o += kMaxRank * 8 * 4;
+  w.wl = o;      o += kMaxRank * (HP == 1 ? 1 : 8) * 4 + 16;
   w.misc = o;    o += 64;
   w.ring = round_up(o, 16);
   // most resident warps (in steps of four: one per scheduler) whose ring still holds two stages; then as many
   // stages as fit
-  const int reg_limit = HP == 1 ? 16 : (HP == 4 ? 12 : 6);
-  for (int warps = reg_limit; warps >= 1; warps -= (warps > 4 ? 4 : 1)) {
+  const int reg_limit = HP == 1 ? 16 : (HP == 4 ? 8 : 6);
+  for (int warps = reg_limit; warps >= 1; warps -= (warps > 8 ? 4 : 1)) {
     const long long per = (long long)smem_budget / warps - 1024;     // the system reserves 1 KB per CTA
     long long ns = (per - w.ring) / stage;
     if (ns < 2) continue;
@@ -240,13 +240,15 @@ int static_shape_id(const SegDesc& s, const CacheConst& c) {
 // ------------------------------------------------------------------ the kernel
 // HEADS = query heads handled per pass: 1 (multi-head attention), 4 or 8 (grouped queries; a pass may hold fewer).
 template <int BITS, int HEADS, int NGV>
-__global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) gear_decode_kernel(const __grid_constant__ DecodeArgs a) {
+__global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) gear_decode_kernel(const __grid_constant__ DecodeArgs a) {
   constexpr int HP = HEADS;
   constexpr int NT = HEADS > 4 ? 2 : 1;           // 8-column tiles of the B operand
   constexpr int GV = kHeadDim / NGV;              // channels per value group
   constexpr int SLABW = kSlab * kHeadDim * BITS / 8 / 16;   // uint4 per slab of codes
   constexpr int kFragStride = frag_row_words(HP);
   constexpr int CMASK = HP == 1 ? 1 : 7;          // fragment columns that exist, as a mask on the lane's column
+  constexpr int WLS = HP == 1 ? 1 : 8;            // row stride of the small factor exchange buffer wl[16][heads]
+  constexpr int HMASK = HP == 1 ? 0 : 7;          // heads that exist in wl, as a mask on the lane's head
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ __align__(8) uint64_t bar[kMaxStages];
 
@@ -264,7 +266,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
   float* ps = reinterpret_cast<float*>(smem + a.ws.ps);          // [HP][maxT] scores, then probabilities
   int* corr_v = reinterpret_cast<int*>(smem + a.ws.corr_v);      // [HP][128]
   float* ocorr = reinterpret_cast<float*>(smem + a.ws.ocorr);    // [HP][128]
-  float* wl = reinterpret_cast<float*>(smem + a.ws.wl);          // [16][8]
+  float* wl = reinterpret_cast<float*>(smem + a.ws.wl);          // [16][heads]
   int* qexp_s = reinterpret_cast<int*>(smem + a.ws.misc);        // [HP]
 
   if (lane == 0)
@@ -496,16 +498,18 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
         __syncwarp();
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {       // D[rho][col 2t] = w[rho][head t + 4nt]
-          wl[gid * 8 + t + 4 * nt] = wacc[nt][0] * a.scale_log2;
-          wl[(gid + 8) * 8 + t + 4 * nt] = wacc[nt][2] * a.scale_log2;
+          if (t + 4 * nt < HP) {
+            wl[gid * WLS + t + 4 * nt] = wacc[nt][0] * a.scale_log2;
+            wl[(gid + 8) * WLS + t + 4 * nt] = wacc[nt][2] * a.scale_log2;
+          }
         }
         __syncwarp();
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           const int h = (gid >> 1) + 4 * nt;
           uint32_t hi0, lo0, hi1, lo1;
-          split_hi_lo(wl[(2 * t) * 8 + h], wl[(2 * t + 1) * 8 + h], hi0, lo0);
-          split_hi_lo(wl[(2 * t + 8) * 8 + h], wl[(2 * t + 9) * 8 + h], hi1, lo1);
+          split_hi_lo(wl[(2 * t) * WLS + (h & HMASK)], wl[(2 * t + 1) * WLS + (h & HMASK)], hi0, lo0);
+          split_hi_lo(wl[(2 * t + 8) * WLS + (h & HMASK)], wl[(2 * t + 9) * WLS + (h & HMASK)], hi1, lo1);
           bw[nt][0] = (gid & 1) ? lo0 : hi0;
           bw[nt][1] = (gid & 1) ? lo1 : hi1;
         }
@@ -952,8 +956,10 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
         __syncwarp();
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          wl[gid * 8 + t + 4 * nt] = U[nt][0] + U[nt][1];
-          wl[(gid + 8) * 8 + t + 4 * nt] = U[nt][2] + U[nt][3];
+          if (t + 4 * nt < HP) {
+            wl[gid * WLS + t + 4 * nt] = U[nt][0] + U[nt][1];
+            wl[(gid + 8) * WLS + t + 4 * nt] = U[nt][2] + U[nt][3];
+          }
 #pragma unroll
           for (int i = 0; i < 4; ++i) U[nt][i] = 0.f;
         }
@@ -963,8 +969,8 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 12 : 6)) g
         for (int nt = 0; nt < NT; ++nt) {
           const int h = (gid >> 1) + 4 * nt;
           uint32_t hi0, lo0, hi1, lo1;
-          split_hi_lo(wl[(2 * t) * 8 + h], wl[(2 * t + 1) * 8 + h], hi0, lo0);
-          split_hi_lo(wl[(2 * t + 8) * 8 + h], wl[(2 * t + 9) * 8 + h], hi1, lo1);
+          split_hi_lo(wl[(2 * t) * WLS + (h & HMASK)], wl[(2 * t + 1) * WLS + (h & HMASK)], hi0, lo0);
+          split_hi_lo(wl[(2 * t + 8) * WLS + (h & HMASK)], wl[(2 * t + 9) * WLS + (h & HMASK)], hi1, lo1);
           bu[nt][0] = (gid & 1) ? lo0 : hi0;
           bu[nt][1] = (gid & 1) ? lo1 : hi1;
         }
