@@ -316,7 +316,7 @@ def run_ours(args, w):
         in_bytes = 2 * B * w.n_kv_heads * w.n * 128 * 2
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f16 codes x f16 hi/lo queries, f32 accumulate",
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32",
                 "data": "synthetic",
                 "config": {"workload": workload_name(w, L), "batch_per_gpu": B, "layers_rotated": L,
                            "l2": "rotating caches: %.0f MB touched between reuses" % (dec_bytes / len(dec_ms) * L / 1e6)},
