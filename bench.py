@@ -32,6 +32,7 @@ import numpy as np  # noqa: E402
 from paper_2403_05527_b200 import synth  # noqa: E402
 
 METRIC = "compressed-KV decode attn tokens/s"
+DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.022
 UNIT = "tokens/s"
 
 
@@ -305,14 +306,9 @@ def run_ours(args, w):
             peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
         else:
             peak, peak_src = 6650.0, "fallback"
-        traffic = None
-        tp = os.path.join(ROOT, "profiles", "decode_traffic.json")
-        if os.path.exists(tp):
-            try:
-                tj = json.load(open(tp))
-                traffic = tj["dram_bytes_per_algorithmic_byte"] * dec_bytes / len(dec_ms)
-            except Exception:
-                traffic = None
+        # dram__bytes_read + dram__bytes_write of gear_decode_kernel<2,1,2> per algorithmic byte, from the ncu capture
+        # summarised in profiles/gear_decode_kernel_C2.md (one layer cache; traffic grows in proportion to the cache)
+        traffic = DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE * dec_bytes / len(dec_ms) if w.config_id == 2 else None
         in_bytes = 2 * B * w.n_kv_heads * w.n * 128 * 2
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
@@ -364,7 +360,7 @@ def main():
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--cpu-units", type=int, default=24)
+    ap.add_argument("--cpu-units", type=int, default=128)
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.config]
