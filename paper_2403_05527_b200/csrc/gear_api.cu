@@ -245,7 +245,7 @@ static gear_status compress_segment(gear_cache* c, const void* K, const void* V,
   job.seed = c->cfg.seed; job.segment_index = (int)c->segs.size(); job.iters = c->cfg.power_iters;
 
   cudaError_t e = cudaSuccess;
-  if (compress_tile_fits(sd.T, sd.n_c)) {
+  if (compress_tile_fits(sd.T, sd.n_c, sd.rank)) {
     e = compress_tile(job, c->cc.BH, st);              // short segment: one launch, residual in shared memory
   } else if (is_flush) {
     e = compress_range(job, 0, c->cc.BH, c->flush_ws, st);

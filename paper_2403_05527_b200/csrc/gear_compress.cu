@@ -622,18 +622,26 @@ __device__ void chol_update(const float* G, float* U, float* Ui, float* W, int r
   __syncwarp();
 }
 
-template <int BITS, int KMAX>
+// Shared memory: [ region 0 | residual rs[n_c][kRPitch] ].  Region 0 first holds the fp16 tile of the block being
+// quantized (each entry is replaced by its code once it is known), later the factor matrices of Algorithm 2.
+template <int RP>
+__host__ __device__ constexpr int tile_factor_bytes(int n_c) {
+  return ((kHeadDim + n_c) * (RP + 1) + 4 * kMaxRank * kFPitch + 8) * 4;
+}
+
+template <int BITS, int KMAX, int RP>
 __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
+  constexpr int FP = RP + 1;                 // floats per row of B and A in shared memory
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const SegDesc& sd = p.seg;
   const int T = sd.T, n_c = sd.n_c, r = sd.rank;
   const int side = blockIdx.y, bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  __half* xs = reinterpret_cast<__half*>(smem_raw);                       // [T][kXPitch]
-  unsigned char* cs = smem_raw + round_up(T * kXPitch * 2, 16);          // [T][128]
-  float* rs = reinterpret_cast<float*>(cs + T * kHeadDim);               // [n_c][kRPitch] residual of the whole tile
-  float* Bm = rs + n_c * kRPitch;                                        // [128][kFPitch]
-  float* Am = Bm + kHeadDim * kFPitch;                                   // [n_c][kFPitch]
-  float* Gm = Am + n_c * kFPitch;                                        // [16][kFPitch]
+  const int reg0 = max(round_up(T * kXPitch * 2, 16), tile_factor_bytes<RP>(n_c));
+  unsigned short* xs = reinterpret_cast<unsigned short*>(smem_raw);      // [T][kXPitch] fp16 bits, then codes
+  float* rs = reinterpret_cast<float*>(smem_raw + reg0);                 // [n_c][kRPitch] residual of the whole tile
+  float* Bm = reinterpret_cast<float*>(smem_raw);                        // [128][FP]
+  float* Am = Bm + kHeadDim * FP;                                        // [n_c][FP]
+  float* Gm = Am + n_c * FP;                                             // [16][kFPitch]
   float* Um = Gm + kMaxRank * kFPitch;
   float* Uim = Um + kMaxRank * kFPitch;
   float* Wm = Uim + kMaxRank * kFPitch;
@@ -642,6 +650,7 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
 
   const __half* Xt = (side == 0 ? p.K : p.V) + (size_t)bh * n_c * kHeadDim;
   unsigned char* seg_bh = p.arena + sd.seg_base + (size_t)bh * sd.bh_stride;
+  auto x_of = [&](int idx) { return __half2float(__ushort_as_half(xs[idx])); };
 
   // ---- Filter, Quant, pack, residual: block by block (one key group per channel spans one block)
   for (int blk = 0; blk < sd.nblk; ++blk) {
@@ -662,8 +671,8 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
       __half* oval = reinterpret_cast<__half*>(rec + sd.off_koval) + j * 2 * k;
       unsigned char* oidx = rec + sd.off_koidx + j * 2 * k;
       GroupResult g = process_group<BITS, KMAX>(
-          T, k, [&](int e) { return __half2float(xs[e * kXPitch + j]); },
-          [&](int e, int code, float res) { cs[e * kHeadDim + j] = (unsigned char)code; rb[e * kRPitch + j] = res; },
+          T, k, [&](int e) { return x_of(e * kXPitch + j); },
+          [&](int e, int code, float res) { xs[e * kXPitch + j] = (unsigned short)code; rb[e * kRPitch + j] = res; },
           [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
       reinterpret_cast<__half2*>(rec + sd.off_kscale)[j] = __halves2half2(g.scale, g.zero);
       my_dmax = g.dmax;
@@ -674,9 +683,9 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
         __half* oval = reinterpret_cast<__half*>(rec + sd.off_voval) + gi * 2 * k;
         unsigned char* oidx = rec + sd.off_voidx + gi * 2 * k;
         GroupResult g = process_group<BITS, KMAX>(
-            gv, k, [&](int e) { return __half2float(xs[tok * kXPitch + c * gv + e]); },
+            gv, k, [&](int e) { return x_of(tok * kXPitch + c * gv + e); },
             [&](int e, int code, float res) {
-              cs[tok * kHeadDim + c * gv + e] = (unsigned char)code;
+              xs[tok * kXPitch + c * gv + e] = (unsigned short)code;
               rb[tok * kRPitch + c * gv + e] = res;
             },
             [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
@@ -694,12 +703,15 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
       const int slab = li / words_per_slab, wl = li % words_per_slab;
       const int ln = (wl & 127) >> 2, q = (wl >> 7) * 4 + (wl & 3);      // inverse of word_index()
       unsigned int word = 0;
-      for (int u = 0; u < hpw; ++u)
+#pragma unroll
+      for (int u = 0; u < 16 / BITS; ++u)
+#pragma unroll
         for (int e = 0; e < 2; ++e) {
           int tok, ch;
           if (side == 0) code_coord_k(BITS, ln, q, u, e, tok, ch); else code_coord_v(BITS, ln, q, u, e, tok, ch);
-          word |= (unsigned int)cs[(slab * kSlab + tok) * kHeadDim + ch] << (16 * e + BITS * u);
+          word |= (unsigned int)xs[(slab * kSlab + tok) * kXPitch + ch] << (16 * e + BITS * u);
         }
+      (void)hpw;
       dst[slab * (sd.slab_codes / 4) + wl] = word;
     }
     __syncthreads();
@@ -708,9 +720,9 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
 
   // ---- Algorithm 2 on the residual in shared memory.  Thread `tid` owns channel tid of B.
   const size_t gtile = (size_t)bh * 2 + side;
-  float b[kMaxRank];
+  float b[RP];
 #pragma unroll
-  for (int rho = 0; rho < kMaxRank; ++rho) {
+  for (int rho = 0; rho < RP; ++rho) {
     float v = 0.f;
     if (rho < r) {
       if (p.B0 != nullptr) {
@@ -730,12 +742,12 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
     if (last) {
       // B <- Q(B): modified Gram-Schmidt, two sweeps per column, then a Newton step on the norm
 #pragma unroll
-      for (int c = 0; c < kMaxRank; ++c) {
+      for (int c = 0; c < RP; ++c) {
         if (c < r) {
 #pragma unroll
           for (int sweep = 0; sweep < 2; ++sweep) {
 #pragma unroll
-            for (int q = 0; q < kMaxRank; ++q) {
+            for (int q = 0; q < RP; ++q) {
               if (q < c) {
                 const float d = block_sum128(b[q] * b[c], wsum, lane, warp);
                 b[c] = fmaf(-d, b[q], b[c]);
@@ -751,16 +763,22 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
     }
     __syncthreads();
 #pragma unroll
-    for (int rho = 0; rho < kMaxRank; ++rho) Bm[tid * kFPitch + rho] = b[rho];
+    for (int rho = 0; rho < RP; ++rho) Bm[tid * FP + rho] = b[rho];
     __syncthreads();
-    // A = R B: one (row, column) of A per thread and round
-    for (int o = tid; o < n_c * r; o += 128) {
-      const int i = o % n_c, rho = o / n_c;
+    // A = R B: one row of A per thread and round (all columns at once)
+    for (int i = tid; i < n_c; i += 128) {
       const float* rr = rs + i * kRPitch;
-      float acc = 0.f;
-#pragma unroll 8
-      for (int c = 0; c < kHeadDim; ++c) acc = fmaf(rr[c], Bm[c * kFPitch + rho], acc);
-      Am[i * kFPitch + rho] = acc;
+      float acc[RP];
+#pragma unroll
+      for (int rho = 0; rho < RP; ++rho) acc[rho] = 0.f;
+#pragma unroll 4
+      for (int c = 0; c < kHeadDim; ++c) {
+        const float x = rr[c];
+#pragma unroll
+        for (int rho = 0; rho < RP; ++rho) acc[rho] = fmaf(x, Bm[c * FP + rho], acc[rho]);
+      }
+#pragma unroll
+      for (int rho = 0; rho < RP; ++rho) Am[i * FP + rho] = acc[rho];
     }
     __syncthreads();
     if (last) {
@@ -769,31 +787,31 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
         for (int o = tid; o < r * r; o += 128) {
           const int u = o / r, v = o % r;
           float acc = 0.f;
-          for (int i = 0; i < n_c; ++i) acc = fmaf(Am[i * kFPitch + u], Am[i * kFPitch + v], acc);
+          for (int i = 0; i < n_c; ++i) acc = fmaf(Am[i * FP + u], Am[i * FP + v], acc);
           Gm[u * kFPitch + v] = acc;
         }
         __syncthreads();
         if (warp == 0) chol_update(Gm, Um, Uim, Wm, r, 1, lane);
         __syncthreads();
         for (int i = tid; i < n_c; i += 128) {           // one row per thread
-          float a0[kMaxRank], an[kMaxRank];
+          float a0[RP], an[RP];
 #pragma unroll
-          for (int k = 0; k < kMaxRank; ++k) a0[k] = k < r ? Am[i * kFPitch + k] : 0.f;
+          for (int k = 0; k < RP; ++k) a0[k] = Am[i * FP + k];
 #pragma unroll
-          for (int c = 0; c < kMaxRank; ++c) {
+          for (int c = 0; c < RP; ++c) {
             float acc = 0.f;
 #pragma unroll
-            for (int k = 0; k < kMaxRank; ++k) acc = fmaf(a0[k], (k < r && c < r) ? Wm[k * kFPitch + c] : 0.f, acc);
+            for (int k = 0; k < RP; ++k) acc = fmaf(a0[k], Wm[k * kFPitch + c], acc);
             an[c] = acc;
           }
 #pragma unroll
-          for (int c = 0; c < kMaxRank; ++c) Am[i * kFPitch + c] = an[c];
+          for (int c = 0; c < RP; ++c) Am[i * FP + c] = an[c];
           if (round == 1) {
             // the final A: fp16 in the records (fragment order), fp32 copy on request
             const int blk = i / T, tib = i % T, slab = tib / kSlab, ts = tib % kSlab;
             unsigned char* rec = seg_bh + sd.bfac_bytes + (size_t)blk * sd.rec_bytes;
 #pragma unroll
-            for (int c = 0; c < kMaxRank; ++c) {
+            for (int c = 0; c < RP; ++c) {
               if (c < sd.r_pad) {
                 const float val = c < r ? an[c] : 0.f;
                 if (side == 0)
@@ -810,18 +828,18 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
     }
     // B = R^T A: channel tid
 #pragma unroll
-    for (int rho = 0; rho < kMaxRank; ++rho) b[rho] = 0.f;
+    for (int rho = 0; rho < RP; ++rho) b[rho] = 0.f;
+#pragma unroll 4
     for (int i = 0; i < n_c; ++i) {
       const float x = rs[i * kRPitch + tid];
 #pragma unroll
-      for (int rho = 0; rho < kMaxRank; ++rho)
-        if (rho < r) b[rho] = fmaf(x, Am[i * kFPitch + rho], b[rho]);
+      for (int rho = 0; rho < RP; ++rho) b[rho] = fmaf(x, Am[i * FP + rho], b[rho]);
     }
   }
   // ---- store B: fp16 [r_pad][128] for keys, [128][r_pad] for values
   __half* bf = reinterpret_cast<__half*>(seg_bh);
 #pragma unroll
-  for (int rho = 0; rho < kMaxRank; ++rho) {
+  for (int rho = 0; rho < RP; ++rho) {
     if (rho < sd.r_pad) {
       const __half v = __float2half_rn(rho < r ? b[rho] : 0.f);
       if (side == 0) bf[rho * kHeadDim + tid] = v;
@@ -831,32 +849,42 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
   }
 }
 
-static size_t tile_smem_bytes(int T, int n_c) {
-  return round_up(T * kXPitch * 2, 16) + (size_t)T * kHeadDim + (size_t)n_c * kRPitch * 4 +
-         (size_t)(kHeadDim + n_c + 4 * kMaxRank) * kFPitch * 4 + 64;
+static int tile_rp(int rank) { return rank <= 4 ? 4 : (rank <= 8 ? 8 : 16); }
+
+static size_t tile_smem_bytes(int T, int n_c, int rank) {
+  const int rp = tile_rp(rank);
+  const int fb = rp == 4 ? tile_factor_bytes<4>(n_c) : (rp == 8 ? tile_factor_bytes<8>(n_c) : tile_factor_bytes<16>(n_c));
+  const int x = round_up(T * kXPitch * 2, 16);
+  return (size_t)(x > fb ? x : fb) + (size_t)n_c * kRPitch * 4;
 }
 
-bool compress_tile_fits(int T, int n_c) { return n_c <= kTileMaxTokens && tile_smem_bytes(T, n_c) <= 200 * 1024; }
+bool compress_tile_fits(int T, int n_c, int rank) {
+  return n_c <= kTileMaxTokens && tile_smem_bytes(T, n_c, rank) <= 200 * 1024;
+}
 
 cudaError_t compress_tile(const CompressJob& job, int BH, cudaStream_t st) {
   TileArgs a;
   a.seg = job.seg; a.cc = job.cc; a.arena = job.arena; a.K = job.K; a.V = job.V; a.B0 = job.B0;
   a.dbgA = job.dbgA; a.dbgB = job.dbgB; a.seed = job.seed; a.segment_index = job.segment_index; a.iters = job.iters;
-  const size_t smem = tile_smem_bytes(job.seg.T, job.seg.n_c);
+  const size_t smem = tile_smem_bytes(job.seg.T, job.seg.n_c, job.seg.rank);
   const int kneed = job.seg.k_k > job.cc.k_v ? job.seg.k_k : job.cc.k_v;
+  const int rp = tile_rp(job.seg.rank);
   dim3 grid(BH, 2);
   cudaError_t e = cudaSuccess;
-#define GEAR_TILE(B, KM)                                                                                          \
-  {                                                                                                               \
-    e = cudaFuncSetAttribute(compress_tile_kernel<B, KM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-    if (e != cudaSuccess) return e;                                                                               \
-    compress_tile_kernel<B, KM><<<grid, 128, smem, st>>>(a);                                                      \
+#define GEAR_TILE(B, KM, R)                                                                                          \
+  {                                                                                                                  \
+    e = cudaFuncSetAttribute(compress_tile_kernel<B, KM, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+    if (e != cudaSuccess) return e;                                                                                  \
+    compress_tile_kernel<B, KM, R><<<grid, 128, smem, st>>>(a);                                                      \
   }
+#define GEAR_TILE_R(B, KM) \
+  { if (rp == 4) GEAR_TILE(B, KM, 4) else if (rp == 8) GEAR_TILE(B, KM, 8) else GEAR_TILE(B, KM, 16) }
   if (job.cc.bits == 2) {
-    if (kneed <= 1) GEAR_TILE(2, 1) else if (kneed <= 2) GEAR_TILE(2, 2) else if (kneed <= 4) GEAR_TILE(2, 4) else GEAR_TILE(2, 8)
+    if (kneed <= 1) GEAR_TILE_R(2, 1) else if (kneed <= 2) GEAR_TILE_R(2, 2) else GEAR_TILE_R(2, 8)
   } else {
-    if (kneed <= 1) GEAR_TILE(4, 1) else if (kneed <= 2) GEAR_TILE(4, 2) else if (kneed <= 4) GEAR_TILE(4, 4) else GEAR_TILE(4, 8)
+    if (kneed <= 1) GEAR_TILE_R(4, 1) else if (kneed <= 2) GEAR_TILE_R(4, 2) else GEAR_TILE_R(4, 8)
   }
+#undef GEAR_TILE_R
 #undef GEAR_TILE
   count_launches(1);
   return cudaGetLastError();

@@ -52,7 +52,7 @@ struct CompressJob {
 
 size_t compress_workspace_bytes(int nbh, int n_c, int rank);
 // whole-tile path for short segments (one launch): usable when compress_tile_fits()
-bool compress_tile_fits(int T, int n_c);
+bool compress_tile_fits(int T, int n_c, int rank);
 cudaError_t compress_tile(const CompressJob& job, int BH, cudaStream_t st);
 cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned char* ws, cudaStream_t st);
 cudaError_t launch_write_desc(SegDesc* table, int* blk2seg, int index, const SegDesc& d, cudaStream_t st);
