@@ -65,17 +65,34 @@ __device__ __forceinline__ GroupResult process_group(int len, int k, XAt x_at, P
   TopList top, bot;
 #pragma unroll
   for (int s = 0; s < KMAX; ++s) { top.v[s] = 0.f; top.i[s] = -1; bot.v[s] = 0.f; bot.i[s] = -1; }
-  if (k > 0) {
-    for (int e = 0; e < len; ++e) list_insert<KMAX, true>(top, k, x_at(e), e);
-    for (int e = 0; e < len; ++e)
-      if (!list_has<KMAX>(top, k, e)) list_insert<KMAX, false>(bot, k, x_at(e), e);
-  }
   float mn = INFINITY, mx = -INFINITY;
-  for (int e = 0; e < len; ++e) {
-    if (k > 0 && (list_has<KMAX>(top, k, e) || list_has<KMAX>(bot, k, e))) continue;
-    const float x = x_at(e);
-    mn = fminf(mn, x);
-    mx = fmaxf(mx, x);
+  if (KMAX == 1 && k == 1) {
+    // One outlier per side: a single pass finds the first maximum, the first minimum and the second largest /
+    // second smallest instances, which bound the kept entries.  (The first maximum is also the first minimum
+    // only when all entries are equal; the bottom entry is then the next index.)
+    float max1 = -INFINITY, max2 = -INFINITY, min1 = INFINITY, min2 = INFINITY;
+    int imax = 0, imin = 0;
+    for (int e = 0; e < len; ++e) {
+      const float x = x_at(e);
+      if (x > max1) { max2 = max1; max1 = x; imax = e; } else if (x > max2) { max2 = x; }
+      if (x < min1) { min2 = min1; min1 = x; imin = e; } else if (x < min2) { min2 = x; }
+    }
+    if (imin == imax) imin = 1;
+    top.v[0] = max1; top.i[0] = imax;
+    bot.v[0] = min1; bot.i[0] = imin;
+    mn = min2; mx = max2;
+  } else {
+    if (k > 0) {
+      for (int e = 0; e < len; ++e) list_insert<KMAX, true>(top, k, x_at(e), e);
+      for (int e = 0; e < len; ++e)
+        if (!list_has<KMAX>(top, k, e)) list_insert<KMAX, false>(bot, k, x_at(e), e);
+    }
+    for (int e = 0; e < len; ++e) {
+      if (k > 0 && (list_has<KMAX>(top, k, e) || list_has<KMAX>(bot, k, e))) continue;
+      const float x = x_at(e);
+      mn = fminf(mn, x);
+      mx = fmaxf(mx, x);
+    }
   }
   // Eq. 2 on the kept entries: binary32, one rounding per operation.
   const float levels = (float)((1 << BITS) - 1);
@@ -130,9 +147,9 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
   const SegDesc& sd = p.seg;
   const int T = sd.T;
   const int side = blockIdx.z, bhl = blockIdx.y, blk = blockIdx.x, tid = threadIdx.x;
-  __half* xs = reinterpret_cast<__half*>(smem_raw);
-  unsigned char* cs = smem_raw + round_up(T * kXPitch * 2, 16);
-  float* rs = reinterpret_cast<float*>(cs + T * kHeadDim);
+  unsigned short* xs = reinterpret_cast<unsigned short*>(smem_raw);   // fp16 bits of the block; each entry is replaced by its code
+  float* rs = reinterpret_cast<float*>(smem_raw + round_up(T * kXPitch * 2, 16));
+  auto x_of = [&](int idx) { return __half2float(__ushort_as_half(xs[idx])); };
   __shared__ unsigned int dmax_bits;
   if (tid == 0) dmax_bits = 0u;
 
@@ -155,8 +172,8 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
     __half* oval = reinterpret_cast<__half*>(rec + sd.off_koval) + j * 2 * k;
     unsigned char* oidx = rec + sd.off_koidx + j * 2 * k;
     GroupResult g = process_group<BITS, KMAX>(
-        T, k, [&](int e) { return __half2float(xs[e * kXPitch + j]); },
-        [&](int e, int code, float r) { cs[e * kHeadDim + j] = (unsigned char)code; rs[e * kRPitch + j] = r; },
+        T, k, [&](int e) { return x_of(e * kXPitch + j); },
+        [&](int e, int code, float r) { xs[e * kXPitch + j] = (unsigned short)code; rs[e * kRPitch + j] = r; },
         [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
     reinterpret_cast<__half2*>(rec + sd.off_kscale)[j] = __halves2half2(g.scale, g.zero);
     my_dmax = g.dmax;
@@ -168,9 +185,9 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
       __half* oval = reinterpret_cast<__half*>(rec + sd.off_voval) + gi * 2 * k;
       unsigned char* oidx = rec + sd.off_voidx + gi * 2 * k;
       GroupResult g = process_group<BITS, KMAX>(
-          gv, k, [&](int e) { return __half2float(xs[tok * kXPitch + c * gv + e]); },
+          gv, k, [&](int e) { return x_of(tok * kXPitch + c * gv + e); },
           [&](int e, int code, float r) {
-            cs[tok * kHeadDim + c * gv + e] = (unsigned char)code;
+            xs[tok * kXPitch + c * gv + e] = (unsigned short)code;
             rs[tok * kRPitch + c * gv + e] = r;
           },
           [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
@@ -194,7 +211,7 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
       for (int e = 0; e < 2; ++e) {
         int tok, ch;
         if (side == 0) code_coord_k(BITS, lane, q, u, e, tok, ch); else code_coord_v(BITS, lane, q, u, e, tok, ch);
-        word |= (unsigned int)cs[(slab * kSlab + tok) * kHeadDim + ch] << (16 * e + BITS * u);
+        word |= (unsigned int)xs[(slab * kSlab + tok) * kXPitch + ch] << (16 * e + BITS * u);
       }
     dst[slab * (sd.slab_codes / 4) + wl] = word;
   }
@@ -913,7 +930,7 @@ __global__ void append_kernel(__half* buf_k, __half* buf_v, const __half* k_new,
 template <int BITS>
 static cudaError_t launch_quant(const CompressArgs& a, int nbh, int kmax_needed, cudaStream_t st) {
   const int T = a.seg.T;
-  const size_t smem = round_up(T * kXPitch * 2, 16) + (size_t)T * kHeadDim + (size_t)T * kRPitch * 4;
+  const size_t smem = round_up(T * kXPitch * 2, 16) + (size_t)T * kRPitch * 4;
   dim3 grid(a.seg.nblk, nbh, 2);
 #define GEAR_LAUNCH_Q(KM)                                                                                   \
   {                                                                                                         \
