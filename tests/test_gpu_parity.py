@@ -178,3 +178,27 @@ def test_fp16_cache_attention_against_textbook():
             w = np.exp(z - z.max()); w /= w.sum()
             ref = w @ vv
             assert np.abs(got[b, h] - ref).max() / np.abs(ref).max() <= 1e-3
+
+
+def test_ties_and_constant_groups_follow_the_fixed_tie_break(pair_factory):
+    """Inputs drawn from a handful of values (plus constant rows and columns): almost every group has ties among
+    its extremes, and some groups are constant.  Outlier sets and codes must still match the oracle bit for bit:
+    larger value first, then lower index; the top entry chosen before the bottom one."""
+    import torch
+    from paper_2403_05527_b200 import binding as G
+    for bits, group, s_pct, n in ((2, 64, 2.0, 128), (4, 32, 4.0, 64), (2, 128, 2.0, 256)):
+        p = pair_factory(11, 1, 2, 2, bits, group, s_pct, 64 if group != 32 else 32, 2, 512, r_max=2)
+        gen = np.random.default_rng(bits * 100 + group)
+        k16 = gen.choice(np.array([-2.0, -0.5, 0.0, -0.0, 0.25, 1.0, 3.0], np.float16), size=(1, 2, n, 128))
+        v16 = gen.choice(np.array([-1.0, 0.0, 0.5, 0.5, 2.0], np.float16), size=(1, 2, n, 128))
+        k16[0, 0, :, 5] = np.float16(1.5)            # a constant key column (one constant group per block)
+        v16[0, 1, 7, :] = np.float16(-0.75)          # a constant value row
+        b0 = gen.standard_normal((1, 2, 2, 128, 2)).astype(np.float32)
+        p.oracle.compress(k16, v16, 2, b0)
+        dev = p.dev
+        G.gear_compress(p.cache, None, torch.from_numpy(k16).to(dev), torch.from_numpy(v16).to(dev), n, 2,
+                        torch.from_numpy(b0).to(dev))
+        torch.cuda.synchronize()
+        p.check_segment(0)
+        p.check_attention()
+        p.close()
