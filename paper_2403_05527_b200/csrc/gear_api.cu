@@ -197,7 +197,7 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   const size_t units = BH * passes;
   const size_t nw_max = (size_t)c->sm_count * 32;        // one warp per CTA, at most 32 CTAs per SM
   c->max_parts = (int)(nw_max / units + 3);
-  c->partial_bytes = units * c->max_parts * (size_t)hp * 130 * 4;
+  c->partial_bytes = units * c->max_parts * (size_t)hp * kPartRow * 4;
   GEAR_TRY_ALLOC(c->partial, c->partial_bytes);
   GEAR_TRY_ALLOC(c->tickets, units * 4);
   GEAR_TRY_ALLOC(c->status, 4);

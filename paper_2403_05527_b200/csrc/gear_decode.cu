@@ -1011,7 +1011,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
     const long long w_last = (eflat * NW + F - 1) / F - 1;
     const int n_parts = (int)(w_last - w_first + 1);
     const int slot = (int)(blockIdx.x - w_first);
-    float* part_base = a.partial + ((size_t)u * a.max_parts + slot) * (HP * 130);
+    float* part_base = a.partial + ((size_t)u * a.max_parts + slot) * (HP * kPartRow);
     float cm_own[NT][NGV], m_own[NT], l_own[NT];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -1038,7 +1038,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
     for (int nt = 0; nt < NT; ++nt) {
       const int h = t + 4 * nt;
       if (h < HPu) {
-        float* dst = part_base + h * 130;
+        float* dst = part_base + h * kPartRow;
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt)
 #pragma unroll
@@ -1056,22 +1056,38 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
     last = __shfl_sync(0xffffffffu, last, 0);
     if (last) {
       __threadfence();
-      const float* pb = a.partial + (size_t)u * a.max_parts * (HP * 130);
+      const float* pb = a.partial + (size_t)u * a.max_parts * (HP * kPartRow);
+      const size_t pstride = (size_t)HP * kPartRow;
       for (int h = 0; h < HPu; ++h) {
+        // lane i looks at partial i (+32, ...): running maxima first, then weights and the weighted sums
         float M = -INFINITY;
-        for (int i = 0; i < n_parts; ++i) M = fmaxf(M, __ldcg(pb + (size_t)i * HP * 130 + h * 130 + 128));
-        float den = 0.f, n0 = 0.f, n1 = 0.f, n2 = 0.f, n3 = 0.f;
-        for (int i = 0; i < n_parts; ++i) {
-          const float* pp = pb + (size_t)i * HP * 130 + h * 130;
-          const float mi = __ldcg(pp + 128);
-          if (mi == -INFINITY) continue;
-          const float wgt = exp2f(mi - M);
-          den = fmaf(wgt, __ldcg(pp + 129), den);
-          n0 = fmaf(wgt, __ldcg(pp + lane * 4 + 0), n0);
-          n1 = fmaf(wgt, __ldcg(pp + lane * 4 + 1), n1);
-          n2 = fmaf(wgt, __ldcg(pp + lane * 4 + 2), n2);
-          n3 = fmaf(wgt, __ldcg(pp + lane * 4 + 3), n3);
+        for (int base = 0; base < n_parts; base += 32) {
+          const int i = base + lane;
+          if (i < n_parts) M = fmaxf(M, __ldcg(pb + i * pstride + h * kPartRow + 128));
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        float den = 0.f, n0 = 0.f, n1 = 0.f, n2 = 0.f, n3 = 0.f;
+        for (int base = 0; base < n_parts; base += 32) {
+          const int i = base + lane;
+          float wgt = 0.f;
+          if (i < n_parts) {
+            const float mi = __ldcg(pb + i * pstride + h * kPartRow + 128);
+            if (mi != -INFINITY) {
+              wgt = exp2f(mi - M);
+              den = fmaf(wgt, __ldcg(pb + i * pstride + h * kPartRow + 129), den);
+            }
+          }
+          const int cnt = min(32, n_parts - base);
+#pragma unroll 4
+          for (int j = 0; j < cnt; ++j) {
+            const float wj = __shfl_sync(0xffffffffu, wgt, j);
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(pb + (base + j) * pstride + h * kPartRow) + lane);
+            n0 = fmaf(wj, v.x, n0); n1 = fmaf(wj, v.y, n1); n2 = fmaf(wj, v.z, n2); n3 = fmaf(wj, v.w, n3);
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
         const float inv = 1.0f / den;
         *reinterpret_cast<float4*>(a.out + (size_t)(hq0 + h) * kHeadDim + lane * 4) =
             make_float4(n0 * inv, n1 * inv, n2 * inv, n3 * inv);

@@ -18,7 +18,7 @@ size_t fp16_attn_scratch(int batch, int n_q_heads) {
   // tickets + status, then partials: one per (unit, warp touching it); units <= batch * n_q_heads
   const size_t units = (size_t)batch * n_q_heads;
   const size_t parts = (size_t)kFp16MaxWarps + 3 * units;
-  return 256 + units * 4 + 256 + parts * 8 * 130 * 4;
+  return 256 + units * 4 + 256 + parts * 8 * kPartRow * 4;
 }
 
 cudaError_t launch_fp16_attn(const void* K, const void* V, const void* q, float* out, int batch, int n_q_heads,
@@ -112,7 +112,7 @@ extern "C" gear_status gear_fp16_decode_attn_static(const void* K, const void* V
   const size_t units = (size_t)batch * n_kv_heads * passes;
   // layout of the array: status word, tickets, then one partial slot per (unit, CTA touching it)
   const size_t header = 256 + ((units * 4 + 255) / 256) * 256;
-  const size_t slot = (size_t)hp * 130 * 4;
+  const size_t slot = (size_t)hp * kPartRow * 4;
   const size_t slots = (kStaticScratchBytes - header) / slot;
   const long long parts_cap = (long long)(slots / units);   // partial slots per unit that fit
   if (parts_cap < 4) return GEAR_ERR_CAPACITY;

@@ -61,6 +61,7 @@ cudaError_t launch_append(void* buf_k, void* buf_v, const void* k_new, const voi
 
 // decode attention over the compressed cache
 constexpr int kMaxStages = 4;
+constexpr int kPartRow = 132;     // floats per head of a partial result: 128 outputs, running max, denominator, padding to 16 bytes
 struct WarpSmem {      // byte offsets of a warp's (= a CTA's) shared-memory regions
   int ring, sdp, sdc, qf, qs, frag, corr_k, ps, corr_v, ocorr, wl, misc, total;
 };
@@ -72,7 +73,7 @@ struct DecodeArgs {
   const __half* buf_v;
   const __half* q;            // [B][Hq][128]
   float* out;                 // [B][Hq][128]
-  float* partial;             // [units][max_parts][HP][130]
+  float* partial;             // [units][max_parts][HP][kPartRow]
   int* tickets;               // [units]
   int* status;
   CacheConst cc;
