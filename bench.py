@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the GEAR hot path on B200: decode steps over a compressed KV cache.
 
-Workload (BASELINE config 2): one LLaMA-2-7B-shaped attention layer, batch 8, 32 heads, d_H = 128,
+Workload (configuration C2): one LLaMA-2-7B-shaped attention layer, batch 8, 32 heads, d_H = 128,
 context 4096, 2-bit codes with group 64, s = 2 % outliers, rank 4, streaming buffer n_b = 64.
 `--layers` independent layer caches are rotated so that the bytes touched between two uses of a cache
 exceed the 126 MB L2.

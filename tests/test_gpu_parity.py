@@ -23,7 +23,7 @@ def pair_factory():
 
 
 def test_config1_single_head_4bit(pair_factory):
-    """BASELINE config 1: n=256, d_H=128, 4-bit, g=64, s=2 %, r=4, 3 loops, n_b=16, one query."""
+    """Configuration C1: n=256, d_H=128, 4-bit, g=64, s=2 %, r=4, 3 loops, n_b=16, one query."""
     p = pair_factory(1, 1, 1, 1, 4, 64, 2.0, 16, 4, 512)
     p.compress(256, 4)
     p.check_segment(0)
