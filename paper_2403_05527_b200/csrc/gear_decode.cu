@@ -1034,21 +1034,27 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
       }
     }
     __syncwarp();
+    // the tensor-core part of the output joins the sparse part in shared memory, so that the partial goes out as
+    // one 16-byte store per lane and head
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       const int h = t + 4 * nt;
       if (h < HPu) {
-        float* dst = part_base + h * kPartRow;
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt)
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             const int ch = 16 * mt + gid + 8 * half;
-            dst[ch] = O[mt][nt][2 * half] + O[mt][nt][2 * half + 1] + ocorr[h * kHeadDim + ch] + cm_own[nt][(mt * 16) / GV];
+            ocorr[h * kHeadDim + ch] += O[mt][nt][2 * half] + O[mt][nt][2 * half + 1] + cm_own[nt][(mt * 16) / GV];
           }
-        if (gid == 0) { dst[128] = m_own[nt]; dst[129] = l_own[nt]; }
+        if (gid == 0) { part_base[h * kPartRow + 128] = m_own[nt]; part_base[h * kPartRow + 129] = l_own[nt]; }
       }
     }
+    __syncwarp();
+#pragma unroll
+    for (int h = 0; h < HP; ++h)
+      if (h < HPu)
+        reinterpret_cast<float4*>(part_base + h * kPartRow)[lane] = reinterpret_cast<const float4*>(ocorr + h * kHeadDim)[lane];
     __threadfence();
     __syncwarp();
     int last = 0;
