@@ -202,3 +202,17 @@ def test_ties_and_constant_groups_follow_the_fixed_tie_break(pair_factory):
         p.check_segment(0)
         p.check_attention()
         p.close()
+
+
+@pytest.mark.parametrize("bits,group,s_pct,hq,hkv,nb,rank", [(4, 16, 10.0, 8, 1, 16, 2), (2, 16, 0.0, 2, 2, 32, 1),
+                                                              (2, 128, 5.0, 16, 2, 128, 8), (4, 32, 6.0, 3, 3, 64, 16)])
+def test_unusual_groupings_head_counts_and_ranks(pair_factory, bits, group, s_pct, hq, hkv, nb, rank):
+    """The less common corners of the parameter space: 16- and 32-channel value groups (eight and four groups per
+    token), eight query heads per kv head, the largest rank, many outliers per group."""
+    p = pair_factory(12, 1, hq, hkv, bits, group, s_pct, nb, min(rank, nb), 1024, r_max=rank)
+    n = 2 * max(group, 64)
+    p.compress(n, rank)
+    p.check_segment(0)
+    p.append(nb + 3)
+    p.check_segment(1)
+    p.check_attention()
