@@ -1065,35 +1065,36 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
       const float* pb = a.partial + (size_t)u * a.max_parts * (HP * kPartRow);
       const size_t pstride = (size_t)HP * kPartRow;
       for (int h = 0; h < HPu; ++h) {
-        // lane i looks at partial i (+32, ...): running maxima first, then weights and the weighted sums
-        float M = -INFINITY;
-        for (int base = 0; base < n_parts; base += 32) {
-          const int i = base + lane;
-          if (i < n_parts) M = fmaxf(M, __ldcg(pb + i * pstride + h * kPartRow + 128));
-        }
+        // Chunks of up to 16 partials: every load of a chunk (lane i: max and denominator of partial i; all lanes: their
+        // four channels of every partial) is issued before anything is used, so a chunk costs one round trip to L2.
+        float M = -INFINITY, den = 0.f, n0 = 0.f, n1 = 0.f, n2 = 0.f, n3 = 0.f;
+        for (int base = 0; base < n_parts; base += 16) {
+          const int cnt = min(16, n_parts - base);
+          const float* ph = pb + (size_t)base * pstride + h * kPartRow;
+          float mi = -INFINITY, li = 0.f;
+          if (lane < cnt) { mi = __ldcg(ph + lane * pstride + 128); li = __ldcg(ph + lane * pstride + 129); }
+          float4 v[16];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-        float den = 0.f, n0 = 0.f, n1 = 0.f, n2 = 0.f, n3 = 0.f;
-        for (int base = 0; base < n_parts; base += 32) {
-          const int i = base + lane;
-          float wgt = 0.f;
-          if (i < n_parts) {
-            const float mi = __ldcg(pb + i * pstride + h * kPartRow + 128);
-            if (mi != -INFINITY) {
-              wgt = exp2f(mi - M);
-              den = fmaf(wgt, __ldcg(pb + i * pstride + h * kPartRow + 129), den);
-            }
-          }
-          const int cnt = min(32, n_parts - base);
-#pragma unroll 4
-          for (int j = 0; j < cnt; ++j) {
+          for (int j = 0; j < 16; ++j)
+            v[j] = j < cnt ? __ldcg(reinterpret_cast<const float4*>(ph + j * pstride) + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+          float cm_ = mi;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) cm_ = fmaxf(cm_, __shfl_xor_sync(0xffffffffu, cm_, o));
+          const float Mn = fmaxf(M, cm_);
+          const float resc = M == -INFINITY ? 0.f : exp2f(M - Mn);
+          const float wgt = mi == -INFINITY ? 0.f : exp2f(mi - Mn);
+          float dsum = wgt * li;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+          den = fmaf(den, resc, dsum);
+          n0 *= resc; n1 *= resc; n2 *= resc; n3 *= resc;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
             const float wj = __shfl_sync(0xffffffffu, wgt, j);
-            const float4 v = __ldcg(reinterpret_cast<const float4*>(pb + (base + j) * pstride + h * kPartRow) + lane);
-            n0 = fmaf(wj, v.x, n0); n1 = fmaf(wj, v.y, n1); n2 = fmaf(wj, v.z, n2); n3 = fmaf(wj, v.w, n3);
+            n0 = fmaf(wj, v[j].x, n0); n1 = fmaf(wj, v[j].y, n1); n2 = fmaf(wj, v[j].z, n2); n3 = fmaf(wj, v[j].w, n3);
           }
+          M = Mn;
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
         const float inv = 1.0f / den;
         *reinterpret_cast<float4*>(a.out + (size_t)(hq0 + h) * kHeadDim + lane * 4) =
             make_float4(n0 * inv, n1 * inv, n2 * inv, n3 * inv);
