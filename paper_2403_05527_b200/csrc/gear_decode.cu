@@ -1055,13 +1055,17 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
     for (int h = 0; h < HP; ++h)
       if (h < HPu)
         reinterpret_cast<float4*>(part_base + h * kPartRow)[lane] = reinterpret_cast<const float4*>(ocorr + h * kHeadDim)[lane];
-    __threadfence();
+    // The ticket is one acquire-release atomic at device scope: it publishes this warp's partial (the warp barrier
+    // before it orders the other lanes' stores) and, for the warp that takes the last ticket, makes the others' visible.
     __syncwarp();
     int last = 0;
-    if (lane == 0) last = (atomicAdd(&a.tickets[u], 1) == n_parts - 1);
+    if (lane == 0) {
+      int old;
+      asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(a.tickets + u) : "memory");
+      last = old == n_parts - 1;
+    }
     last = __shfl_sync(0xffffffffu, last, 0);
     if (last) {
-      __threadfence();
       const float* pb = a.partial + (size_t)u * a.max_parts * (HP * kPartRow);
       const size_t pstride = (size_t)HP * kPartRow;
       for (int h = 0; h < HPu; ++h) {
