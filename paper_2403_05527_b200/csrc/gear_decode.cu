@@ -78,6 +78,14 @@ __device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], 
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// d = a * b (no accumulator input)
+__device__ __forceinline__ void mma16816_z(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  const float z = 0.f;
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(z));
+}
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* p) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -88,44 +96,41 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                : "r"(smem_u32(p)));
 }
-__device__ __forceinline__ uint32_t lop3_and_or(uint32_t x, uint32_t mask, uint32_t orv) {
-  uint32_t r;
-  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(x), "r"(mask), "r"(orv));
-  return r;
-}
 __device__ __forceinline__ uint32_t h2_as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
 
-// (x & mask) | 0x6400 puts each masked field into the mantissa of 1024.0; one
-// half2 fma with exact constants brings it back to the integer code.
-// `mul`, `add`: half2 bit patterns of the constants.
-__device__ __forceinline__ uint32_t field_to_h2(uint32_t x, uint32_t mask, uint32_t mul, uint32_t add) {
-  uint32_t r;
-  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(lop3_and_or(x, mask, 0x64006400u)), "r"(mul), "r"(add));
-  return r;
+// Codes become fragment registers with one AND each.  A masked field left in place, read as fp16, is the
+// subnormal  code * 2^(field_shift - 24)  (the tensor cores take subnormal inputs exactly); fields above the
+// 10-bit mantissa are reached through one shifted copy of the word.  The power of two is undone where it is free:
+// in the B operand for keys, in the output row for values.
+template <int BITS>
+__host__ __device__ constexpr int field_shift(int u) {     // bit position of field u once it sits in the mantissa
+  return BITS == 2 ? 2 * (u < 5 ? u : u - 5) : 4 * (u & 1);
 }
 // One 32-bit word of codes -> its fragment registers r[0 .. 16/BITS).
 template <int BITS>
 __device__ __forceinline__ void unpack_word(uint32_t x, uint32_t* r) {
   if (BITS == 2) {
-    // (1, -1024), (1/4, -256), (1/16, -64), (1/64, -16), (1/256, -4) as half2
     const uint32_t y = x >> 10;
-    r[0] = field_to_h2(x, 0x00030003u, 0x3C003C00u, 0xE400E400u);
-    r[1] = field_to_h2(x, 0x000C000Cu, 0x34003400u, 0xDC00DC00u);
-    r[2] = field_to_h2(x, 0x00300030u, 0x2C002C00u, 0xD400D400u);
-    r[3] = field_to_h2(x, 0x00C000C0u, 0x24002400u, 0xCC00CC00u);
-    r[4] = field_to_h2(x, 0x03000300u, 0x1C001C00u, 0xC400C400u);
-    r[5] = field_to_h2(y, 0x00030003u, 0x3C003C00u, 0xE400E400u);
-    r[6] = field_to_h2(y, 0x000C000Cu, 0x34003400u, 0xDC00DC00u);
-    r[7] = field_to_h2(y, 0x00300030u, 0x2C002C00u, 0xD400D400u);
+    r[0] = x & 0x00030003u;
+    r[1] = x & 0x000C000Cu;
+    r[2] = x & 0x00300030u;
+    r[3] = x & 0x00C000C0u;
+    r[4] = x & 0x03000300u;
+    r[5] = y & 0x00030003u;
+    r[6] = y & 0x000C000Cu;
+    r[7] = y & 0x00300030u;
   } else {
     const uint32_t y = x >> 8;
-    r[0] = field_to_h2(x, 0x000F000Fu, 0x3C003C00u, 0xE400E400u);
-    r[1] = field_to_h2(x, 0x00F000F0u, 0x2C002C00u, 0xD400D400u);
-    r[2] = field_to_h2(y, 0x000F000Fu, 0x3C003C00u, 0xE400E400u);
-    r[3] = field_to_h2(y, 0x00F000F0u, 0x2C002C00u, 0xD400D400u);
+    r[0] = x & 0x000F000Fu;
+    r[1] = x & 0x00F000F0u;
+    r[2] = y & 0x000F000Fu;
+    r[3] = y & 0x00F000F0u;
   }
 }
+// Keys: the B register that meets fields 2j (b0) / 2j+1 (b1) holds q * scale * 2^(kKeyExp - field_shift), so every
+// product carries 2^(kKeyExp - 24); the exponent keeps the scaled operand inside the fp16 range both ways.
+template <int BITS> constexpr int kKeyExp = BITS == 2 ? 4 : 2;
 
 // fp32 pair -> half2 of the high parts and half2 of the rounding remainders
 __device__ __forceinline__ void split_hi_lo(float x0, float x1, uint32_t& hi, uint32_t& lo) {
@@ -269,6 +274,13 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
   float* wl = reinterpret_cast<float*>(smem + a.ws.wl);          // [16][heads]
   int* qexp_s = reinterpret_cast<int*>(smem + a.ws.misc);        // [HP]
 
+  // this lane's four channels in the key set-up sit in B register (lane / 2) % 2 of channel chunk lane / 4, which
+  // meets field 2 * (chunk % 4) + register of the 2-bit words (any field of that parity of the 4-bit words)
+  const float kfac = pow2i(kKeyExp<BITS> - (BITS == 2 ? 2 * ((2 * ((lane >> 2) & 3) + ((lane >> 1) & 1)) % 5)
+                                                      : 4 * ((lane >> 1) & 1)));
+  constexpr float kKeyBack = (float)(1 << (24 - kKeyExp<BITS>));       // undoes 2^(kKeyExp - 24)
+  const bool o_plain = a.n_blocks_c == 0;       // no compressed block: the output rows carry no factor
+
   if (lane == 0)
     for (int s = 0; s < NS; ++s) mbar_init(&bar[s], 1);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -368,6 +380,18 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
   auto release = [&]() {       // the oldest item is consumed: refill its stage
     __syncwarp();
     issue();
+  };
+
+  // Output rows fed by the codes carry the factor of the field their codes came from: row half hf (channel gid + 8 hf)
+  // of channel tile mt holds  value * 2^(row_shift - 24).  A product of full-range operands (buffer rows, B_V U) joins
+  // such a row through a zero-based product and one multiply-add per element.
+  auto row_shift = [](int mt, int hf) { return field_shift<BITS>(2 * (mt % (8 / BITS)) + hf); };
+  auto add_scaled = [&](float (&o)[4], int mt, const uint32_t (&av)[4], uint32_t b0, uint32_t b1) {
+    float d[4];
+    mma16816_z(d, av, b0, b1);
+    const float f0 = 1.f / (float)(1 << (24 - row_shift(mt, 0))), f1 = 1.f / (float)(1 << (24 - row_shift(mt, 1)));
+    o[0] = fmaf(d[0], f0, o[0]); o[1] = fmaf(d[1], f0, o[1]);
+    o[2] = fmaf(d[2], f1, o[2]); o[3] = fmaf(d[3], f1, o[3]);
   };
 
   // ---- loop over the units this warp touches
@@ -529,7 +553,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
           const uint32_t w4[4] = {kz.x, kz.y, kz.z, kz.w};
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            sc4[j] = __low2float(u32_as_h2(w4[j]));
+            sc4[j] = __low2float(u32_as_h2(w4[j])) * kfac;
             zr4[j] = __high2float(u32_as_h2(w4[j]));
           }
         }
@@ -661,6 +685,10 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
                   mma16816(acc[hf][nt], af[k4], bq[nt][4 * hf + k4][0], bq[nt][4 * hf + k4][1]);
             }
             if (!kBuf) {                                // low-rank key term: A_K rows times w (zero rows when r = 0)
+#pragma unroll
+              for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[1][nt][i] *= kKeyBack;
               uint32_t aa[4] = {0u, 0u, 0u, 0u};
               if (pa0) {
                 aa[0] = *reinterpret_cast<const uint32_t*>(akp);
@@ -678,8 +706,9 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
             for (int nt = 0; nt < NT; ++nt) {
               if (t + 4 * nt < HPu) {
                 // raw sums only: the zero-point constant and the sparse term are added in the softmax pass
-                const float v0 = (acc[0][nt][0] + acc[0][nt][1]) + (acc[1][nt][0] + acc[1][nt][1]);
-                const float v1 = (acc[0][nt][2] + acc[0][nt][3]) + (acc[1][nt][2] + acc[1][nt][3]);
+                const float back = kBuf ? 1.f : kKeyBack;
+                const float v0 = fmaf(acc[0][nt][0] + acc[0][nt][1], back, acc[1][nt][0] + acc[1][nt][1]);
+                const float v1 = fmaf(acc[0][nt][2] + acc[0][nt][3], back, acc[1][nt][2] + acc[1][nt][3]);
                 float* pr = ps + psoff[nt] + tok0;
                 pr[0] = v0; pr[8] = v1;
               }
@@ -839,31 +868,20 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
                   bv[nt][g][0] = v.x; bv[nt][g][1] = v.y;
                 }
               fvp += kFragStride;
-              if (BITS == 2) {
-                const uint4 w = cwp[0];
+              constexpr int TPP = 8 / BITS;               // channel tiles per pair of words
+#pragma unroll
+              for (int pl = 0; pl < BITS / 2; ++pl) {
+                const uint4 w = cwp[pl * 32];
                 const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                  uint32_t r[8];
-                  unpack_word<2>(wv[q4], r);
+                for (int wp = 0; wp < 2; ++wp) {
+                  uint32_t rA[16 / BITS], rB[16 / BITS];
+                  unpack_word<BITS>(wv[2 * wp], rA);
+                  unpack_word<BITS>(wv[2 * wp + 1], rB);
 #pragma unroll
-                  for (int m2 = 0; m2 < 2; ++m2) {
-                    const int mt = 2 * q4 + m2, g = (mt * 16) / GV;
-                    const uint32_t av[4] = {r[4 * m2], r[4 * m2 + 1], r[4 * m2 + 2], r[4 * m2 + 3]};
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) mma16816(O[mt][nt], av, bv[nt][g][0], bv[nt][g][1]);
-                  }
-                }
-              } else {
-#pragma unroll
-                for (int pl = 0; pl < 2; ++pl) {
-                  const uint4 w = cwp[pl * 32];
-                  const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                  for (int q4 = 0; q4 < 4; ++q4) {
-                    const int mt = 4 * pl + q4, g = (mt * 16) / GV;
-                    uint32_t av[4];
-                    unpack_word<4>(wv[q4], av);
+                  for (int j = 0; j < TPP; ++j) {
+                    const int mt = TPP * (2 * pl + wp) + j, g = (mt * 16) / GV;
+                    const uint32_t av[4] = {rA[2 * j], rA[2 * j + 1], rB[2 * j], rB[2 * j + 1]};
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) mma16816(O[mt][nt], av, bv[nt][g][0], bv[nt][g][1]);
                   }
@@ -889,7 +907,10 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
                 uint32_t av[4];
                 ldmatrix_x4_trans(av, stV + ((lane & 7) + 8 * (lane >> 4)) * kBufPitch + (16 * mt + 8 * ((lane >> 3) & 1)) * 2);
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) mma16816(O[mt][nt], av, bp[nt][0], bp[nt][1]);
+                for (int nt = 0; nt < NT; ++nt) {
+                  if (o_plain) mma16816(O[mt][nt], av, bp[nt][0], bp[nt][1]);
+                  else add_scaled(O[mt][nt], mt, av, bp[nt][0], bp[nt][1]);
+                }
               }
             }
           }
@@ -988,7 +1009,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
             aa[3] = *reinterpret_cast<const uint32_t*>(r1 + 2 * t + 8);
           }
 #pragma unroll
-          for (int nt = 0; nt < NT; ++nt) mma16816(O[mt][nt], aa, bu[nt][0], bu[nt][1]);
+          for (int nt = 0; nt < NT; ++nt) add_scaled(O[mt][nt], mt, aa, bu[nt][0], bu[nt][1]);
         }
         u_pending = false;
       }
@@ -1045,7 +1066,8 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             const int ch = 16 * mt + gid + 8 * half;
-            ocorr[h * kHeadDim + ch] += O[mt][nt][2 * half] + O[mt][nt][2 * half + 1] + cm_own[nt][(mt * 16) / GV];
+            const float back = o_plain ? 1.f : (float)(1 << (24 - row_shift(mt, half)));
+            ocorr[h * kHeadDim + ch] += fmaf(O[mt][nt][2 * half] + O[mt][nt][2 * half + 1], back, cm_own[nt][(mt * 16) / GV]);
           }
         if (gid == 0) { part_base[h * kPartRow + 128] = m_own[nt]; part_base[h * kPartRow + 129] = l_own[nt]; }
       }

@@ -30,9 +30,9 @@ __device__ __forceinline__ unsigned int load_code(const unsigned char* rec, cons
     const int a = (c16 >> 3) | ((ts >> 3) << 1), t = (ts & 7) >> 1;
     e = ts & 1;
     lane = gid * 4 + t;
-    const int mpw = hpw / 4;
-    q = mt / mpw;
-    u = 4 * (mt % mpw) + a;
+    const int tpp = hpw / 2;
+    q = 2 * (mt / tpp) + (a >> 1);
+    u = 2 * (mt % tpp) + (a & 1);
   }
   const unsigned int* words =
       reinterpret_cast<const unsigned int*>(rec + (side == 0 ? sd.off_kcodes : sd.off_vcodes) + slab * sd.slab_codes);

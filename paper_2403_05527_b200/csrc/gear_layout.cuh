@@ -112,6 +112,18 @@ __host__ __device__ inline void layout_segment(SegDesc& s, const CacheConst& c) 
 // Values are the A operand (channels x tokens): for channel tile mt
 //   a0 = {ch gid,   tok 2t, 2t+1}   a1 = {ch gid+8, tok 2t, 2t+1}
 //   a2 = {ch gid,   tok 2t+8, +9}   a3 = {ch gid+8, tok 2t+8, +9}
+//
+// The decode kernel turns a word into fragment registers with one AND per
+// register: the masked field, left where it is, read as fp16 is the subnormal
+// code * 2^(b*u' - 24) (u' = u for the fields the 10-bit mantissa holds, after
+// one shift of the word for the others).  A power of two per register is
+// harmless only where the product can absorb it, which fixes who shares a field
+// position: for keys a0 and a1 (they meet the same B register: its q * scale is
+// pre-divided), for values a0 and a2 (they feed the same output row, which
+// carries the factor until the end).  Hence keys take (a0, a2) of a tile from
+// fields 2j, 2j+1 of one word and (a1, a3) from the same fields of a second
+// word; values take (a0, a1) from fields 2j, 2j+1 of one word and (a2, a3) from
+// a second word.
 // ---------------------------------------------------------------------------
 __host__ __device__ inline int words_per_lane(int bits) { return bits == 2 ? 4 : 8; }
 __host__ __device__ inline int regs_per_word(int bits) { return bits == 2 ? 8 : 4; }   // half2 per word
@@ -129,10 +141,9 @@ __host__ __device__ inline void code_coord_k(int bits, int lane, int q, int u, i
 
 // value code at (lane, q, u, e) -> token in slab, channel
 __host__ __device__ inline void code_coord_v(int bits, int lane, int q, int u, int e, int& tok, int& ch) {
-  const int hpw = regs_per_word(bits);
-  const int mpw = hpw / 4;                  // channel tiles per word (2 or 1)
-  const int mt = mpw * q + (u >> 2);
-  const int a = u & 3;                      // fragment register a0..a3
+  const int tpp = regs_per_word(bits) / 2;  // channel tiles per pair of words (4 or 2)
+  const int mt = tpp * (q >> 1) + (u >> 1);
+  const int a = (u & 1) + 2 * (q & 1);      // fragment register a0..a3
   ch = 16 * mt + 8 * (a & 1) + (lane >> 2);
   tok = 2 * (lane & 3) + 8 * (a >> 1) + e;
 }
