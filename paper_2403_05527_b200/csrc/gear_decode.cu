@@ -139,6 +139,12 @@ __device__ __forceinline__ void split_hi_lo(float x0, float x1, uint32_t& hi, ui
   lo = h2_as_u32(__floats2half2_rn(x0 - __low2float(h), x1 - __high2float(h)));
 }
 
+// maximum over the warp in one instruction
+__device__ __forceinline__ float warp_max(float x) {
+  float r;
+  asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
+  return r;
+}
 __device__ __forceinline__ int float_exponent(float x) { return (int)((__float_as_uint(x) >> 23) & 0xFFu) - 127; }
 // 2^e for |e| <= 60
 __device__ __forceinline__ float pow2i(int e) { return __uint_as_float((uint32_t)(127 + e) << 23); }
@@ -170,7 +176,7 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
   w.corr_v = o;  o += HP * kHeadDim * 4;
   w.ocorr = o;   o += HP * kHeadDim * 4;
   w.wl = o;      o += kMaxRank * (HP == 1 ? 1 : 8) * 4 + 16;
-  w.misc = o;    o += 64;
+  w.misc = o;    o += 32 + kMaxStages * 8;   // exponents of max |q| per head, then the ring's mbarriers
   w.ring = round_up(o, 16);
   // most resident warps (in steps of four: one per scheduler) whose ring still holds two stages; then as many
   // stages as fit
@@ -193,20 +199,20 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
 // an immediate and the slab loops unroll); any other segment runs through the same code with run-time values.
 struct DynShape {                      // values read from the segment descriptor
   static constexpr bool kDyn = true, kBuf = false;
-  static constexpr int T = 0, k2k = 0, r_pad = 0, k2v = 0, unroll = 1;
+  static constexpr int T = 0, k2k = 0, r_pad = 0, k2v = 0, unroll = 1, tok_unroll = 1;
   static constexpr int off_kscale = 0, off_koval = 0, off_koidx = 0, off_kcodes = 0, off_ak = 0, off_av = 0, off_vscale = 0,
                        off_voval = 0, off_voidx = 0;
 };
 struct BufShape {                      // one slab of fp16 rows of the streaming buffer
   static constexpr bool kDyn = false, kBuf = true;
-  static constexpr int T = kSlab, k2k = 0, r_pad = 0, k2v = 0, unroll = 1;
+  static constexpr int T = kSlab, k2k = 0, r_pad = 0, k2v = 0, unroll = 1, tok_unroll = 1;
   static constexpr int off_kscale = 0, off_koval = 0, off_koidx = 0, off_kcodes = 0, off_ak = 0, off_av = 0, off_vscale = 0,
                        off_voval = 0, off_voidx = 0;
 };
 template <int BITS, int NGV, int T_, int KK, int RP, int KV>
 struct StaticShape {                   // mirrors layout_segment(); checked against it on the host (static_shape_id)
   static constexpr bool kDyn = false, kBuf = false;
-  static constexpr int T = T_, k2k = 2 * KK, r_pad = RP, k2v = 2 * KV, unroll = 2;
+  static constexpr int T = T_, k2k = 2 * KK, r_pad = RP, k2v = 2 * KV, unroll = 2, tok_unroll = T_ / 32;
   static constexpr int nslab = T_ / kSlab, slab_codes = kSlab * kHeadDim * BITS / 8;
   static constexpr int off_kscale = kRecHeader;
   static constexpr int off_koval = off_kscale + kHeadDim * 4;
@@ -255,7 +261,6 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
   constexpr int WLS = HP == 1 ? 1 : 8;            // row stride of the small factor exchange buffer wl[16][heads]
   constexpr int HMASK = HP == 1 ? 0 : 7;          // heads that exist in wl, as a mask on the lane's head
   extern __shared__ __align__(128) unsigned char smem[];
-  __shared__ __align__(8) uint64_t bar[kMaxStages];
 
   const int lane = threadIdx.x, gid = lane >> 2, t = lane & 3;
   const int G = a.group_heads;
@@ -273,6 +278,8 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
   float* ocorr = reinterpret_cast<float*>(smem + a.ws.ocorr);    // [HP][128]
   float* wl = reinterpret_cast<float*>(smem + a.ws.wl);          // [16][heads]
   int* qexp_s = reinterpret_cast<int*>(smem + a.ws.misc);        // [HP]
+  uint64_t* bar = reinterpret_cast<uint64_t*>(smem + a.ws.misc + 32);   // [kMaxStages]; no static shared memory, so
+                                                                         // that sixteen warps fit one SM
 
   // this lane's four channels in the key set-up sit in B register (lane / 2) % 2 of channel chunk lane / 4, which
   // meets field 2 * (chunk % 4) + register of the 2-bit words (any field of that parity of the 4-bit words)
@@ -454,6 +461,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
       auto body = [&](auto shape_tag) {
       using S = decltype(shape_tag);
       constexpr bool is_buf = S::kBuf;
+      constexpr int TU = HP == 1 ? S::tok_unroll : 1;     // unrolling of the per-token loops (latency, one head only)
       // ---------------- block geometry
       const int T = S::kDyn ? sdc->T : S::T;
       const int r_pad = S::kDyn ? sdc->r_pad : S::r_pad;
@@ -732,7 +740,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
             int* crow = corr_k + h * maxT;
             const float Sik = pow2i(-sexp_k[h]);
             float mx = -INFINITY;
-#pragma unroll 1
+#pragma unroll (TU)
             for (int tk = lane; tk < valid_tokens; tk += 32) {
               float v = row[tk] + c_zero[h];
               if (!is_buf && k2k > 0) {
@@ -742,8 +750,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
               row[tk] = v;
               mx = fmaxf(mx, v);
             }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            mx = warp_max(mx);
             const float m_new = fmaxf(m_run[h], mx);       // finite: every block holds a valid token
             if (m_new > m_run[h]) {
               alpha[h] = exp2f(m_run[h] - m_new);
@@ -751,7 +758,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
               m_run[h] = m_new;
             }
             float l = 0.f;
-#pragma unroll 1
+#pragma unroll (TU)
             for (int tk = lane; tk < T; tk += 32) {
               const float p = tk < valid_tokens ? exp2f(row[tk] - m_new) : 0.f;   // tokens past the end of the buffer
               l += p;
@@ -806,7 +813,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
 
       // ---------------- B operands of the value products: p * scale (per token and group) and p, split hi / lo;
       //                  the zero-point term goes to the fp32 side sums cm
-#pragma unroll 1
+#pragma unroll (TU)
       for (int pr = lane; pr < T / 2; pr += 32) {      // this lane's token pairs
         const int s = pr >> 3, pi = pr & 7, tw = pi & 3, rg = pi >> 2;
         const int tp = 2 * pr;
@@ -926,7 +933,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
         const __half2* vsz = reinterpret_cast<const __half2*>(vp + o_vsz);
         const unsigned char* voval = vp + o_voval;
         const unsigned char* voidx = vp + o_voidx;
-#pragma unroll 1
+#pragma unroll (TU)
         for (int tk = lane; tk < T; tk += 32) {
           float pS[HP];
 #pragma unroll
