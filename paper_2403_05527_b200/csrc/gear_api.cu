@@ -365,6 +365,17 @@ extern "C" gear_status gear_decode_attn(gear_cache* c, const void* q, float* out
   const long long work = (long long)c->cc.BH * ((c->G + hp - 1) / hp) * (c->n_blocks_c + (c->buf_len + 15) / 16);
   long long grid = (long long)c->sm_count * c->plan_occ;
   if (grid > work) grid = work;
+  // When the warps that fit divide almost evenly among the units, cut every unit into the same number of ranges: a
+  // warp that runs from one unit into the next pays a second prologue and epilogue, and with few blocks per warp those
+  // warps finish last.  Otherwise (many blocks per warp, or a poor fit) cut the flat space evenly.
+  {
+    const long long units = (long long)c->cc.BH * ((c->G + hp - 1) / hp), nb = work / units;
+    const long long ppu = grid / units;
+    if (ppu >= 1 && ppu <= nb && ppu < c->max_parts && units * ppu * 100 >= grid * 96) {
+      a.parts_per_unit = (int)ppu;
+      grid = units * ppu;
+    }
+  }
   if (launch_decode(a, (int)grid, (cudaStream_t)stream) != cudaSuccess) {
     cudaGetLastError();
     return GEAR_ERR_CUDA;

@@ -187,6 +187,7 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
     if (ns < 2) continue;
     if (ns > kMaxStages) ns = kMaxStages;
     w.total = w.ring + (int)ns * stage;
+    a->parts_per_unit = 0;
     a->nstage = (int)ns; a->stage_bytes = stage; a->bregion = bregion; a->max_T = max_T; a->hpa = HP; a->ws = w;
     return true;
   }
@@ -300,7 +301,23 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
   const int nbuf_blocks = (a.buf_len + kSlab - 1) / kSlab;
   const int NB = a.n_blocks_c + nbuf_blocks;
   int n_left, u, blk_lo;                        // blocks left for this warp, current unit, first block in it
-  {
+  int part = 0;                                 // unit-aligned split: this warp's range inside its unit
+  if (a.parts_per_unit > 0) {
+    // No warp crosses from one unit into the next.  NB blocks over P ranges leave NB % P ranges one block longer;
+    // those get the lowest CTA indices of the grid (longest first: they are dispatched first and finish with the rest).
+    const int P = a.parts_per_unit, base = NB / P, rem = NB - base * P;     // base > 0: the host keeps P <= NB
+    const int n_long = a.cc.BH * passes * rem;
+    if ((int)blockIdx.x < n_long) {
+      u = blockIdx.x / rem;
+      part = blockIdx.x - u * rem;
+    } else {
+      const int b2 = blockIdx.x - n_long;
+      u = b2 / (P - rem);
+      part = rem + b2 - u * (P - rem);
+    }
+    blk_lo = part * base + min(part, rem);
+    n_left = base + (part < rem ? 1 : 0);
+  } else {
     const long long F = (long long)a.cc.BH * passes * NB;
     const long long NW = gridDim.x, gw = blockIdx.x;
     const long long f0 = gw * F / NW, f1 = (gw + 1) * F / NW;
@@ -1033,12 +1050,18 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
     if (!alive) break;
 
     // ---------------- partial result of this unit: (m, l, o) per head
-    const long long F = (long long)a.cc.BH * passes * NB, NW = gridDim.x;
-    const long long bflat = (long long)u * NB, eflat = bflat + NB;
-    const long long w_first = ((bflat + 1) * NW + F - 1) / F - 1;
-    const long long w_last = (eflat * NW + F - 1) / F - 1;
-    const int n_parts = (int)(w_last - w_first + 1);
-    const int slot = (int)(blockIdx.x - w_first);
+    int n_parts, slot;
+    if (a.parts_per_unit > 0) {
+      n_parts = a.parts_per_unit;
+      slot = part;
+    } else {
+      const long long F = (long long)a.cc.BH * passes * NB, NW = gridDim.x;
+      const long long bflat = (long long)u * NB, eflat = bflat + NB;
+      const long long w_first = ((bflat + 1) * NW + F - 1) / F - 1;
+      const long long w_last = (eflat * NW + F - 1) / F - 1;
+      n_parts = (int)(w_last - w_first + 1);
+      slot = (int)(blockIdx.x - w_first);
+    }
     float* part_base = a.partial + ((size_t)u * a.max_parts + slot) * (HP * kPartRow);
     float cm_own[NT][NGV], m_own[NT], l_own[NT];
 #pragma unroll

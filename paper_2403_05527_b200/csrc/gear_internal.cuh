@@ -81,6 +81,8 @@ struct DecodeArgs {
   int buf_len;                // tokens in the fp16 buffer
   int n_kv_heads, group_heads;   // H, G = Hq / H
   int max_parts;
+  int parts_per_unit;         // > 0: every unit is cut into this many ranges, one per warp (grid = units * parts);
+                              // 0: the flat (unit, block) space is cut into gridDim.x equal ranges
   int nstage;                 // ring stages (<= kMaxStages)
   int stage_bytes;            // bytes of one ring stage
   int bregion;                // bytes at the front of a stage reserved for one B factor
