@@ -267,6 +267,38 @@ __global__ void pi_init_kernel(PiArgs p, const float* B0, int bh0, int BH_total_
   (void)BH_total_rank_stride;
 }
 
+// Sums over the warp of RP values per lane, every lane getting all RP sums.  The first log2(RP) exchange steps
+// halve the number of values a lane carries (each lane hands the half it drops to its partner), the remaining steps are
+// a butterfly on the single value left, and a broadcast per value returns the sums: RP - 1 + (5 - log2 RP) + RP
+// shuffles instead of 5 RP.  The order of the additions is fixed, so results are reproducible.
+template <int RP>
+__device__ __forceinline__ void warp_sum_all(float (&s)[RP], int lane) {
+  constexpr int LOG = RP == 4 ? 2 : (RP == 8 ? 3 : 4);
+  static_assert(RP == 4 || RP == 8 || RP == 16, "rank padding");
+  int cnt = RP;
+#pragma unroll
+  for (int step = 0; step < 5; ++step) {
+    const int o = 16 >> step;
+    if (step < LOG) {
+      const bool upper = (lane & o) != 0;
+      cnt >>= 1;
+#pragma unroll
+      for (int i = 0; i < RP / 2; ++i) {
+        if (i < cnt) {
+          const float send = upper ? s[i] : s[i + cnt];
+          const float keep = upper ? s[i + cnt] : s[i];
+          s[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+        }
+      }
+    } else {
+      s[0] += __shfl_xor_sync(0xffffffffu, s[0], o);
+    }
+  }
+  const float mine = s[0];                    // the sum of value (lane >> (5 - LOG)) % RP
+#pragma unroll
+  for (int r = 0; r < RP; ++r) s[r] = __shfl_sync(0xffffffffu, mine, r << (5 - LOG));
+}
+
 // mode 0: a = R b ; partial of R^T a                         (loops before the last)
 // mode 1: a = R b -> A0 ; partial Gram a^T a                  (last loop, first product)
 // mode 2: a = A0 W (W = R1^-1 R2^-1) -> stored A ; partial of R^T a   (last loop, second product)
@@ -301,9 +333,27 @@ __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) gram[i] = 0.f;
 
-  for (int row = row0 + warp; row < row1; row += kPassWarps) {
-    const float4 x4 = *reinterpret_cast<const float4*>(R + (size_t)row * kHeadDim + lane * 4);
-    const float x[4] = {x4.x, x4.y, x4.z, x4.w};
+  // U rows of a warp are requested before the first is used: with one row in flight per warp the pass is bound by
+  // the latency of that load, not by bandwidth
+  constexpr int U = RP <= 8 ? 4 : 2;
+  for (int rowu = row0 + warp; rowu < row1; rowu += kPassWarps * U) {
+    float4 xs[U];
+    float a0v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int r = rowu + u * kPassWarps;
+      xs[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      a0v[u] = 0.f;
+      if (r < row1) {
+        xs[u] = *reinterpret_cast<const float4*>(R + (size_t)r * kHeadDim + lane * 4);
+        if (MODE == 2 && lane < RP) a0v[u] = A0[(size_t)r * kMaxRank + lane];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+    const int row = rowu + u * kPassWarps;
+    if (row >= row1) break;                      // uniform over the warp
+    const float x[4] = {xs[u].x, xs[u].y, xs[u].z, xs[u].w};
     float a[RP];
     if (MODE != 2) {
 #pragma unroll
@@ -311,12 +361,13 @@ __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
         float s = 0.f;
 #pragma unroll
         for (int j = 0; j < 4; ++j) s = fmaf(x[j], b[j][r], s);
-        a[r] = warp_sum(s);
+        a[r] = s;
       }
+      warp_sum_all<RP>(a, lane);
     } else {
       float a0[RP];
 #pragma unroll
-      for (int r = 0; r < RP; ++r) a0[r] = A0[(size_t)row * kMaxRank + r];
+      for (int r = 0; r < RP; ++r) a0[r] = __shfl_sync(0xffffffffu, a0v[u], r);
 #pragma unroll
       for (int r = 0; r < RP; ++r) {
         float s = 0.f;
@@ -363,6 +414,7 @@ __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
             p.dbgA[(((size_t)(p.bh0 + bhl) * 2 + side) * sd.n_c + row) * sd.rank + lane] = val;
         }
       }
+    }
     }
   }
   // combine the warps of this block in a fixed order, write the chunk's partial
