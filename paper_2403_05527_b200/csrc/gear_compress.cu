@@ -300,8 +300,9 @@ __device__ __forceinline__ void warp_sum_all(float (&s)[RP], int lane) {
 }
 
 // mode 0: a = R b ; partial of R^T a                         (loops before the last)
-// mode 1: a = R b -> A0 ; partial Gram a^T a                  (last loop, first product)
-// mode 2: a = A0 W (W = R1^-1 R2^-1) -> stored A ; partial of R^T a   (last loop, second product)
+// mode 1: a = R b -> A0 ; partial Gram a^T a ; partial of R^T a   (last loop: both products in one pass over R,
+//         since R^T (A0 W) = (R^T A0) W and W is only 16 x 16)
+// mode 2: a = A0 W (W = R1^-1 R2^-1) -> stored A             (last loop; R is not read again)
 template <int RP, int MODE>
 __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
   __shared__ float red[kHeadDim * RP];            // cross-warp sum, accumulated warp by warp
@@ -345,7 +346,7 @@ __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
       xs[u] = make_float4(0.f, 0.f, 0.f, 0.f);
       a0v[u] = 0.f;
       if (r < row1) {
-        xs[u] = *reinterpret_cast<const float4*>(R + (size_t)r * kHeadDim + lane * 4);
+        if (MODE != 2) xs[u] = *reinterpret_cast<const float4*>(R + (size_t)r * kHeadDim + lane * 4);
         if (MODE == 2 && lane < RP) a0v[u] = A0[(size_t)r * kMaxRank + lane];
       }
     }
@@ -389,12 +390,14 @@ __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
         const int pr = lane * 8 + i;
         if (pr < RP * RP) gram[i] = fmaf(arow[warp][pr / RP], arow[warp][pr % RP], gram[i]);
       }
-    } else {
+    }
+    if (MODE != 2) {
 #pragma unroll
       for (int j = 0; j < 4; ++j)
 #pragma unroll
         for (int r = 0; r < RP; ++r) acc[j][r] = fmaf(x[j], a[r], acc[j][r]);
-      if (MODE == 2) {
+    } else {
+      {
         // store the final A row: fp16 in fragment order inside the record, fp32 copy on request
         float mine = 0.f;
 #pragma unroll
@@ -417,27 +420,33 @@ __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
     }
     }
   }
-  // combine the warps of this block in a fixed order, write the chunk's partial
-  for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x) red[i] = 0.f;
-  __syncthreads();
-  for (int w = 0; w < kPassWarps; ++w) {
-    if (warp == w) {
-      if (MODE == 1) {
+  // combine the warps of this block in a fixed order, write the chunk's partials
+  if (MODE == 1) {
+    for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x) red[i] = 0.f;
+    __syncthreads();
+    for (int w = 0; w < kPassWarps; ++w) {
+      if (warp == w) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) red[lane * 8 + i] += gram[i];
-      } else {
+      }
+      __syncthreads();
+    }
+    for (int i = threadIdx.x; i < RP * RP; i += blockDim.x)
+      p.Gp[((size_t)tile * p.nchunk + chunk) * 256 + (i / RP) * kMaxRank + i % RP] = red[i];
+    __syncthreads();
+  }
+  if (MODE != 2) {
+    for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x) red[i] = 0.f;
+    __syncthreads();
+    for (int w = 0; w < kPassWarps; ++w) {
+      if (warp == w) {
 #pragma unroll
         for (int j = 0; j < 4; ++j)
 #pragma unroll
           for (int r = 0; r < RP; ++r) red[(lane * 4 + j) * RP + r] += acc[j][r];
       }
+      __syncthreads();
     }
-    __syncthreads();
-  }
-  if (MODE == 1) {
-    for (int i = threadIdx.x; i < RP * RP; i += blockDim.x)
-      p.Gp[((size_t)tile * p.nchunk + chunk) * 256 + (i / RP) * kMaxRank + i % RP] = red[i];
-  } else {
     for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x)
       p.Bp[(((size_t)tile * p.nchunk + chunk) * kHeadDim + i / RP) * kMaxRank + i % RP] = red[i];
   }
@@ -447,7 +456,7 @@ __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
 // `orth`, orthonormalise its columns (modified Gram-Schmidt, two sweeps per
 // column) -- the QR of B at the top of Algorithm 2's last loop.  With `store`,
 // write the final B as fp16 ([r_pad][128] for keys, [128][r_pad] for values).
-__global__ void __launch_bounds__(kHeadDim) pi_reduce_b_kernel(PiArgs p, int orth, int store) {
+__global__ void __launch_bounds__(kHeadDim) pi_reduce_b_kernel(PiArgs p, int orth, int store, int apply_w) {
   __shared__ float wsum[4];
   const int tile = blockIdx.x, j = threadIdx.x, lane = j & 31, warp = j >> 5;
   float b[kMaxRank];
@@ -457,6 +466,19 @@ __global__ void __launch_bounds__(kHeadDim) pi_reduce_b_kernel(PiArgs p, int ort
     if (r < p.rank)
       for (int c = 0; c < p.nchunk; ++c) s += p.Bp[(((size_t)tile * p.nchunk + c) * kHeadDim + j) * kMaxRank + r];
     b[r] = s;
+  }
+  if (apply_w) {                 // the sums are R^T A0: the factor of the orthonormalised A = A0 W is (R^T A0) W
+    float bw[kMaxRank];
+#pragma unroll
+    for (int r = 0; r < kMaxRank; ++r) {
+      float v = 0.f;
+#pragma unroll
+      for (int q = 0; q < kMaxRank; ++q)
+        if (q < p.rank && r < p.rank) v = fmaf(b[q], p.W[(size_t)tile * 256 + q * kMaxRank + r], v);
+      bw[r] = v;
+    }
+#pragma unroll
+    for (int r = 0; r < kMaxRank; ++r) b[r] = bw[r];
   }
   auto block_sum = [&](float v) {
     v = warp_sum(v);
@@ -1061,21 +1083,21 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
     if (!last) {
       launch_pass<0>(pa, st);                                   // A = R B ; B = R^T A
       // the loop after this one is the last: its QR of B is folded into the reduction
-      pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(pa, (l + 1 == job.iters - 1) ? 1 : 0, 0);
+      pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(pa, (l + 1 == job.iters - 1) ? 1 : 0, 0, 0);
     } else {
       if (job.iters == 1) {                                     // single loop: orthonormalise the start itself
         PiArgs q = pa; q.nchunk = 0;
         // Bp unused with zero chunks: re-use the reduce kernel on Bcur through a one-chunk view
         cudaMemcpyAsync(pa.Bp, pa.Bcur, ntiles * kHeadDim * kMaxRank * 4, cudaMemcpyDeviceToDevice, st);
         q.nchunk = 1;
-        pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(q, 1, 0);
+        pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(q, 1, 0, 0);
       }
-      launch_pass<1>(pa, st);                                   // A = R B, Gram of A
+      launch_pass<1>(pa, st);                                   // A0 = R B, Gram of A0, R^T A0
       pi_chol_kernel<<<(int)ntiles, 32, 0, st>>>(pa, 1);        // A <- Q(A) by CholeskyQR, twice
       pi_gram2_kernel<<<dim3(nchunk, (int)ntiles), 256, 0, st>>>(pa);
       pi_chol_kernel<<<(int)ntiles, 32, 0, st>>>(pa, 0);
-      launch_pass<2>(pa, st);                                   // store A ; B = R^T A
-      pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(pa, 0, 1);
+      launch_pass<2>(pa, st);                                   // store A = A0 W
+      pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(pa, 0, 1, 1);
     }
   }
   return cudaGetLastError();
