@@ -299,15 +299,13 @@ __device__ __forceinline__ void warp_sum_all(float (&s)[RP], int lane) {
   for (int r = 0; r < RP; ++r) s[r] = __shfl_sync(0xffffffffu, mine, r << (5 - LOG));
 }
 
-// mode 0: a = R b ; partial of R^T a                         (loops before the last)
-// mode 1: a = R b -> A0 ; partial Gram a^T a ; partial of R^T a   (last loop: both products in one pass over R,
-//         since R^T (A0 W) = (R^T A0) W and W is only 16 x 16)
-// mode 2: a = A0 W (W = R1^-1 R2^-1) -> stored A             (last loop; R is not read again)
+// One pass over the residual: a = R b for every row, and this chunk's partial of R^T a.
+// mode 0: loops before the last.
+// mode 1: last loop: the rows a are also stored (A0).  Its Gram matrix and the orthonormalising factor W come from
+//         the small kernels below, and since R^T (A0 W) = (R^T A0) W, with W only 16 x 16, R is not read again.
 template <int RP, int MODE>
 __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
   __shared__ float red[kHeadDim * RP];            // cross-warp sum, accumulated warp by warp
-  __shared__ float arow[kPassWarps][kMaxRank];     // mode 1: the current row of A, one per warp
-  __shared__ float Wm[kMaxRank * kMaxRank];
   const int tile = blockIdx.y, chunk = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row0 = chunk * kChunkRows;
@@ -316,47 +314,33 @@ __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
   float* A0 = p.A0 + (size_t)tile * p.n_c * kMaxRank;
 
   float b[4][RP];
-  if (MODE != 2) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
+  for (int j = 0; j < 4; ++j)
 #pragma unroll
-      for (int r = 0; r < RP; ++r) b[j][r] = p.Bcur[((size_t)tile * kHeadDim + lane * 4 + j) * kMaxRank + r];
-  } else {
-    for (int i = threadIdx.x; i < kMaxRank * kMaxRank; i += blockDim.x) Wm[i] = p.W[(size_t)tile * 256 + i];
-    __syncthreads();
-  }
-  float acc[4][RP];       // mode 0 / 2: this lane's 4 channels of R^T a
-  float gram[8];          // mode 1: this lane's 8 Gram entries (pairs lane*8 .. lane*8+7 of RP*RP)
+    for (int r = 0; r < RP; ++r) b[j][r] = p.Bcur[((size_t)tile * kHeadDim + lane * 4 + j) * kMaxRank + r];
+  float acc[4][RP];       // this lane's 4 channels of R^T a
 #pragma unroll
   for (int j = 0; j < 4; ++j)
 #pragma unroll
     for (int r = 0; r < RP; ++r) acc[j][r] = 0.f;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) gram[i] = 0.f;
 
   // U rows of a warp are requested before the first is used: with one row in flight per warp the pass is bound by
   // the latency of that load, not by bandwidth
   constexpr int U = RP <= 8 ? 4 : 2;
   for (int rowu = row0 + warp; rowu < row1; rowu += kPassWarps * U) {
     float4 xs[U];
-    float a0v[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int r = rowu + u * kPassWarps;
       xs[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-      a0v[u] = 0.f;
-      if (r < row1) {
-        if (MODE != 2) xs[u] = *reinterpret_cast<const float4*>(R + (size_t)r * kHeadDim + lane * 4);
-        if (MODE == 2 && lane < RP) a0v[u] = A0[(size_t)r * kMaxRank + lane];
-      }
+      if (r < row1) xs[u] = *reinterpret_cast<const float4*>(R + (size_t)r * kHeadDim + lane * 4);
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-    const int row = rowu + u * kPassWarps;
-    if (row >= row1) break;                      // uniform over the warp
-    const float x[4] = {xs[u].x, xs[u].y, xs[u].z, xs[u].w};
-    float a[RP];
-    if (MODE != 2) {
+      const int row = rowu + u * kPassWarps;
+      if (row >= row1) break;                      // uniform over the warp
+      const float x[4] = {xs[u].x, xs[u].y, xs[u].z, xs[u].w};
+      float a[RP];
 #pragma unroll
       for (int r = 0; r < RP; ++r) {
         float s = 0.f;
@@ -365,90 +349,78 @@ __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
         a[r] = s;
       }
       warp_sum_all<RP>(a, lane);
-    } else {
-      float a0[RP];
+      if (MODE == 1) {
+        float mine = 0.f;
 #pragma unroll
-      for (int r = 0; r < RP; ++r) a0[r] = __shfl_sync(0xffffffffu, a0v[u], r);
-#pragma unroll
-      for (int r = 0; r < RP; ++r) {
-        float s = 0.f;
-#pragma unroll
-        for (int q = 0; q < RP; ++q) s = fmaf(a0[q], Wm[q * kMaxRank + r], s);
-        a[r] = s;
+        for (int r = 0; r < RP; ++r) if (r == lane) mine = a[r];
+        if (lane < RP) A0[(size_t)row * kMaxRank + lane] = mine;
       }
-    }
-    if (MODE == 1) {
-      __syncwarp();
-      if (lane == 0) {
-#pragma unroll
-        for (int r = 0; r < RP; ++r) arow[warp][r] = a[r];
-      }
-      __syncwarp();
-      if (lane < RP) A0[(size_t)row * kMaxRank + lane] = arow[warp][lane];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int pr = lane * 8 + i;
-        if (pr < RP * RP) gram[i] = fmaf(arow[warp][pr / RP], arow[warp][pr % RP], gram[i]);
-      }
-    }
-    if (MODE != 2) {
 #pragma unroll
       for (int j = 0; j < 4; ++j)
 #pragma unroll
         for (int r = 0; r < RP; ++r) acc[j][r] = fmaf(x[j], a[r], acc[j][r]);
-    } else {
-      {
-        // store the final A row: fp16 in fragment order inside the record, fp32 copy on request
-        float mine = 0.f;
-#pragma unroll
-        for (int r = 0; r < RP; ++r) if (r == lane) mine = a[r];
-        if (lane < p.seg.r_pad) {
-          const SegDesc& sd = p.seg;
-          const int bhl = tile >> 1, side = tile & 1;
-          const int blk = row / sd.T, tib = row % sd.T, slab = tib / kSlab, ts = tib % kSlab;
-          unsigned char* rec = p.arena + sd.seg_base + (size_t)(p.bh0 + bhl) * sd.bh_stride + sd.bfac_bytes +
-                               (size_t)blk * sd.rec_bytes;
-          const float val = lane < sd.rank ? mine : 0.f;
-          if (side == 0)
-            reinterpret_cast<__half*>(rec + sd.off_ak + slab * sd.slab_a)[ts * sd.r_pad + lane] = __float2half_rn(val);
-          else
-            reinterpret_cast<__half*>(rec + sd.off_av + slab * sd.slab_a)[lane * kSlab + ts] = __float2half_rn(val);
-          if (p.dbgA != nullptr && lane < sd.rank)
-            p.dbgA[(((size_t)(p.bh0 + bhl) * 2 + side) * sd.n_c + row) * sd.rank + lane] = val;
-        }
-      }
-    }
     }
   }
-  // combine the warps of this block in a fixed order, write the chunk's partials
-  if (MODE == 1) {
-    for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x) red[i] = 0.f;
-    __syncthreads();
-    for (int w = 0; w < kPassWarps; ++w) {
-      if (warp == w) {
+  // combine the warps of this block in a fixed order, write the chunk's partial
+  for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x) red[i] = 0.f;
+  __syncthreads();
+  for (int w = 0; w < kPassWarps; ++w) {
+    if (warp == w) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) red[lane * 8 + i] += gram[i];
-      }
-      __syncthreads();
+      for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int r = 0; r < RP; ++r) red[(lane * 4 + j) * RP + r] += acc[j][r];
     }
-    for (int i = threadIdx.x; i < RP * RP; i += blockDim.x)
-      p.Gp[((size_t)tile * p.nchunk + chunk) * 256 + (i / RP) * kMaxRank + i % RP] = red[i];
     __syncthreads();
   }
-  if (MODE != 2) {
-    for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x) red[i] = 0.f;
-    __syncthreads();
-    for (int w = 0; w < kPassWarps; ++w) {
-      if (warp == w) {
+  for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x)
+    p.Bp[(((size_t)tile * p.nchunk + chunk) * kHeadDim + i / RP) * kMaxRank + i % RP] = red[i];
+}
+
+// The stored A = A0 W (W = R1^-1 R2^-1 of the two CholeskyQR rounds): one thread per row.  Keys: a row is r_pad
+// consecutive fp16 of its slab; values: the slab is transposed ([r_pad][16 tokens]), so the threads of a slab fill
+// 32 contiguous bytes per rank index.  fp32 copy on request.
+__global__ void __launch_bounds__(256) pi_store_a_kernel(PiArgs p) {
+  __shared__ float Wm[kMaxRank * kMaxRank];
+  const int tile = blockIdx.y;
+  for (int i = threadIdx.x; i < kMaxRank * kMaxRank; i += blockDim.x) Wm[i] = p.W[(size_t)tile * 256 + i];
+  __syncthreads();
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= p.n_c) return;
+  const SegDesc& sd = p.seg;
+  const int r = sd.rank;
+  const float* a0p = p.A0 + ((size_t)tile * p.n_c + row) * kMaxRank;
+  float a0[kMaxRank], a[kMaxRank];
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
+  for (int q = 0; q < kMaxRank; ++q) a0[q] = q < r ? a0p[q] : 0.f;
 #pragma unroll
-          for (int r = 0; r < RP; ++r) red[(lane * 4 + j) * RP + r] += acc[j][r];
-      }
-      __syncthreads();
-    }
-    for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x)
-      p.Bp[(((size_t)tile * p.nchunk + chunk) * kHeadDim + i / RP) * kMaxRank + i % RP] = red[i];
+  for (int c = 0; c < kMaxRank; ++c) {
+    float v = 0.f;
+#pragma unroll
+    for (int q = 0; q < kMaxRank; ++q)
+      if (q < r && c < r) v = fmaf(a0[q], Wm[q * kMaxRank + c], v);
+    a[c] = v;
+  }
+  const int bhl = tile >> 1, side = tile & 1;
+  const int blk = row / sd.T, tib = row % sd.T, slab = tib / kSlab, ts = tib % kSlab;
+  unsigned char* rec = p.arena + sd.seg_base + (size_t)(p.bh0 + bhl) * sd.bh_stride + sd.bfac_bytes +
+                       (size_t)blk * sd.rec_bytes;
+  if (side == 0) {
+    __half2* dst = reinterpret_cast<__half2*>(rec + sd.off_ak + slab * sd.slab_a) + ts * (sd.r_pad / 2);
+#pragma unroll
+    for (int c = 0; c < kMaxRank; c += 2)
+      if (c < sd.r_pad) dst[c / 2] = __floats2half2_rn(a[c], a[c + 1]);
+  } else {
+    __half* dst = reinterpret_cast<__half*>(rec + sd.off_av + slab * sd.slab_a) + ts;
+#pragma unroll
+    for (int c = 0; c < kMaxRank; ++c)
+      if (c < sd.r_pad) dst[c * kSlab] = __float2half_rn(a[c]);
+  }
+  if (p.dbgA != nullptr) {
+    float* dd = p.dbgA + (((size_t)(p.bh0 + bhl) * 2 + side) * sd.n_c + row) * r;
+#pragma unroll
+    for (int c = 0; c < kMaxRank; ++c)
+      if (c < r) dd[c] = a[c];
   }
 }
 
@@ -582,13 +554,14 @@ __global__ void __launch_bounds__(32) pi_chol_kernel(PiArgs p, int first) {
   }
 }
 
-// Gram partials of A0 W (second round of CholeskyQR): one thread per row.
-__global__ void __launch_bounds__(256) pi_gram2_kernel(PiArgs p) {
+// Gram partials of A0 W (W = identity in the first round of CholeskyQR): one thread per row.
+__global__ void __launch_bounds__(256) pi_gram2_kernel(PiArgs p, int identity) {
   __shared__ float Wm[kMaxRank * kMaxRank];
   __shared__ float rows[8][32][kMaxRank + 1];
   __shared__ float red[8][256];
   const int tile = blockIdx.y, chunk = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int i = threadIdx.x; i < 256; i += blockDim.x) Wm[i] = p.W[(size_t)tile * 256 + i];
+  for (int i = threadIdx.x; i < 256; i += blockDim.x)
+    Wm[i] = identity ? (i / kMaxRank == i % kMaxRank ? 1.f : 0.f) : p.W[(size_t)tile * 256 + i];
   __syncthreads();
   const int r = p.rank;
   const int row0 = chunk * kChunkRows, row1 = min(p.n_c, row0 + kChunkRows);
@@ -1072,8 +1045,8 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
   if (e != cudaSuccess) return e;
   count_launches(1);
   if (sd.rank == 0) return cudaSuccess;
-  // init + per early loop (pass, reduce) + last loop (pass, chol, gram, chol, pass, reduce)
-  count_launches(1 + 2 * (job.iters - 1) + 6 + (job.iters == 1 ? 1 : 0));
+  // init + per early loop (pass, reduce) + last loop (pass, gram, chol, gram, chol, store, reduce)
+  count_launches(1 + 2 * (job.iters - 1) + 7 + (job.iters == 1 ? 1 : 0));
 
   const int tot = (int)ntiles * kHeadDim * kMaxRank;
   const float* b0 = job.B0 ? job.B0 : nullptr;
@@ -1092,11 +1065,12 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
         q.nchunk = 1;
         pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(q, 1, 0, 0);
       }
-      launch_pass<1>(pa, st);                                   // A0 = R B, Gram of A0, R^T A0
+      launch_pass<1>(pa, st);                                   // A0 = R B, R^T A0
+      pi_gram2_kernel<<<dim3(nchunk, (int)ntiles), 256, 0, st>>>(pa, 1);
       pi_chol_kernel<<<(int)ntiles, 32, 0, st>>>(pa, 1);        // A <- Q(A) by CholeskyQR, twice
-      pi_gram2_kernel<<<dim3(nchunk, (int)ntiles), 256, 0, st>>>(pa);
+      pi_gram2_kernel<<<dim3(nchunk, (int)ntiles), 256, 0, st>>>(pa, 0);
       pi_chol_kernel<<<(int)ntiles, 32, 0, st>>>(pa, 0);
-      launch_pass<2>(pa, st);                                   // store A = A0 W
+      pi_store_a_kernel<<<dim3((sd.n_c + 255) / 256, (int)ntiles), 256, 0, st>>>(pa);   // A = A0 W
       pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(pa, 0, 1, 1);
     }
   }
