@@ -57,30 +57,37 @@ def main():
     ap.add_argument("--buffer", type=int, default=64)
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--fp16-max-batch", type=int, default=64)
+    ap.add_argument("--state", default="s1", choices=["s1", "s2"],
+                    help="s1: one prefill segment of `context` tokens + half a buffer; "
+                         "s2: prefill of context/2 tokens, then context/2 tokens pushed one by one "
+                         "(context/2/buffer flushed segments) + half a buffer")
     args = ap.parse_args()
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     H, n, L = args.heads, args.context, args.layers
     for B in [int(x) for x in args.batches.split(",")]:
-        shape = (B, H, n, 128)
         cfg = G.make_config(B, H, H, args.bits, args.group, args.s_pct, args.buffer, args.rank, n + 2 * args.buffer,
                             rank_max=args.rank, seed=B)
-        k, v = _kv(shape, H, dev, 100 + B)
-        probe = G.gear_compress(None, cfg, k, v, n, args.rank, None)
-        tok = torch.randn(B, H, 128, device=dev).half()
-        for _ in range(args.buffer // 2):
-            G.gear_append_buffer(probe, tok, tok)
+        n_pre = n if args.state == "s1" else n // 2
+        n_push = args.buffer // 2 + (0 if args.state == "s1" else n - n_pre)
+        shape = (B, H, n_pre, 128)
+        toks = torch.randn(16, B, H, 128, device=dev).half()
+
+        def build(seed):
+            k, v = _kv(shape, H, dev, seed)
+            c = G.gear_compress(None, cfg, k, v, n_pre, args.rank, None)
+            del k, v
+            for i in range(n_push):
+                G.gear_append_buffer(c, toks[i % 16], toks[(i + 5) % 16])
+            return c
+        probe = build(100 + B)
         by = G.gear_cache_bytes(probe)
         read = by.codes + by.scale_zero + by.outliers + by.lowrank_a + by.lowrank_b + by.buffer
         # distinct resident caches: enough that a step's working set is well beyond the 126 MB L2
         resident = max(1, min(L, int(1.2e9 // max(read, 1)) + 1))
         caches = [probe]
         for i in range(1, resident):
-            k, v = _kv(shape, H, dev, 100 + B + 1000 * i)
-            c = G.gear_compress(None, cfg, k, v, n, args.rank, None)
-            for _ in range(args.buffer // 2):
-                G.gear_append_buffer(c, tok, tok)
-            caches.append(c)
+            caches.append(build(100 + B + 1000 * i))
         q = torch.randn(B, H, 128, device=dev).half()
         out = torch.empty(B, H, 128, dtype=torch.float32, device=dev)
 
@@ -88,7 +95,7 @@ def main():
             for layer in range(L):
                 G.gear_decode_attn(caches[layer % resident], q, out)
         t_gear = _time(step, args.reps)
-        line = {"batch": B, "layers": L, "context": n, "resident_caches": resident,
+        line = {"batch": B, "layers": L, "context": n, "state": args.state, "resident_caches": resident,
                 "gear": {"step_ms": t_gear * 1e3, "tokens_per_s": B / t_gear, "gbs": L * read / t_gear / 1e9,
                          "cache_gb_all_layers": L * by.stored_total / 1e9}}
         fp16_bytes = 2 * B * H * (n + args.buffer // 2) * 128 * 2
@@ -111,7 +118,6 @@ def main():
         print(json.dumps(line), flush=True)
         for c in caches:
             G.gear_free(c)
-        del k, v
         G.gear_release_workspace()
         torch.cuda.empty_cache()
 
