@@ -168,7 +168,7 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
   int o = 0;
   w.sdp = 0;
   w.sdc = o;     o += 128;
-  w.qf = o;      o += HP * kHeadDim * 4;
+  w.qf = o;      o += HP == 1 ? kHeadDim * 4 : 0;   // grouped queries rebuild it from qs: their warps are short of shared memory
   w.qs = o;      o += HP * kHeadDim * 2;
   w.frag = o;    o += round_up(NT * frag_rows * frs * 4, 16);
   w.corr_k = o;  o += HP * max_T * 4;
@@ -270,7 +270,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
   const int NS = a.nstage;
   unsigned char* ring = smem + a.ws.ring;
   SegDesc* sdc = reinterpret_cast<SegDesc*>(smem + a.ws.sdc);
-  float* qf = reinterpret_cast<float*>(smem + a.ws.qf);          // [HP][128] q * scale * log2(e)
+  float* qf = reinterpret_cast<float*>(smem + a.ws.qf);          // [128] q * scale * log2(e) (one query head per pass only)
   __half* qs = reinterpret_cast<__half*>(smem + a.ws.qs);        // [HP][128] q
   uint32_t* frag = reinterpret_cast<uint32_t*>(smem + a.ws.frag);
   int* corr_k = reinterpret_cast<int*>(smem + a.ws.corr_k);      // [HP][maxT]
@@ -456,7 +456,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
         const __half2 q01 = u32_as_h2(v.x), q23 = u32_as_h2(v.y);
         const float4 qv = make_float4(__low2float(q01) * a.scale_log2, __high2float(q01) * a.scale_log2,
                                       __low2float(q23) * a.scale_log2, __high2float(q23) * a.scale_log2);
-        *reinterpret_cast<float4*>(qf + h * kHeadDim + lane * 4) = qv;
+        if (HP == 1) *reinterpret_cast<float4*>(qf + h * kHeadDim + lane * 4) = qv;
         *reinterpret_cast<float4*>(ocorr + h * kHeadDim + lane * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
         float mx = fmaxf(fmaxf(fabsf(qv.x), fabsf(qv.y)), fmaxf(fabsf(qv.z), fabsf(qv.w)));
 #pragma unroll
@@ -587,7 +587,15 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
 #pragma unroll
         for (int h = 0; h < HP; ++h) {
           if (h < HPu) {
-            const float4 qv = *reinterpret_cast<const float4*>(qf + h * kHeadDim + lane * 4);
+            float4 qv;
+            if (HP == 1) {
+              qv = *reinterpret_cast<const float4*>(qf + h * kHeadDim + lane * 4);
+            } else {
+              const uint2 qh = *reinterpret_cast<const uint2*>(qs + h * kHeadDim + lane * 4);
+              const __half2 q01 = u32_as_h2(qh.x), q23 = u32_as_h2(qh.y);
+              qv = make_float4(__low2float(q01) * a.scale_log2, __high2float(q01) * a.scale_log2,
+                               __low2float(q23) * a.scale_log2, __high2float(q23) * a.scale_log2);
+            }
             uint32_t hiA, loA, hiB, loB;
             split_hi_lo(qv.x * sc4[0], qv.y * sc4[1], hiA, loA);
             split_hi_lo(qv.z * sc4[2], qv.w * sc4[3], hiB, loB);
