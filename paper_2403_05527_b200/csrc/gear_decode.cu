@@ -753,6 +753,39 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
       }
       release();                                      // the key item is consumed
 
+      // after the running maximum grew: everything accumulated so far is scaled by alpha (per head)
+      auto apply_alpha = [&](const float (&alpha)[HP]) {                                      // warp-uniform: m_run is the same in every lane
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            float al = alpha[4 * nt];
+#pragma unroll
+            for (int hh = 1; hh < 4; ++hh)
+              if (4 * nt + hh < HP && t == hh) al = alpha[4 * nt + hh];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) U[nt][i] *= al;
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+              for (int i = 0; i < 4; ++i) O[mt][nt][i] *= al;
+          }
+#pragma unroll
+          for (int h = 0; h < HP; ++h) {
+            if (h < HPu) {
+#pragma unroll
+              for (int g = 0; g < NGV; ++g) cm[h][g] *= alpha[h];
+              float4* oc = reinterpret_cast<float4*>(ocorr + h * kHeadDim + lane * 4);
+              float4 v = *oc;
+              v.x *= alpha[h]; v.y *= alpha[h]; v.z *= alpha[h]; v.w *= alpha[h];
+              *oc = v;
+            }
+          }
+              };
+      // One query head and a compile-time block shape: the softmax, the value operands and the value outliers run as
+      // one pass over this lane's token pairs with the probabilities in registers (the value item is waited for
+      // first, since its scales are needed).  Every other case takes the separate passes below.
+      constexpr bool kFuse = HP == 1 && !S::kDyn && !is_buf;
+      unsigned char* stV = nullptr;
+      if (!kFuse) {
       // ---------------- online softmax over the block: one rescale at most
       {
         float alpha[HP];
@@ -792,37 +825,13 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
             l_run[h] = fmaf(l_run[h], alpha[h], l);
           }
         }
-        if (grew) {                                      // warp-uniform: m_run is the same in every lane
-#pragma unroll
-          for (int nt = 0; nt < NT; ++nt) {
-            float al = alpha[4 * nt];
-#pragma unroll
-            for (int hh = 1; hh < 4; ++hh)
-              if (4 * nt + hh < HP && t == hh) al = alpha[4 * nt + hh];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) U[nt][i] *= al;
-#pragma unroll
-            for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-              for (int i = 0; i < 4; ++i) O[mt][nt][i] *= al;
-          }
-#pragma unroll
-          for (int h = 0; h < HP; ++h) {
-            if (h < HPu) {
-#pragma unroll
-              for (int g = 0; g < NGV; ++g) cm[h][g] *= alpha[h];
-              float4* oc = reinterpret_cast<float4*>(ocorr + h * kHeadDim + lane * 4);
-              float4 v = *oc;
-              v.x *= alpha[h]; v.y *= alpha[h]; v.z *= alpha[h]; v.w *= alpha[h];
-              *oc = v;
-            }
-          }
-        }
+        if (grew) apply_alpha(alpha);
       }
       __syncwarp();
+      }
 
       // ================================================================ value item
-      unsigned char* stV = acquire();
+      stV = acquire();
       if (!alive) return;
       const unsigned char* vp = stV + a.bregion;          // value part of the record
       uint32_t* fragV = frag;                                         // [NT][NGV][nslab] rows of kFragStride words
@@ -836,6 +845,87 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
         fence_async_smem();
       }
 
+      if (kFuse) {
+        constexpr int NPR = S::T >= 64 ? S::T / 64 : 1;   // token pairs per lane
+        const float Sik = pow2i(-sexp_k[0]);
+        float2 sc[NPR];
+        float mx = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < NPR; ++i) {
+          const int tp = 2 * (lane + 32 * i);
+          float2 v = *reinterpret_cast<const float2*>(ps + tp);
+          v.x += c_zero[0]; v.y += c_zero[0];
+          if (k2k > 0) {
+            const int2 c = *reinterpret_cast<const int2*>(corr_k + tp);
+            v.x = fmaf((float)c.x, Sik, v.x);
+            v.y = fmaf((float)c.y, Sik, v.y);
+            *reinterpret_cast<int2*>(corr_k + tp) = make_int2(0, 0);
+          }
+          sc[i] = v;
+          mx = fmaxf(mx, fmaxf(v.x, v.y));
+        }
+        mx = warp_max(mx);
+        float alpha[HP];
+        alpha[0] = 1.f;
+        const float m_new = fmaxf(m_run[0], mx);
+        if (m_new > m_run[0]) {                           // warp-uniform
+          alpha[0] = exp2f(m_run[0] - m_new);
+          m_run[0] = m_new;
+          apply_alpha(alpha);
+        }
+        const float Sv = pow2i(clamp60(21 - float_exponent(dmax_v)));
+        const __half2* vsz = reinterpret_cast<const __half2*>(vp + o_vsz);
+        float l = 0.f;
+#pragma unroll
+        for (int i = 0; i < NPR; ++i) {
+          const int pr = lane + 32 * i, tp = 2 * pr;
+          const int s = pr >> 3, pi = pr & 7, tw = pi & 3, rg = pi >> 2;
+          const float p0 = exp2f(sc[i].x - m_new), p1 = exp2f(sc[i].y - m_new);
+          l += p0 + p1;
+          uint32_t hi, lo;
+          split_hi_lo(p0, p1, hi, lo);
+          uint32_t* bp = fragP + s * kFragStride + rg;
+          bp[tw * 2] = hi;
+          bp[(4 + tw) * 2] = lo;
+          float zero[2][NGV];
+#pragma unroll
+          for (int g = 0; g < NGV; ++g) {
+            const __half2 z0 = vsz[tp * NGV + g], z1 = vsz[(tp + 1) * NGV + g];
+            split_hi_lo(p0 * __low2float(z0), p1 * __low2float(z1), hi, lo);
+            uint32_t* bv = fragV + (g * nslab + s) * kFragStride + rg;
+            bv[tw * 2] = hi;
+            bv[(4 + tw) * 2] = lo;
+            zero[0][g] = __high2float(z0); zero[1][g] = __high2float(z1);
+            cm[0][g] = fmaf(p0, zero[0][g], fmaf(p1, zero[1][g], cm[0][g]));
+          }
+          if (k2v > 0) {                                  // sparse value term of the two tokens, scattered in fixed point
+#pragma unroll
+            for (int e2 = 0; e2 < 2; ++e2) {
+              const int tk = tp + e2;
+              const float pS = (e2 == 0 ? p0 : p1) * Sv;
+              auto v_entry = [&](int g, float val, int idx) {
+                atomicAdd(&corr_v[g * GV + idx], __float2int_rn(pS * (val - zero[e2][g])));
+              };
+              if (NGV * k2v == 4) {
+                const uint2 ov = reinterpret_cast<const uint2*>(vp + o_voval)[tk];
+                const uint32_t oi = reinterpret_cast<const uint32_t*>(vp + o_voidx)[tk];
+                v_entry(0, __low2float(u32_as_h2(ov.x)), oi & 0xFFu);
+                v_entry(0, __high2float(u32_as_h2(ov.x)), (oi >> 8) & 0xFFu);
+                v_entry(NGV == 2 ? 1 : 0, __low2float(u32_as_h2(ov.y)), (oi >> 16) & 0xFFu);
+                v_entry(NGV == 2 ? 1 : 0, __high2float(u32_as_h2(ov.y)), oi >> 24);
+              } else {
+                const __half* ov = reinterpret_cast<const __half*>(vp + o_voval) + (size_t)tk * NGV * k2v;
+                const unsigned char* oi = vp + o_voidx + (size_t)tk * NGV * k2v;
+#pragma unroll
+                for (int g = 0; g < NGV; ++g)
+#pragma unroll 1
+                  for (int e = 0; e < k2v; ++e) v_entry(g, __half2float(ov[g * k2v + e]), oi[g * k2v + e]);
+              }
+            }
+          }
+        }
+        l_run[0] = fmaf(l_run[0], alpha[0], l);
+      } else {
       // ---------------- B operands of the value products: p * scale (per token and group) and p, split hi / lo;
       //                  the zero-point term goes to the fp32 side sums cm
 #pragma unroll (TU)
@@ -868,6 +958,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
             }
           }
         }
+      }
       }
       __syncwarp();
 
@@ -959,7 +1050,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
         const unsigned char* voval = vp + o_voval;
         const unsigned char* voidx = vp + o_voidx;
 #pragma unroll (TU)
-        for (int tk = lane; tk < T; tk += 32) {
+        for (int tk = lane; tk < (kFuse ? 0 : T); tk += 32) {      // the fused pass above has scattered them already
           float pS[HP];
 #pragma unroll
           for (int h = 0; h < HP; ++h) pS[h] = h < HPu ? ps[h * maxT + tk] * S : 0.f;
