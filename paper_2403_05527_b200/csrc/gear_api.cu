@@ -365,15 +365,33 @@ extern "C" gear_status gear_decode_attn(gear_cache* c, const void* q, float* out
   const long long work = (long long)c->cc.BH * ((c->G + hp - 1) / hp) * (c->n_blocks_c + (c->buf_len + 15) / 16);
   long long grid = (long long)c->sm_count * c->plan_occ;
   if (grid > work) grid = work;
-  // When the warps that fit divide almost evenly among the units, cut every unit into the same number of ranges: a
-  // warp that runs from one unit into the next pays a second prologue and epilogue, and with few blocks per warp those
-  // warps finish last.  Otherwise (many blocks per warp, or a poor fit) cut the flat space evenly.
+  // With few blocks per warp, a warp that runs from one unit into the next pays a second prologue and epilogue and
+  // finishes last.  When every unit gets at least six warps, cut each unit into ranges of its own instead: the first
+  // units into one range more than the others so that every resident warp has work, and order the CTAs by the length
+  // of their range, longest first (the hardware dispatches them in index order, and the oldest warps of an SM
+  // finish first).  Otherwise (many blocks per warp) cut the flat space evenly.
   {
     const long long units = (long long)c->cc.BH * ((c->G + hp - 1) / hp), nb = work / units;
-    const long long ppu = grid / units;
-    if (ppu >= 1 && ppu <= nb && ppu < c->max_parts && units * ppu * 100 >= grid * 96) {
-      a.parts_per_unit = (int)ppu;
-      grid = units * ppu;
+    const long long pb = grid / units, ua = grid - pb * units;         // ua units get pb + 1 ranges
+    if (pb >= 6 && pb + 1 <= nb && pb + 1 < c->max_parts) {
+      a.aligned = 1;
+      a.units_a = (int)ua; a.parts_a = (int)pb + 1; a.parts_b = (int)pb;
+      struct Cls { int len, u0, nu, p0, n; } cls[4];
+      const int base_a = (int)(nb / (pb + 1)), rem_a = (int)(nb % (pb + 1));
+      const int base_b = (int)(nb / pb), rem_b = (int)(nb % pb);
+      cls[0] = {base_b + 1, (int)ua, (int)(units - ua), 0, rem_b};
+      cls[1] = {base_b, (int)ua, (int)(units - ua), rem_b, (int)pb - rem_b};
+      cls[2] = {base_a + 1, 0, (int)ua, 0, rem_a};
+      cls[3] = {base_a, 0, (int)ua, rem_a, (int)pb + 1 - rem_a};
+      for (int i = 1; i < 4; ++i)                                       // insertion sort, longest first, stable
+        for (int j = i; j > 0 && cls[j].len > cls[j - 1].len; --j) { const Cls t = cls[j]; cls[j] = cls[j - 1]; cls[j - 1] = t; }
+      int start = 0;
+      for (int k = 0; k < 4; ++k) {
+        a.cls_start[k] = start; a.cls_u0[k] = cls[k].u0; a.cls_n[k] = cls[k].n > 0 ? cls[k].n : 1; a.cls_p0[k] = cls[k].p0;
+        start += cls[k].nu * cls[k].n;
+      }
+      a.cls_start[4] = start;
+      grid = start;                                                     // = units * pb + ua
     }
   }
   if (launch_decode(a, (int)grid, (cudaStream_t)stream) != cudaSuccess) {

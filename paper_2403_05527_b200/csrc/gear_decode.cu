@@ -187,7 +187,7 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
     if (ns < 2) continue;
     if (ns > kMaxStages) ns = kMaxStages;
     w.total = w.ring + (int)ns * stage;
-    a->parts_per_unit = 0;
+    a->aligned = 0;
     a->nstage = (int)ns; a->stage_bytes = stage; a->bregion = bregion; a->max_T = max_T; a->hpa = HP; a->ws = w;
     return true;
   }
@@ -301,21 +301,16 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
   const int nbuf_blocks = (a.buf_len + kSlab - 1) / kSlab;
   const int NB = a.n_blocks_c + nbuf_blocks;
   int n_left, u, blk_lo;                        // blocks left for this warp, current unit, first block in it
-  int part = 0;                                 // unit-aligned split: this warp's range inside its unit
-  if (a.parts_per_unit > 0) {
-    // No warp crosses from one unit into the next.  NB blocks over P ranges leave NB % P ranges one block longer;
-    // those get the lowest CTA indices of the grid (longest first: they are dispatched first and finish with the rest).
-    const int P = a.parts_per_unit, base = NB / P, rem = NB - base * P;     // base > 0: the host keeps P <= NB
-    const int n_long = a.cc.BH * passes * rem;
-    if ((int)blockIdx.x < n_long) {
-      u = blockIdx.x / rem;
-      part = blockIdx.x - u * rem;
-    } else {
-      const int b2 = blockIdx.x - n_long;
-      u = b2 / (P - rem);
-      part = rem + b2 - u * (P - rem);
-    }
-    blk_lo = part * base + min(part, rem);
+  int part = 0, parts_u = 0;                    // unit-aligned split: this warp's range inside its unit, ranges of the unit
+  if (a.aligned) {
+    int k = 0;
+    while (k < 3 && (int)blockIdx.x >= a.cls_start[k + 1]) ++k;
+    const int idx = blockIdx.x - a.cls_start[k];
+    u = a.cls_u0[k] + idx / a.cls_n[k];
+    part = a.cls_p0[k] + idx % a.cls_n[k];
+    parts_u = u < a.units_a ? a.parts_a : a.parts_b;
+    const int base = NB / parts_u, rem = NB - base * parts_u;       // base > 0: the host keeps parts <= NB
+    blk_lo = part * base + min(part, rem);                          // the first `rem` ranges are one block longer
     n_left = base + (part < rem ? 1 : 0);
   } else {
     const long long F = (long long)a.cc.BH * passes * NB;
@@ -1150,8 +1145,8 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
 
     // ---------------- partial result of this unit: (m, l, o) per head
     int n_parts, slot;
-    if (a.parts_per_unit > 0) {
-      n_parts = a.parts_per_unit;
+    if (a.aligned) {
+      n_parts = parts_u;
       slot = part;
     } else {
       const long long F = (long long)a.cc.BH * passes * NB, NW = gridDim.x;

@@ -81,8 +81,13 @@ struct DecodeArgs {
   int buf_len;                // tokens in the fp16 buffer
   int n_kv_heads, group_heads;   // H, G = Hq / H
   int max_parts;
-  int parts_per_unit;         // > 0: every unit is cut into this many ranges, one per warp (grid = units * parts);
-                              // 0: the flat (unit, block) space is cut into gridDim.x equal ranges
+  // Unit-aligned split (aligned != 0): no warp crosses from one unit into the next.  Units [0, units_a) are cut into
+  // parts_a ranges, the others into parts_b = parts_a - 1; the CTAs are ordered by the length of their range,
+  // longest first, in up to four classes (unit type x one-block-longer or not): class k holds the CTAs
+  // [cls_start[k], cls_start[k + 1]), cls_n[k] consecutive parts from cls_p0[k] on per unit, units from cls_u0[k] on.
+  // aligned == 0: the flat (unit, block) space is cut into gridDim.x equal ranges.
+  int aligned, units_a, parts_a, parts_b;
+  int cls_start[5], cls_u0[4], cls_n[4], cls_p0[4];
   int nstage;                 // ring stages (<= kMaxStages)
   int stage_bytes;            // bytes of one ring stage
   int bregion;                // bytes at the front of a stage reserved for one B factor
