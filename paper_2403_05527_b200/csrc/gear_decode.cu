@@ -775,10 +775,10 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
             }
           }
               };
-      // One query head and a compile-time block shape: the softmax, the value operands and the value outliers run as
-      // one pass over this lane's token pairs with the probabilities in registers (the value item is waited for
-      // first, since its scales are needed).  Every other case takes the separate passes below.
-      constexpr bool kFuse = HP == 1 && !S::kDyn && !is_buf;
+      // Up to four query heads and a compile-time block shape: the softmax, the value operands and the value outliers
+      // run as one pass over this lane's token pairs with the probabilities in registers (the value item is waited
+      // for first, since its scales are needed).  Every other case takes the separate passes below.
+      constexpr bool kFuse = HP <= 4 && !S::kDyn && !is_buf;
       unsigned char* stV = nullptr;
       if (!kFuse) {
       // ---------------- online softmax over the block: one rescale at most
@@ -842,64 +842,84 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
 
       if (kFuse) {
         constexpr int NPR = S::T >= 64 ? S::T / 64 : 1;   // token pairs per lane
-        const float Sik = pow2i(-sexp_k[0]);
-        float2 sc[NPR];
-        float mx = -INFINITY;
+        float2 sc[HP][NPR];
+        float alpha[HP], m_new[HP];
+        bool grew = false;
 #pragma unroll
-        for (int i = 0; i < NPR; ++i) {
-          const int tp = 2 * (lane + 32 * i);
-          float2 v = *reinterpret_cast<const float2*>(ps + tp);
-          v.x += c_zero[0]; v.y += c_zero[0];
-          if (k2k > 0) {
-            const int2 c = *reinterpret_cast<const int2*>(corr_k + tp);
-            v.x = fmaf((float)c.x, Sik, v.x);
-            v.y = fmaf((float)c.y, Sik, v.y);
-            *reinterpret_cast<int2*>(corr_k + tp) = make_int2(0, 0);
+        for (int h = 0; h < HP; ++h) {
+          alpha[h] = 1.f; m_new[h] = 0.f;
+          if (h < HPu) {
+            const float Sik = pow2i(-sexp_k[h]);
+            float mx = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < NPR; ++i) {
+              const int tp = 2 * (lane + 32 * i);
+              float2 v = *reinterpret_cast<const float2*>(ps + h * maxT + tp);
+              v.x += c_zero[h]; v.y += c_zero[h];
+              if (k2k > 0) {
+                const int2 c = *reinterpret_cast<const int2*>(corr_k + h * maxT + tp);
+                v.x = fmaf((float)c.x, Sik, v.x);
+                v.y = fmaf((float)c.y, Sik, v.y);
+                *reinterpret_cast<int2*>(corr_k + h * maxT + tp) = make_int2(0, 0);
+              }
+              sc[h][i] = v;
+              mx = fmaxf(mx, fmaxf(v.x, v.y));
+            }
+            mx = warp_max(mx);
+            m_new[h] = fmaxf(m_run[h], mx);
+            if (m_new[h] > m_run[h]) {                    // warp-uniform
+              alpha[h] = exp2f(m_run[h] - m_new[h]);
+              m_run[h] = m_new[h];
+              grew = true;
+            }
           }
-          sc[i] = v;
-          mx = fmaxf(mx, fmaxf(v.x, v.y));
         }
-        mx = warp_max(mx);
-        float alpha[HP];
-        alpha[0] = 1.f;
-        const float m_new = fmaxf(m_run[0], mx);
-        if (m_new > m_run[0]) {                           // warp-uniform
-          alpha[0] = exp2f(m_run[0] - m_new);
-          m_run[0] = m_new;
-          apply_alpha(alpha);
-        }
+        if (grew) apply_alpha(alpha);
         const float Sv = pow2i(clamp60(21 - float_exponent(dmax_v)));
         const __half2* vsz = reinterpret_cast<const __half2*>(vp + o_vsz);
-        float l = 0.f;
+        float l[HP];
+#pragma unroll
+        for (int h = 0; h < HP; ++h) l[h] = 0.f;
 #pragma unroll
         for (int i = 0; i < NPR; ++i) {
           const int pr = lane + 32 * i, tp = 2 * pr;
           const int s = pr >> 3, pi = pr & 7, tw = pi & 3, rg = pi >> 2;
-          const float p0 = exp2f(sc[i].x - m_new), p1 = exp2f(sc[i].y - m_new);
-          l += p0 + p1;
-          uint32_t hi, lo;
-          split_hi_lo(p0, p1, hi, lo);
-          uint32_t* bp = fragP + s * kFragStride + rg;
-          bp[tw * 2] = hi;
-          bp[(4 + tw) * 2] = lo;
-          float zero[2][NGV];
+          float p[HP][2];
+          __half2 z[2][NGV];
 #pragma unroll
-          for (int g = 0; g < NGV; ++g) {
-            const __half2 z0 = vsz[tp * NGV + g], z1 = vsz[(tp + 1) * NGV + g];
-            split_hi_lo(p0 * __low2float(z0), p1 * __low2float(z1), hi, lo);
-            uint32_t* bv = fragV + (g * nslab + s) * kFragStride + rg;
-            bv[tw * 2] = hi;
-            bv[(4 + tw) * 2] = lo;
-            zero[0][g] = __high2float(z0); zero[1][g] = __high2float(z1);
-            cm[0][g] = fmaf(p0, zero[0][g], fmaf(p1, zero[1][g], cm[0][g]));
+          for (int g = 0; g < NGV; ++g) { z[0][g] = vsz[tp * NGV + g]; z[1][g] = vsz[(tp + 1) * NGV + g]; }
+#pragma unroll
+          for (int h = 0; h < HP; ++h) {
+            p[h][0] = p[h][1] = 0.f;
+            if (h < HPu) {
+              const float p0 = exp2f(sc[h][i].x - m_new[h]), p1 = exp2f(sc[h][i].y - m_new[h]);
+              p[h][0] = p0; p[h][1] = p1;
+              l[h] += p0 + p1;
+              const int col = 2 * (h & 3);
+              uint32_t hi, lo;
+              split_hi_lo(p0, p1, hi, lo);
+              uint32_t* bp = fragP + ((h >> 2) * nslab + s) * kFragStride + rg;
+              bp[(col * 4 + tw) * 2] = hi;
+              bp[((col + 1) * 4 + tw) * 2] = lo;
+#pragma unroll
+              for (int g = 0; g < NGV; ++g) {
+                split_hi_lo(p0 * __low2float(z[0][g]), p1 * __low2float(z[1][g]), hi, lo);
+                uint32_t* bv = fragV + (((h >> 2) * NGV + g) * nslab + s) * kFragStride + rg;
+                bv[(col * 4 + tw) * 2] = hi;
+                bv[((col + 1) * 4 + tw) * 2] = lo;
+                cm[h][g] = fmaf(p0, __high2float(z[0][g]), fmaf(p1, __high2float(z[1][g]), cm[h][g]));
+              }
+            }
           }
           if (k2v > 0) {                                  // sparse value term of the two tokens, scattered in fixed point
 #pragma unroll
             for (int e2 = 0; e2 < 2; ++e2) {
               const int tk = tp + e2;
-              const float pS = (e2 == 0 ? p0 : p1) * Sv;
               auto v_entry = [&](int g, float val, int idx) {
-                atomicAdd(&corr_v[g * GV + idx], __float2int_rn(pS * (val - zero[e2][g])));
+                const float d = (val - __high2float(z[e2][g])) * Sv;
+#pragma unroll
+                for (int h = 0; h < HP; ++h)
+                  if (h < HPu) atomicAdd(&corr_v[h * kHeadDim + g * GV + idx], __float2int_rn(p[h][e2] * d));
               };
               if (NGV * k2v == 4) {
                 const uint2 ov = reinterpret_cast<const uint2*>(vp + o_voval)[tk];
@@ -919,7 +939,9 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
             }
           }
         }
-        l_run[0] = fmaf(l_run[0], alpha[0], l);
+#pragma unroll
+        for (int h = 0; h < HP; ++h)
+          if (h < HPu) l_run[h] = fmaf(l_run[h], alpha[h], l[h]);
       } else {
       // ---------------- B operands of the value products: p * scale (per token and group) and p, split hi / lo;
       //                  the zero-point term goes to the fp32 side sums cm
