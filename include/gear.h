@@ -124,12 +124,15 @@ void gear_free(gear_cache* cache);
  * to the driver.  This call synchronises the current device and returns that memory to the driver. */
 gear_status gear_release_workspace(void);
 
-/* ---- host-buffer variants (copies inside the call; they synchronise `stream`) ---- */
+/* ---- host-buffer variants (copies inside the call) ---- */
 
-/* gear_append_buffer with k_new, v_new (and B0_flush) in HOST memory. */
+/* gear_append_buffer with k_new, v_new (and B0_flush) in HOST memory (pinned or pageable).  The rows are copied
+ * to pinned memory of the library before the call returns, so the caller may reuse its buffers at once; the call
+ * does not wait for the device, except when it passes B0_flush on to a flush (that array is read in place, and
+ * the call then synchronises `stream`).  Calls on one cache must use one stream. */
 gear_status gear_append_buffer_host(gear_cache* cache, const void* k_new_host, const void* v_new_host,
                                     const float* B0_flush_host, void* stream);
-/* gear_decode_attn with q and out in HOST memory. */
+/* gear_decode_attn with q and out in HOST memory; synchronises `stream` (out_host is valid on return). */
 gear_status gear_decode_attn_host(gear_cache* cache, const void* q_host, float* out_host,
                                   float softmax_scale, void* stream);
 

@@ -71,6 +71,10 @@ struct gear_cache {
   float* partial; size_t partial_bytes; int max_parts;
   int* tickets; int* status;
   void* stage_k; void* stage_v; void* stage_q; float* stage_out; float* stage_b0;   // for the *_host calls
+  // gear_append_buffer_host: pinned copies of the caller's rows, so that the call neither waits for the device nor
+  // holds on to the caller's memory.  A slot is reused once the copy that read it has finished (its event).
+  static constexpr int kHostSlots = 4;
+  unsigned char* host_ring[kHostSlots]; cudaEvent_t host_ev[kHostSlots]; bool host_used[kHostSlots]; int host_next;
   // host state
   std::vector<SegDesc> segs;
   std::vector<long long> dbgA_off, dbgB_off;             // float offsets into dbg (or -1)
@@ -127,7 +131,11 @@ extern "C" void gear_free(gear_cache* c) {
   if (!c) return;
   cudaFree(c->arena); cudaFree(c->dbg); cudaFree(c->table_dev); cudaFree(c->blk2seg); cudaFree(c->buf_k); cudaFree(c->buf_v);
   cudaFree(c->flush_ws); cudaFree(c->partial); cudaFree(c->tickets); cudaFree(c->status);
-  cudaFree(c->stage_k); cudaFree(c->stage_v); cudaFree(c->stage_q); cudaFree(c->stage_out); cudaFree(c->stage_b0);
+  cudaFree(c->stage_k); cudaFree(c->stage_q); cudaFree(c->stage_out); cudaFree(c->stage_b0);
+  for (int i = 0; i < gear_cache::kHostSlots; ++i) {
+    if (c->host_ring[i]) cudaFreeHost(c->host_ring[i]);
+    if (c->host_ev[i]) cudaEventDestroy(c->host_ev[i]);
+  }
   delete c;
 }
 
@@ -150,6 +158,8 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   c->arena = nullptr; c->dbg = nullptr; c->table_dev = nullptr; c->blk2seg = nullptr; c->buf_k = c->buf_v = nullptr; c->flush_ws = nullptr;
   c->partial = nullptr; c->tickets = nullptr; c->status = nullptr;
   c->stage_k = c->stage_v = c->stage_q = nullptr; c->stage_out = nullptr; c->stage_b0 = nullptr;
+  for (int i = 0; i < gear_cache::kHostSlots; ++i) { c->host_ring[i] = nullptr; c->host_ev[i] = nullptr; c->host_used[i] = false; }
+  c->host_next = 0;
   c->cc.bits = cfg->bits;
   c->cc.g_v = cfg->group < kHeadDim ? cfg->group : kHeadDim;
   c->cc.ngv = kHeadDim / c->cc.g_v;
@@ -204,8 +214,16 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   cudaMemset(c->tickets, 0, units * 4);
   cudaMemset(c->status, 0, 4);
   const size_t tok_bytes = BH * kHeadDim * 2;
-  GEAR_TRY_ALLOC(c->stage_k, tok_bytes);
-  GEAR_TRY_ALLOC(c->stage_v, tok_bytes);
+  GEAR_TRY_ALLOC(c->stage_k, 2 * tok_bytes);          // key row, then value row: one copy brings both
+  c->stage_v = reinterpret_cast<unsigned char*>(c->stage_k) + tok_bytes;
+  for (int i = 0; i < gear_cache::kHostSlots; ++i) {
+    if (cudaHostAlloc((void**)&c->host_ring[i], 2 * tok_bytes, cudaHostAllocDefault) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->host_ev[i], cudaEventDisableTiming) != cudaSuccess) {
+      cudaGetLastError();
+      gear_free(c);
+      return GEAR_ERR_ALLOC;
+    }
+  }
   GEAR_TRY_ALLOC(c->stage_q, (size_t)cfg->batch * cfg->n_q_heads * kHeadDim * 2);
   GEAR_TRY_ALLOC(c->stage_out, (size_t)cfg->batch * cfg->n_q_heads * kHeadDim * 4);
   GEAR_TRY_ALLOC(c->stage_b0, BH * 2 * kHeadDim * (size_t)(cfg->rank_flush > 0 ? cfg->rank_flush : 1) * 4);
@@ -406,13 +424,22 @@ extern "C" gear_status gear_append_buffer_host(gear_cache* c, const void* k_host
   if (!c || !k_host || !v_host) return GEAR_ERR_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t tok_bytes = (size_t)c->cc.BH * kHeadDim * 2;
-  if (cudaMemcpyAsync(c->stage_k, k_host, tok_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(c->stage_v, v_host, tok_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+  // the rows go through a pinned slot of the library's own, so the caller's memory is free again on return and
+  // nothing waits for the device (a slot is waited for only if its copy of four calls ago is still running)
+  const int slot = c->host_next;
+  c->host_next = (slot + 1) % gear_cache::kHostSlots;
+  if (c->host_used[slot] && cudaEventSynchronize(c->host_ev[slot]) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
+  memcpy(c->host_ring[slot], k_host, tok_bytes);
+  memcpy(c->host_ring[slot] + tok_bytes, v_host, tok_bytes);
+  if (cudaMemcpyAsync(c->stage_k, c->host_ring[slot], 2 * tok_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaEventRecord(c->host_ev[slot], st) != cudaSuccess) {
     cudaGetLastError();
     return GEAR_ERR_CUDA;
   }
+  c->host_used[slot] = true;
   const float* b0 = nullptr;
-  if (B0_host && c->cfg.rank_flush > 0 && c->buf_len + 1 == c->cfg.buffer_cap) {
+  const bool with_b0 = B0_host && c->cfg.rank_flush > 0 && c->buf_len + 1 == c->cfg.buffer_cap;
+  if (with_b0) {
     if (cudaMemcpyAsync(c->stage_b0, B0_host, (size_t)c->cc.BH * 2 * kHeadDim * c->cfg.rank_flush * 4,
                         cudaMemcpyHostToDevice, st) != cudaSuccess) {
       cudaGetLastError();
@@ -422,7 +449,8 @@ extern "C" gear_status gear_append_buffer_host(gear_cache* c, const void* k_host
   }
   gear_status s = gear_append_buffer(c, c->stage_k, c->stage_v, b0, stream);
   if (s < 0) return s;
-  if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
+  // the start vectors are read straight from the caller's memory: only then wait for the copy
+  if (with_b0 && cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
   return s;
 }
 
