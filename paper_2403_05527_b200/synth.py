@@ -46,6 +46,9 @@ WORKLOADS = {
     3: Workload(3, "C3 LLaMA-2-13B layer B16 H40 n8192 4-bit g64 s1 r8 nb64", 16, 40, 40, 128, 8192, 4, 64, 1.0, 8, 64),
     32: Workload(32, "C3 LLaMA-2-13B layer B16 H40 n8192 2-bit g64 s1 r8 nb64", 16, 40, 40, 128, 8192, 2, 64, 1.0, 8, 64),
     4: Workload(4, "C4 Mistral-7B GQA layer B4 Hq32 Hkv8 n32768 2-bit g128 s2 r4 nb64", 4, 32, 8, 128, 32768, 2, 128, 2.0, 4, 64),
+    # parity-only shapes that land in other branches of the decode kernel's work split (many warps per unit)
+    21: Workload(21, "T1 B2 H32 n4096 2-bit g64 s2 r4 nb64", 2, 32, 32, 128, 4096, 2, 64, 2.0, 4, 64),
+    22: Workload(22, "T2 B4 H32 n4096 4-bit g64 s2 r4 nb64", 4, 32, 32, 128, 4096, 4, 64, 2.0, 4, 64),
 }
 
 

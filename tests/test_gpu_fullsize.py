@@ -36,7 +36,8 @@ def _device_inputs(torch, w, dev, seed, n_app):
     return k, v, b0, b0f, ks, vs, q
 
 
-@pytest.mark.parametrize("config_id,units", [(2, [(0, 0), (3, 17), (7, 31)]), (4, [(0, 0), (3, 7)]), (3, [(5, 11), (15, 39)]), (32, [(2, 3)])])
+@pytest.mark.parametrize("config_id,units", [(2, [(0, 0), (3, 17), (7, 31)]), (4, [(0, 0), (3, 7)]), (3, [(5, 11), (15, 39)]), (32, [(2, 3)]),
+                                             (21, [(1, 30)]), (22, [(0, 5), (3, 31)])])
 def test_full_size_layer_sampled_units_match_the_oracle(config_id, units):
     import torch
     from oracle import gear_oracle as O
