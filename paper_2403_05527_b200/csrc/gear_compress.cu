@@ -310,14 +310,15 @@ __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row0 = chunk * kChunkRows;
   const int row1 = min(p.n_c, row0 + kChunkRows);
+  const int rho0 = blockIdx.z * RP;               // this CTA's rank columns [rho0, rho0 + RP)
   const float* R = p.R + (size_t)tile * p.n_c * kHeadDim;
-  float* A0 = p.A0 + (size_t)tile * p.n_c * kMaxRank;
+  float* A0 = p.A0 + (size_t)tile * p.n_c * kMaxRank + rho0;
 
   float b[4][RP];
 #pragma unroll
   for (int j = 0; j < 4; ++j)
 #pragma unroll
-    for (int r = 0; r < RP; ++r) b[j][r] = p.Bcur[((size_t)tile * kHeadDim + lane * 4 + j) * kMaxRank + r];
+    for (int r = 0; r < RP; ++r) b[j][r] = p.Bcur[((size_t)tile * kHeadDim + lane * 4 + j) * kMaxRank + rho0 + r];
   float acc[4][RP];       // this lane's 4 channels of R^T a
 #pragma unroll
   for (int j = 0; j < 4; ++j)
@@ -374,7 +375,7 @@ __global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
     __syncthreads();
   }
   for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x)
-    p.Bp[(((size_t)tile * p.nchunk + chunk) * kHeadDim + i / RP) * kMaxRank + i % RP] = red[i];
+    p.Bp[(((size_t)tile * p.nchunk + chunk) * kHeadDim + i / RP) * kMaxRank + rho0 + i % RP] = red[i];
 }
 
 // The stored A = A0 W (W = R1^-1 R2^-1 of the two CholeskyQR rounds): one thread per row.  Keys: a row is r_pad
@@ -996,11 +997,11 @@ static cudaError_t launch_quant(const CompressArgs& a, int nbh, int kmax_needed,
 
 template <int MODE>
 static void launch_pass(const PiArgs& p, cudaStream_t st) {
-  dim3 grid(p.nchunk, p.ntiles);
-  const int rp = p.rank <= 4 ? 4 : (p.rank <= 8 ? 8 : 16);
-  if (rp == 4) pi_pass_kernel<4, MODE><<<grid, kPassWarps * 32, 0, st>>>(p);
-  else if (rp == 8) pi_pass_kernel<8, MODE><<<grid, kPassWarps * 32, 0, st>>>(p);
-  else pi_pass_kernel<16, MODE><<<grid, kPassWarps * 32, 0, st>>>(p);
+  // Four rank columns per CTA; a higher rank is spread over gridDim.z CTAs that read the same chunk of R (the second
+  // reader finds it in L2).  With eight or sixteen columns per CTA the registers allow half the resident warps and
+  // the pass runs three times slower per byte.
+  dim3 grid(p.nchunk, p.ntiles, p.rank <= 4 ? 1 : (p.rank <= 8 ? 2 : 4));
+  pi_pass_kernel<4, MODE><<<grid, kPassWarps * 32, 0, st>>>(p);
 }
 
 size_t compress_workspace_bytes(int nbh, int n_c, int rank) {
