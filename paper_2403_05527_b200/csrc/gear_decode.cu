@@ -628,6 +628,20 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
               k_entry(j, __low2float(u32_as_h2(o4[j])), (i2[j >> 1] >> (16 * (j & 1))) & 0xFFu);
               k_entry(j, __high2float(u32_as_h2(o4[j])), (i2[j >> 1] >> (16 * (j & 1) + 8)) & 0xFFu);
             }
+          } else if (k2k == 4) {
+            // this lane's 4 channels x 4 entries: 32 bytes of values, 16 bytes of token indices
+            const uint4 ova = reinterpret_cast<const uint4*>(kp + off_koval)[2 * lane];
+            const uint4 ovb = reinterpret_cast<const uint4*>(kp + off_koval)[2 * lane + 1];
+            const uint4 oi = reinterpret_cast<const uint4*>(kp + off_koidx)[lane];
+            const uint32_t o8[8] = {ova.x, ova.y, ova.z, ova.w, ovb.x, ovb.y, ovb.z, ovb.w};
+            const uint32_t i4[4] = {oi.x, oi.y, oi.z, oi.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              k_entry(j, __low2float(u32_as_h2(o8[2 * j])), i4[j] & 0xFFu);
+              k_entry(j, __high2float(u32_as_h2(o8[2 * j])), (i4[j] >> 8) & 0xFFu);
+              k_entry(j, __low2float(u32_as_h2(o8[2 * j + 1])), (i4[j] >> 16) & 0xFFu);
+              k_entry(j, __high2float(u32_as_h2(o8[2 * j + 1])), i4[j] >> 24);
+            }
           } else {
             const __half* ov = reinterpret_cast<const __half*>(kp + off_koval) + lane * 4 * k2k;
             const unsigned char* oi = kp + off_koidx + lane * 4 * k2k;
