@@ -32,7 +32,7 @@ import numpy as np  # noqa: E402
 from paper_2403_05527_b200 import synth  # noqa: E402
 
 METRIC = "compressed-KV decode attn tokens/s"
-DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.016
+DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.015
 UNIT = "tokens/s"
 
 
@@ -190,6 +190,11 @@ def run_ours(args, w):
     cfg = G.make_config(B, w.n_q_heads, w.n_kv_heads, w.bits, w.group, w.s_pct, nb, w.rank, max_tokens,
                         rank_max=w.rank, power_iters=w.power_iters, seed=1234 + rank)
     caches, compress_ms = [], []
+    # one untimed compress first: it grows the library's workspace pool to its working size (a driver allocation
+    # that later calls do not repeat)
+    k, v = device_kv(torch, w, dev, 999 + 1000 * rank)
+    G.gear_free(G.gear_compress(G.gear_create(cfg), None, k, v, w.n, w.rank, None))
+    del k, v
     for layer in range(L):
         k, v = device_kv(torch, w, dev, 1000 * rank + layer)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
