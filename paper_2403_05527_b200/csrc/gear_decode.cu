@@ -601,14 +601,39 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
             base[(4 * cl + tA + 1) * 2] = hiB;
             base[(4 * (cl + 1) + tA + 1) * 2] = loB;
             if (!is_buf) {
-              float c = fmaf(qv.x, zr4[0], fmaf(qv.y, zr4[1], fmaf(qv.z, zr4[2], qv.w * zr4[3])));
+              float c = fmaf(qv.x, zr4[0], fmaf(qv.y, zr4[1], fmaf(qv.z, zr4[2], qv.w * zr4[3])));   // this lane's part
+              if (HP != 4) {
 #pragma unroll
-              for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+                for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+              }
               const int sexp = clamp60(21 - qexp_s[h] - ed);
               const float S = pow2i(sexp);
               qS[h][0] = qv.x * S; qS[h][1] = qv.y * S; qS[h][2] = qv.z * S; qS[h][3] = qv.w * S;
               c_zero[h] = c; sexp_k[h] = sexp;
             }
+          }
+        }
+        if (!is_buf && HP == 4) {            // c_zero of four heads: sums over the warp
+          {
+            // four sums at once: two exchange steps halve what a lane carries, a butterfly finishes the one value left
+            // (head 2 * bit4 + bit3 of the lane), four broadcasts hand the sums back: 10 shuffles instead of 20
+            float s0 = c_zero[0], s1 = c_zero[1];
+            {
+              const bool up = (lane & 16) != 0;
+              const float send0 = up ? c_zero[0] : c_zero[2], keep0 = up ? c_zero[2] : c_zero[0];
+              const float send1 = up ? c_zero[1] : c_zero[3], keep1 = up ? c_zero[3] : c_zero[1];
+              s0 = keep0 + __shfl_xor_sync(0xffffffffu, send0, 16);
+              s1 = keep1 + __shfl_xor_sync(0xffffffffu, send1, 16);
+            }
+            {
+              const bool up = (lane & 8) != 0;
+              const float send = up ? s0 : s1, keep = up ? s1 : s0;
+              s0 = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+            }
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) s0 += __shfl_xor_sync(0xffffffffu, s0, o);
+#pragma unroll
+            for (int h = 0; h < HP; ++h) c_zero[h] = __shfl_sync(0xffffffffu, s0, 8 * h);
           }
         }
         if (!is_buf && k2k > 0) {
