@@ -202,8 +202,8 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
     GEAR_TRY_ALLOC(c->dbg, c->dbg_bytes);
   }
   // decode scratch: one partial per (unit, warp touching it); upper bound of warps in a launch
-  const int hp = c->G <= 4 ? 4 : 8;
-  const int passes = (c->G + hp - 1) / hp;
+  const int hp = decode_heads_per_pass(c->G);
+  const int passes = decode_passes(c->G);
   const size_t units = BH * passes;
   const size_t nw_max = (size_t)c->sm_count * 32;        // one warp per CTA, at most 32 CTAs per SM
   c->max_parts = (int)(nw_max / units + 3);
@@ -379,8 +379,8 @@ extern "C" gear_status gear_decode_attn(gear_cache* c, const void* q, float* out
   const float sc = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)kHeadDim);
   a.scale_log2 = sc * 1.4426950408889634f;
   // one warp per CTA; never more warps than blocks of work
-  const int hp = c->G <= 4 ? 4 : 8;
-  const long long work = (long long)c->cc.BH * ((c->G + hp - 1) / hp) * (c->n_blocks_c + (c->buf_len + 15) / 16);
+  const int passes = decode_passes(c->G);
+  const long long work = (long long)c->cc.BH * passes * (c->n_blocks_c + (c->buf_len + 15) / 16);
   long long grid = (long long)c->sm_count * c->plan_occ;
   if (grid > work) grid = work;
   // With few blocks per warp, a warp that runs from one unit into the next pays a second prologue and epilogue and
@@ -389,7 +389,7 @@ extern "C" gear_status gear_decode_attn(gear_cache* c, const void* q, float* out
   // of their range, longest first (the hardware dispatches them in index order, and the oldest warps of an SM
   // finish first).  Otherwise (many blocks per warp) cut the flat space evenly.
   {
-    const long long units = (long long)c->cc.BH * ((c->G + hp - 1) / hp), nb = work / units;
+    const long long units = (long long)c->cc.BH * passes, nb = work / units;
     const long long pb = grid / units, ua = grid - pb * units;         // ua units get pb + 1 ranges
     if (pb >= 6 && pb + 1 <= nb && pb + 1 < c->max_parts) {
       a.aligned = 1;
@@ -479,6 +479,7 @@ extern "C" gear_status gear_fp16_decode_attn(const void* K, const void* V, const
                                              void* stream) {
   if (!K || !V || !q || !out || !scratch) return GEAR_ERR_ARG;
   if (batch < 1 || n_kv_heads < 1 || n_q_heads < 1 || n < 1 || n_alloc < n) return GEAR_ERR_ARG;
+  if (n_alloc > 0x7fffffffLL) return GEAR_ERR_ARG;                  // token counts travel as 32-bit integers
   if (head_dim != kHeadDim || n_q_heads % n_kv_heads) return GEAR_ERR_SHAPE;
   if (((uintptr_t)K | (uintptr_t)V | (uintptr_t)q | (uintptr_t)out | (uintptr_t)scratch) & 15) return GEAR_ERR_ALIGN;
   if (scratch_bytes < gear_fp16_attn_scratch_bytes(batch, n_q_heads, head_dim)) return GEAR_ERR_CAPACITY;

@@ -141,6 +141,49 @@ __device__ __forceinline__ GroupResult process_group(int len, int k, XAt x_at, P
   return r;
 }
 
+// Pack the codes of one block (T tokens x 128 channels, xs[token * kXPitch + channel]) into the fragment order of
+// the integer tensor-core product (gear_layout.cuh); one 32-bit word per thread and step, stores coalesced.
+template <int BITS>
+__device__ __forceinline__ void pack_block_codes(const unsigned short* xs, int T, int side, unsigned int* dst, int tid,
+                                                 int nthreads) {
+  constexpr int F = 8 / BITS;
+  if (side == 0) {
+    constexpr int kWords = kSlab * kHeadDim * BITS / 32;            // words per slab
+    for (int li = tid; li < (T / kSlab) * kWords; li += nthreads) {
+      const int slab = li / kWords, wl = li % kWords;
+      const int w = wl & 3, lane = (wl >> 2) & 31, tau = wl >> 7;
+      unsigned int word = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < F; ++j) {
+          int tok, ch;
+          code_coord_k(BITS, lane, tau, w, i, j, tok, ch);
+          word |= (unsigned int)xs[(slab * kSlab + tok) * kXPitch + ch] << (8 * i + BITS * j);
+        }
+      dst[li] = word;
+    }
+  } else {
+    constexpr int kWords = 32 * kHeadDim * BITS / 32;               // words per 32-token chunk
+    const int nchunk = (T + 31) / 32;
+    for (int li = tid; li < nchunk * kWords; li += nthreads) {
+      const int chunk = li / kWords, wl = li % kWords;
+      const int w = wl & 3, lane = (wl >> 2) & 31, tau = wl >> 7;
+      unsigned int word = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < F; ++j) {
+          int tok, ch;
+          code_coord_v(BITS, lane, tau, w, i, j, tok, ch);
+          tok += chunk * 32;
+          if (tok < T) word |= (unsigned int)xs[tok * kXPitch + ch] << (8 * i + BITS * j);
+        }
+      dst[li] = word;
+    }
+  }
+}
+
 template <int BITS, int KMAX>
 __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -150,8 +193,8 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
   unsigned short* xs = reinterpret_cast<unsigned short*>(smem_raw);   // fp16 bits of the block; each entry is replaced by its code
   float* rs = reinterpret_cast<float*>(smem_raw + round_up(T * kXPitch * 2, 16));
   auto x_of = [&](int idx) { return __half2float(__ushort_as_half(xs[idx])); };
-  __shared__ unsigned int dmax_bits;
-  if (tid == 0) dmax_bits = 0u;
+  __shared__ unsigned int dmax_bits, smax_bits;
+  if (tid == 0) { dmax_bits = 0u; smax_bits = 0u; }
 
   const __half* X = (side == 0 ? p.K : p.V) + ((size_t)bhl * sd.n_c + (size_t)blk * T) * kHeadDim;
   for (int i = tid; i < T * 16; i += 128) {
@@ -164,7 +207,7 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
 
   unsigned char* rec = p.arena + sd.seg_base + (size_t)(p.bh0 + bhl) * sd.bh_stride + sd.bfac_bytes +
                        (size_t)blk * sd.rec_bytes;
-  float my_dmax = 0.f;
+  float my_dmax = 0.f, my_smax = 0.f;
   if (side == 0) {
     // keys: one group per channel over the T tokens of the block (per-channel grouping)
     const int j = tid;
@@ -177,6 +220,7 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
         [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
     reinterpret_cast<__half2*>(rec + sd.off_kscale)[j] = __halves2half2(g.scale, g.zero);
     my_dmax = g.dmax;
+    my_smax = __half2float(g.scale);
   } else {
     // values: one group per token over g_V consecutive channels (per-token grouping)
     const int k = p.cc.k_v, gv = p.cc.g_v, ngv = p.cc.ngv;
@@ -193,28 +237,20 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
           [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
       reinterpret_cast<__half2*>(rec + sd.off_vscale)[gi] = __halves2half2(g.scale, g.zero);
       my_dmax = fmaxf(my_dmax, g.dmax);
+      my_smax = fmaxf(my_smax, __half2float(g.scale));
     }
   }
   atomicMax(&dmax_bits, __float_as_uint(my_dmax));   // non-negative floats order like their bit patterns
+  atomicMax(&smax_bits, __float_as_uint(my_smax));
   __syncthreads();
-  if (tid == 0) reinterpret_cast<float*>(rec)[side] = __uint_as_float(dmax_bits);
+  if (tid == 0) {
+    reinterpret_cast<float*>(rec)[side] = __uint_as_float(dmax_bits);
+    reinterpret_cast<float*>(rec)[2 + side] = __uint_as_float(smax_bits);
+  }
 
   // pack the codes into mma-fragment order
-  const int nq = words_per_lane(BITS), hpw = regs_per_word(BITS);
-  const int words_per_slab = 32 * nq;
-  unsigned int* dst = reinterpret_cast<unsigned int*>(rec + (side == 0 ? sd.off_kcodes : sd.off_vcodes));
-  for (int li = tid; li < (T / kSlab) * words_per_slab; li += 128) {
-    const int slab = li / words_per_slab, wl = li % words_per_slab;
-    const int plane = wl >> 7, lane = (wl & 127) >> 2, q = plane * 4 + (wl & 3);
-    unsigned int word = 0;
-    for (int u = 0; u < hpw; ++u)
-      for (int e = 0; e < 2; ++e) {
-        int tok, ch;
-        if (side == 0) code_coord_k(BITS, lane, q, u, e, tok, ch); else code_coord_v(BITS, lane, q, u, e, tok, ch);
-        word |= (unsigned int)xs[(slab * kSlab + tok) * kXPitch + ch] << (16 * e + BITS * u);
-      }
-    dst[slab * (sd.slab_codes / 4) + wl] = word;
-  }
+  pack_block_codes<BITS>(xs, T, side, reinterpret_cast<unsigned int*>(rec + (side == 0 ? sd.off_kcodes : sd.off_vcodes)),
+                         tid, 128);
   // residual tile -> workspace (only needed when a low-rank part is fitted)
   if (p.R != nullptr) {
     float* R = p.R + (((size_t)bhl * 2 + side) * sd.n_c + (size_t)blk * T) * kHeadDim;
@@ -711,7 +747,7 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
   float* Uim = Um + kMaxRank * kFPitch;
   float* Wm = Uim + kMaxRank * kFPitch;
   float* wsum = Wm + kMaxRank * kFPitch;                                 // [4]
-  __shared__ unsigned int dmax_bits;
+  __shared__ unsigned int dmax_bits, smax_bits;
 
   const __half* Xt = (side == 0 ? p.K : p.V) + (size_t)bh * n_c * kHeadDim;
   unsigned char* seg_bh = p.arena + sd.seg_base + (size_t)bh * sd.bh_stride;
@@ -719,7 +755,7 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
 
   // ---- Filter, Quant, pack, residual: block by block (one key group per channel spans one block)
   for (int blk = 0; blk < sd.nblk; ++blk) {
-    if (tid == 0) dmax_bits = 0u;
+    if (tid == 0) { dmax_bits = 0u; smax_bits = 0u; }
     const __half* X = Xt + (size_t)blk * T * kHeadDim;
     for (int i = tid; i < T * 16; i += 128) {
       const int row = i >> 4, c = i & 15;
@@ -730,7 +766,7 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
     __syncthreads();
     unsigned char* rec = seg_bh + sd.bfac_bytes + (size_t)blk * sd.rec_bytes;
     float* rb = rs + (size_t)blk * T * kRPitch;
-    float my_dmax = 0.f;
+    float my_dmax = 0.f, my_smax = 0.f;
     if (side == 0) {
       const int j = tid, k = sd.k_k;
       __half* oval = reinterpret_cast<__half*>(rec + sd.off_koval) + j * 2 * k;
@@ -741,6 +777,7 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
           [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
       reinterpret_cast<__half2*>(rec + sd.off_kscale)[j] = __halves2half2(g.scale, g.zero);
       my_dmax = g.dmax;
+      my_smax = __half2float(g.scale);
     } else {
       const int k = p.cc.k_v, gv = p.cc.g_v, ngv = p.cc.ngv;
       for (int gi = tid; gi < T * ngv; gi += 128) {
@@ -756,29 +793,18 @@ __global__ void __launch_bounds__(128) compress_tile_kernel(TileArgs p) {
             [&](int slot, int idx, float v) { oval[slot] = __float2half_rn(v); oidx[slot] = (unsigned char)idx; });
         reinterpret_cast<__half2*>(rec + sd.off_vscale)[gi] = __halves2half2(g.scale, g.zero);
         my_dmax = fmaxf(my_dmax, g.dmax);
+        my_smax = fmaxf(my_smax, __half2float(g.scale));
       }
     }
     atomicMax(&dmax_bits, __float_as_uint(my_dmax));
+    atomicMax(&smax_bits, __float_as_uint(my_smax));
     __syncthreads();
-    if (tid == 0) reinterpret_cast<float*>(rec)[side] = __uint_as_float(dmax_bits);
-    const int nq = words_per_lane(BITS), hpw = regs_per_word(BITS);
-    const int words_per_slab = 32 * nq;
-    unsigned int* dst = reinterpret_cast<unsigned int*>(rec + (side == 0 ? sd.off_kcodes : sd.off_vcodes));
-    for (int li = tid; li < (T / kSlab) * words_per_slab; li += 128) {
-      const int slab = li / words_per_slab, wl = li % words_per_slab;
-      const int ln = (wl & 127) >> 2, q = (wl >> 7) * 4 + (wl & 3);      // inverse of word_index()
-      unsigned int word = 0;
-#pragma unroll
-      for (int u = 0; u < 16 / BITS; ++u)
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          int tok, ch;
-          if (side == 0) code_coord_k(BITS, ln, q, u, e, tok, ch); else code_coord_v(BITS, ln, q, u, e, tok, ch);
-          word |= (unsigned int)xs[(slab * kSlab + tok) * kXPitch + ch] << (16 * e + BITS * u);
-        }
-      (void)hpw;
-      dst[slab * (sd.slab_codes / 4) + wl] = word;
+    if (tid == 0) {
+      reinterpret_cast<float*>(rec)[side] = __uint_as_float(dmax_bits);
+      reinterpret_cast<float*>(rec)[2 + side] = __uint_as_float(smax_bits);
     }
+    pack_block_codes<BITS>(xs, T, side, reinterpret_cast<unsigned int*>(rec + (side == 0 ? sd.off_kcodes : sd.off_vcodes)),
+                           tid, 128);
     __syncthreads();
   }
   if (r == 0) return;

@@ -4,22 +4,29 @@
 // fp16 K / V are never materialised.
 //
 // Every warp is its own CTA and an independent stream processor.  The
-// (batch, kv head, head pass, block) space is cut into equal contiguous ranges,
-// one per warp.  A block travels as two items -- its key part and its value
-// part -- through a private shared-memory ring filled by bulk asynchronous
-// copies (cp.async.bulk + mbarrier), so that the copies of the next items run
-// while the warp works on the current one.
+// (batch, kv head, head pass, block) space is cut into contiguous ranges, one per
+// warp.  A block travels as two items -- its key part and its value part --
+// through a private shared-memory ring filled by bulk asynchronous copies
+// (cp.async.bulk + mbarrier), so that the copies of the next items run while the
+// warp works on the current one.
 //
-// Codes are unpacked in registers straight into the A operand of
-// mma.sync.m16n8k16 (tokens x channels for keys, channels x tokens for values).
-// The B operand holds the query heads of the GQA group, each split into an fp16
-// high and low part (two columns), so that every product is exact and every sum
-// is fp32.  Per-group scales are folded into the B operand (q * scale per channel
-// for keys, p * scale per token for values), zero-points into one constant per
-// block (keys) or an fp32 side sum (values).  Outlier corrections are scattered
-// with 32-bit fixed-point shared-memory adds, which keeps the result independent
-// of the order of the adds.  A warp writes one partial (m, l, o) per (batch,
-// head) it touched; the last warp to arrive for a (batch, head) merges them.
+// Codes meet the query on the integer tensor cores (mma.sync.m16n8k32, u8 x s8,
+// s32 accumulation).  A packed word becomes fragment registers of the A operand
+// with one AND per register: a b-bit field left where it sits in its byte is the
+// code times a power of two, which the B operand (keys) or the output row
+// (values) absorbs.  The B operand is a block-wide fixed-point image of
+// q * scale (keys, per channel) or p * scale (values, per token and group), cut
+// into signed base-256 digits ("limbs"), one column per limb: integer products
+// are exact, so the result does not depend on any order of summation.  Key
+// scores leave the integers once per 16-token slab; value sums stay in 32-bit
+// integers across blocks and are folded into an fp32 copy in shared memory only
+// when the running maximum, the fixed-point scale or the integer range demands
+// it.  Zero-points go into one constant per block (keys) or an fp32 side sum
+// (values); outlier corrections are scattered with 32-bit fixed-point
+// shared-memory adds; the low-rank terms and the fp16 rows of the streaming
+// buffer use the fp16 tensor-core path with an exact high / low split of the
+// query-side operand.  A warp writes one partial (m, l, o) per (batch, head) it
+// touched; the last warp to arrive for a (batch, head) merges them.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <math.h>
@@ -32,8 +39,11 @@ namespace gear {
 
 constexpr int kBufPitch = 272;                  // bytes per fp16 row of a buffer slab in shared memory
 constexpr int kBufItem = kSlab * kBufPitch;     // one slab of key rows or of value rows
-constexpr int kSpinLimit = 4000000;
-// 32-bit words per B-fragment row set.  A row set holds, for every column that carries a query head (hi, lo) and
+constexpr int kFragKRow = 40;                   // 32-bit words per (head, limb) row of the key B-operand staging area
+constexpr int kTokLimit = 16384;                // tokens a value accumulator takes before it is folded (int32 headroom)
+constexpr float kMagic = 12582912.0f;           // 1.5 * 2^23: x + kMagic carries rint(x) in its low mantissa bits, |x| < 2^22
+constexpr uint32_t kMagicBits = 0x4B400000u;
+// 32-bit words per fp16 B-fragment row set.  A row set holds, for every column that carries a query head (hi, lo) and
 // every lane column t, two registers; with one head only two of the eight columns exist and the lanes of the other
 // columns read those (their results are never used).  Padded against bank conflicts.
 __host__ __device__ constexpr int frag_row_words(int hp) { return hp == 1 ? 24 : 72; }
@@ -63,10 +73,10 @@ __device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after kSpinLimit polls and reports through `status`.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, int* status) {
+// Bounded wait: gives up after `limit` polls and reports through `status`.
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, int limit, int* status) {
 #pragma unroll 1
-  for (int i = 0; i < kSpinLimit; ++i)
+  for (int i = 0; i < limit; ++i)
     if (mbar_try(b, parity)) return true;
   atomicExch(status, -7 /* GEAR_ERR_TIMEOUT */);
   return false;
@@ -86,6 +96,13 @@ __device__ __forceinline__ void mma16816_z(float (&d)[4], const uint32_t (&a)[4]
       : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(z));
 }
+// integer product: A unsigned bytes (codes in place), B signed bytes (limbs), 32-bit sums
+__device__ __forceinline__ void imma16832(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* p) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -99,38 +116,14 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
 __device__ __forceinline__ uint32_t h2_as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
 
-// Codes become fragment registers with one AND each.  A masked field left in place, read as fp16, is the
-// subnormal  code * 2^(field_shift - 24)  (the tensor cores take subnormal inputs exactly); fields above the
-// 10-bit mantissa are reached through one shifted copy of the word.  The power of two is undone where it is free:
-// in the B operand for keys, in the output row for values.
+// mask of field j of every byte of a word of packed codes
 template <int BITS>
-__host__ __device__ constexpr int field_shift(int u) {     // bit position of field u once it sits in the mantissa
-  return BITS == 2 ? 2 * (u < 5 ? u : u - 5) : 4 * (u & 1);
+__host__ __device__ constexpr uint32_t field_mask(int j) {
+  return BITS == 2 ? (0x03030303u << (2 * j)) : (0x0F0F0F0Fu << (4 * j));
 }
-// One 32-bit word of codes -> its fragment registers r[0 .. 16/BITS).
-template <int BITS>
-__device__ __forceinline__ void unpack_word(uint32_t x, uint32_t* r) {
-  if (BITS == 2) {
-    const uint32_t y = x >> 10;
-    r[0] = x & 0x00030003u;
-    r[1] = x & 0x000C000Cu;
-    r[2] = x & 0x00300030u;
-    r[3] = x & 0x00C000C0u;
-    r[4] = x & 0x03000300u;
-    r[5] = y & 0x00030003u;
-    r[6] = y & 0x000C000Cu;
-    r[7] = y & 0x00300030u;
-  } else {
-    const uint32_t y = x >> 8;
-    r[0] = x & 0x000F000Fu;
-    r[1] = x & 0x00F000F0u;
-    r[2] = y & 0x000F000Fu;
-    r[3] = y & 0x00F000F0u;
-  }
-}
-// Keys: the B register that meets fields 2j (b0) / 2j+1 (b1) holds q * scale * 2^(kKeyExp - field_shift), so every
-// product carries 2^(kKeyExp - 24); the exponent keeps the scaled operand inside the fp16 range both ways.
-template <int BITS> constexpr int kKeyExp = BITS == 2 ? 4 : 2;
+// Signed base-256 digits of a 32-bit integer y, |y| < 2^31 - 2^23: byte l of the result, read as a signed byte, is
+// digit l, and sum digit_l * 256^l = y.
+__device__ __forceinline__ uint32_t balanced_digits(uint32_t y) { return (y + 0x80808080u) ^ 0x80808080u; }
 
 // fp32 pair -> half2 of the high parts and half2 of the rounding remainders
 __device__ __forceinline__ void split_hi_lo(float x0, float x1, uint32_t& hi, uint32_t& lo) {
@@ -145,8 +138,9 @@ __device__ __forceinline__ float warp_max(float x) {
   asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
   return r;
 }
+__device__ __forceinline__ uint32_t warp_max_u32(uint32_t x) { return __reduce_max_sync(0xffffffffu, x); }
 __device__ __forceinline__ int float_exponent(float x) { return (int)((__float_as_uint(x) >> 23) & 0xFFu) - 127; }
-// 2^e for |e| <= 60
+// 2^e for |e| <= 120
 __device__ __forceinline__ float pow2i(int e) { return __uint_as_float((uint32_t)(127 + e) << 23); }
 __device__ __forceinline__ int clamp60(int e) { return max(-60, min(60, e)); }
 
@@ -154,7 +148,7 @@ __device__ __forceinline__ int clamp60(int e) { return max(-60, min(60, e)); }
 bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int max_bfac, int max_T, size_t smem_budget,
                  DecodeArgs* a) {
   (void)bits;
-  const int HP = heads == 1 ? 1 : (heads <= 4 ? 4 : 8), NT = HP > 4 ? 2 : 1;
+  const int HP = decode_heads_per_pass(heads);
   const int frs = frag_row_words(HP);
   const int bregion = round_up(max_bfac / 2, 16);
   int part = max_kpart > max_vpart ? max_kpart : max_vpart;
@@ -162,25 +156,33 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
   if (stage < kBufItem) stage = kBufItem;
   stage = round_up(stage, 16);
   if (max_T < kSlab) max_T = kSlab;
-  const int nslab = max_T / kSlab;
-  const int frag_rows = 8 > nslab * (ngv + 1) ? 8 : nslab * (ngv + 1);
+  const int nslab = max_T / kSlab, nchunk = (max_T + 31) / 32;
+  // one region serves, in turn, the key B operand (limb rows), the value B operand (limb rows) with the fp16
+  // probability fragments behind it, and the fp16 query / probability fragments of buffer slabs
+  const int fragk = HP * 4 * kFragKRow * 4;
+  const int fv_stride = nchunk * 8 + 8;
+  const int fragv = round_up(ngv * HP * 4 * fv_stride * 4, 16);
+  const int fragp = nslab * frs * 4;
+  const int fragf = 9 * frs * 4;
+  int xr = fragk > fragv + fragp ? fragk : fragv + fragp;
+  if (fragf > xr) xr = fragf;
   WarpSmem w;
   int o = 0;
-  w.sdp = 0;
   w.sdc = o;     o += 128;
-  w.qf = o;      o += HP == 1 ? kHeadDim * 4 : 0;   // grouped queries rebuild it from qs: their warps are short of shared memory
   w.qs = o;      o += HP * kHeadDim * 2;
-  w.frag = o;    o += round_up(NT * frag_rows * frs * 4, 16);
-  w.corr_k = o;  o += HP * max_T * 4;
+  w.xr = o;      o += round_up(xr, 16);
   w.ps = o;      o += HP * max_T * 4;
+  w.corr_k = o;  o += HP * max_T * 4;
   w.corr_v = o;  o += HP * kHeadDim * 4;
   w.ocorr = o;   o += HP * kHeadDim * 4;
   w.wl = o;      o += kMaxRank * (HP == 1 ? 1 : 8) * 4 + 16;
-  w.misc = o;    o += 32 + kMaxStages * 8;   // exponents of max |q| per head, then the ring's mbarriers
+  w.misc = o;    o += 32 + (kMaxStages + 1) * 8 + 8;   // exponents of max |q| per head, the ring's mbarriers, one test barrier
   w.ring = round_up(o, 16);
+  w.fragv_stride = fv_stride;
+  w.fragp = fragv;
   // most resident warps (in steps of four: one per scheduler) whose ring still holds two stages; then as many
   // stages as fit
-  const int reg_limit = HP == 1 ? 16 : (HP == 4 ? 8 : 6);
+  const int reg_limit = HP == 1 ? 16 : 8;
   for (int warps = reg_limit; warps >= 1; warps -= (warps > 8 ? 4 : 1)) {
     const long long per = (long long)smem_budget / warps - 1024;     // the system reserves 1 KB per CTA
     long long ns = (per - w.ring) / stage;
@@ -189,6 +191,7 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
     w.total = w.ring + (int)ns * stage;
     a->aligned = 0;
     a->nstage = (int)ns; a->stage_bytes = stage; a->bregion = bregion; a->max_T = max_T; a->hpa = HP; a->ws = w;
+    a->spin_limit = kDecodeSpinLimit; a->test_dead_wait = 0;
     return true;
   }
   return false;
@@ -197,24 +200,18 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
 // ------------------------------------------------------------------ block shapes
 // The work on a block depends on its shape: tokens T, outliers per key group, padded rank, outliers per value
 // group.  The shapes of the usual configurations are compile-time constants (every offset inside the record becomes
-// an immediate and the slab loops unroll); any other segment runs through the same code with run-time values.
+// an immediate and the loops unroll); any other segment runs through the same code with run-time values.
 struct DynShape {                      // values read from the segment descriptor
-  static constexpr bool kDyn = true, kBuf = false;
-  static constexpr int T = 0, k2k = 0, r_pad = 0, k2v = 0, unroll = 1, tok_unroll = 1;
-  static constexpr int off_kscale = 0, off_koval = 0, off_koidx = 0, off_kcodes = 0, off_ak = 0, off_av = 0, off_vscale = 0,
-                       off_voval = 0, off_voidx = 0;
-};
-struct BufShape {                      // one slab of fp16 rows of the streaming buffer
-  static constexpr bool kDyn = false, kBuf = true;
-  static constexpr int T = kSlab, k2k = 0, r_pad = 0, k2v = 0, unroll = 1, tok_unroll = 1;
+  static constexpr bool kDyn = true;
+  static constexpr int T = 0, k2k = 0, r_pad = 0, k2v = 0, unroll = 1;
   static constexpr int off_kscale = 0, off_koval = 0, off_koidx = 0, off_kcodes = 0, off_ak = 0, off_av = 0, off_vscale = 0,
                        off_voval = 0, off_voidx = 0;
 };
 template <int BITS, int NGV, int T_, int KK, int RP, int KV>
 struct StaticShape {                   // mirrors layout_segment(); checked against it on the host (static_shape_id)
-  static constexpr bool kDyn = false, kBuf = false;
-  static constexpr int T = T_, k2k = 2 * KK, r_pad = RP, k2v = 2 * KV, unroll = 2, tok_unroll = T_ / 32;
-  static constexpr int nslab = T_ / kSlab, slab_codes = kSlab * kHeadDim * BITS / 8;
+  static constexpr bool kDyn = false;
+  static constexpr int T = T_, k2k = 2 * KK, r_pad = RP, k2v = 2 * KV, unroll = 2;
+  static constexpr int nslab = T_ / kSlab, slab_codes = kSlab * kHeadDim * BITS / 8, nchunk = (T_ + 31) / 32;
   static constexpr int off_kscale = kRecHeader;
   static constexpr int off_koval = off_kscale + kHeadDim * 4;
   static constexpr int off_koidx = off_koval + kHeadDim * 2 * KK * 2;
@@ -222,7 +219,7 @@ struct StaticShape {                   // mirrors layout_segment(); checked agai
   static constexpr int off_ak = off_kcodes + nslab * slab_codes;
   static constexpr int off_vpart = off_ak + (nslab * kSlab * RP * 2 + 15) / 16 * 16;
   // value part, relative to its start
-  static constexpr int off_av = nslab * slab_codes;
+  static constexpr int off_av = nchunk * 2 * slab_codes;
   static constexpr int off_vscale = off_av + (nslab * kSlab * RP * 2 + 15) / 16 * 16;
   static constexpr int off_voval = off_vscale + T_ * NGV * 4;
   static constexpr int off_voidx = off_voval + (T_ * NGV * 2 * KV * 2 + 15) / 16 * 16;
@@ -250,17 +247,19 @@ int static_shape_id(const SegDesc& s, const CacheConst& c) {
 }
 
 // ------------------------------------------------------------------ the kernel
-// HEADS = query heads handled per pass: 1 (multi-head attention), 4 or 8 (grouped queries; a pass may hold fewer).
+// HEADS = query heads handled per pass: 1 (multi-head attention) or 4 (grouped queries; a pass may hold fewer).
 template <int BITS, int HEADS, int NGV>
-__global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) gear_decode_kernel(const __grid_constant__ DecodeArgs a) {
+__global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(const __grid_constant__ DecodeArgs a) {
   constexpr int HP = HEADS;
-  constexpr int NT = HEADS > 4 ? 2 : 1;           // 8-column tiles of the B operand
+  constexpr int NT = HP == 1 ? 1 : 2;             // 8-column tiles of the integer B operands: four limb columns per head
+  constexpr int F = 8 / BITS;                     // code fields per byte
+  constexpr int kTop = BITS * (F - 1);            // the shift of the highest field
   constexpr int GV = kHeadDim / NGV;              // channels per value group
-  constexpr int SLABW = kSlab * kHeadDim * BITS / 8 / 16;   // uint4 per slab of codes
+  constexpr int KT = 4 / F;                       // key tuples per slab
+  constexpr int VT = 8 / F;                       // value tuples per 32-token chunk
   constexpr int kFragStride = frag_row_words(HP);
-  constexpr int CMASK = HP == 1 ? 1 : 7;          // fragment columns that exist, as a mask on the lane's column
+  constexpr int CMASK = HP == 1 ? 1 : 7;          // fp16 fragment columns that exist, as a mask on the lane's column
   constexpr int WLS = HP == 1 ? 1 : 8;            // row stride of the small factor exchange buffer wl[16][heads]
-  constexpr int HMASK = HP == 1 ? 0 : 7;          // heads that exist in wl, as a mask on the lane's head
   extern __shared__ __align__(128) unsigned char smem[];
 
   const int lane = threadIdx.x, gid = lane >> 2, t = lane & 3;
@@ -268,31 +267,32 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
   const int passes = (G + HP - 1) / HP;
   const int maxT = a.max_T;
   const int NS = a.nstage;
+  const int RS = a.ws.fragv_stride;
   unsigned char* ring = smem + a.ws.ring;
   SegDesc* sdc = reinterpret_cast<SegDesc*>(smem + a.ws.sdc);
-  float* qf = reinterpret_cast<float*>(smem + a.ws.qf);          // [128] q * scale * log2(e) (one query head per pass only)
   __half* qs = reinterpret_cast<__half*>(smem + a.ws.qs);        // [HP][128] q
-  uint32_t* frag = reinterpret_cast<uint32_t*>(smem + a.ws.frag);
+  uint32_t* xr = reinterpret_cast<uint32_t*>(smem + a.ws.xr);    // B-operand staging, see decode_plan
+  uint32_t* fragPc = reinterpret_cast<uint32_t*>(smem + a.ws.xr + a.ws.fragp);   // fp16 probability fragments (compressed blocks)
+  uint32_t* fragPb = xr + 8 * kFragStride;                       // the same for buffer slabs
   int* corr_k = reinterpret_cast<int*>(smem + a.ws.corr_k);      // [HP][maxT]
   float* ps = reinterpret_cast<float*>(smem + a.ws.ps);          // [HP][maxT] scores, then probabilities
   int* corr_v = reinterpret_cast<int*>(smem + a.ws.corr_v);      // [HP][128]
-  float* ocorr = reinterpret_cast<float*>(smem + a.ws.ocorr);    // [HP][128]
+  float* ocorr = reinterpret_cast<float*>(smem + a.ws.ocorr);    // [HP][128] fp32 copy of the output accumulators
   float* wl = reinterpret_cast<float*>(smem + a.ws.wl);          // [16][heads]
   int* qexp_s = reinterpret_cast<int*>(smem + a.ws.misc);        // [HP]
-  uint64_t* bar = reinterpret_cast<uint64_t*>(smem + a.ws.misc + 32);   // [kMaxStages]; no static shared memory, so
-                                                                         // that sixteen warps fit one SM
+  uint64_t* bar = reinterpret_cast<uint64_t*>(smem + a.ws.misc + 32);   // [kMaxStages] ring, [kMaxStages] test barrier
 
-  // this lane's four channels in the key set-up sit in B register (lane / 2) % 2 of channel chunk lane / 4, which
-  // meets field 2 * (chunk % 4) + register of the 2-bit words (any field of that parity of the 4-bit words)
-  const float kfac = pow2i(kKeyExp<BITS> - (BITS == 2 ? 2 * ((2 * ((lane >> 2) & 3) + ((lane >> 1) & 1)) % 5)
-                                                      : 4 * ((lane >> 1) & 1)));
-  constexpr float kKeyBack = (float)(1 << (24 - kKeyExp<BITS>));       // undoes 2^(kKeyExp - 24)
-  const bool o_plain = a.n_blocks_c == 0;       // no compressed block: the output rows carry no factor
+  // lane roles in the integer products: B / D column n of tile nt is limb n % 4 of head 2 nt + n / 4.  As owner of
+  // B column gid the lane fetches limb gid % 4 of head hcol(nt); as owner of D columns 2t, 2t + 1 it holds the limb
+  // pair t % 2 of head hacc(nt).
+  const int limb_b = gid & 3;
+  const bool pair_hi = (t & 1) != 0;
+  const bool writer = HP == 1 ? (t == 0) : !pair_hi;    // lanes that hold the low limb pair of a real head finish the sums
 
   if (lane == 0)
-    for (int s = 0; s < NS; ++s) mbar_init(&bar[s], 1);
+    for (int s = 0; s <= kMaxStages; ++s) mbar_init(&bar[s], 1);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  for (int i = lane; i < (a.ws.corr_k - a.ws.frag) / 4; i += 32) frag[i] = 0u;
+  for (int i = lane; i < (a.ws.ps - a.ws.xr) / 4; i += 32) xr[i] = 0u;
   for (int i = lane; i < HP * maxT; i += 32) corr_k[i] = 0;
   for (int i = lane; i < HP * kHeadDim; i += 32) corr_v[i] = 0;
   __syncwarp();
@@ -313,9 +313,9 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
     blk_lo = part * base + min(part, rem);                          // the first `rem` ranges are one block longer
     n_left = base + (part < rem ? 1 : 0);
   } else {
-    const long long F = (long long)a.cc.BH * passes * NB;
+    const long long Fl = (long long)a.cc.BH * passes * NB;
     const long long NW = gridDim.x, gw = blockIdx.x;
-    const long long f0 = gw * F / NW, f1 = (gw + 1) * F / NW;
+    const long long f0 = gw * Fl / NW, f1 = (gw + 1) * Fl / NW;
     if (f0 >= f1) return;                       // the host launches no more warps than blocks
     n_left = (int)(f1 - f0);
     u = (int)(f0 / NB);
@@ -388,10 +388,12 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
 
   int c_stage = 0, c_par = 0, c_seg_lo = 0, c_seg_hi = 0, c_shape = 0;
   bool alive = true;
+  // test only: a wait that nothing ends, so that the give-up path runs; the copies in flight are drained below
+  if (a.test_dead_wait && !mbar_wait(&bar[kMaxStages], 0u, 64, a.status)) alive = false;
   // wait for the next item (items are consumed in order); returns its stage
   auto acquire = [&]() -> unsigned char* {
     unsigned char* st = ring + c_stage * a.stage_bytes;
-    if (!mbar_wait(&bar[c_stage], (uint32_t)c_par, a.status)) alive = false;
+    if (!mbar_wait(&bar[c_stage], (uint32_t)c_par, a.spin_limit, a.status)) alive = false;
     if (++c_stage == NS) { c_stage = 0; c_par ^= 1; }
     --n_inflight;
     return st;
@@ -401,47 +403,21 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
     issue();
   };
 
-  // Output rows fed by the codes carry the factor of the field their codes came from: row half hf (channel gid + 8 hf)
-  // of channel tile mt holds  value * 2^(row_shift - 24).  A product of full-range operands (buffer rows, B_V U) joins
-  // such a row through a zero-based product and one multiply-add per element.
-  auto row_shift = [](int mt, int hf) { return field_shift<BITS>(2 * (mt % (8 / BITS)) + hf); };
-  auto add_scaled = [&](float (&o)[4], int mt, const uint32_t (&av)[4], uint32_t b0, uint32_t b1) {
-    float d[4];
-    mma16816_z(d, av, b0, b1);
-    const float f0 = 1.f / (float)(1 << (24 - row_shift(mt, 0))), f1 = 1.f / (float)(1 << (24 - row_shift(mt, 1)));
-    o[0] = fmaf(d[0], f0, o[0]); o[1] = fmaf(d[1], f0, o[1]);
-    o[2] = fmaf(d[2], f1, o[2]); o[3] = fmaf(d[3], f1, o[3]);
-  };
-
   // ---- loop over the units this warp touches
   while (n_left > 0 && alive) {
     const int blk_hi = min(NB, blk_lo + n_left);
+    const int c_hi = min(blk_hi, a.n_blocks_c);          // end of the compressed blocks of this range
     const int bh = u / passes, pass = u - bh * passes;
     const int HPu = HEADS == 1 ? 1 : min(HP, G - pass * HP);
     const int hq0 = bh * G + pass * HP;                 // first query head of this pass
 
     // unit state
-    float O[8][NT][4], U[NT][4], m_run[HP], l_run[HP], cm[HP][NGV];
-    uint32_t bw[NT][2];                                  // low-rank key term: B operand (q B_K) of the current segment
+    float m_run[HP], l_run[HP];
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      bw[nt][0] = bw[nt][1] = 0u;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) U[nt][i] = 0.f;
-#pragma unroll
-      for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) O[mt][nt][i] = 0.f;
-    }
-#pragma unroll
-    for (int h = 0; h < HP; ++h) {
-      m_run[h] = -INFINITY; l_run[h] = 0.f;
-#pragma unroll
-      for (int g = 0; g < NGV; ++g) cm[h][g] = 0.f;
-    }
-    bool u_pending = false;
+    for (int h = 0; h < HP; ++h) { m_run[h] = -INFINITY; l_run[h] = 0.f; }
 
-    // query rows of this pass -> shared (fp16 as given, and fp32 times scale * log2 e); exponent of max |q|
+    // query rows of this pass -> shared (fp16 as given); exponent of max |q * scale|; the fp32 output copy starts at 0
+    float qreg[4] = {0.f, 0.f, 0.f, 0.f};               // one head per pass: this lane's four channels of q * scale * log2 e
     __syncwarp();
 #pragma unroll
     for (int h = 0; h < HP; ++h) {
@@ -451,311 +427,344 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
         const __half2 q01 = u32_as_h2(v.x), q23 = u32_as_h2(v.y);
         const float4 qv = make_float4(__low2float(q01) * a.scale_log2, __high2float(q01) * a.scale_log2,
                                       __low2float(q23) * a.scale_log2, __high2float(q23) * a.scale_log2);
-        if (HP == 1) *reinterpret_cast<float4*>(qf + h * kHeadDim + lane * 4) = qv;
-        *reinterpret_cast<float4*>(ocorr + h * kHeadDim + lane * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (HP == 1) { qreg[0] = qv.x; qreg[1] = qv.y; qreg[2] = qv.z; qreg[3] = qv.w; }
         float mx = fmaxf(fmaxf(fabsf(qv.x), fabsf(qv.y)), fmaxf(fabsf(qv.z), fabsf(qv.w)));
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         if (lane == 0) qexp_s[h] = float_exponent(mx);
       }
+      *reinterpret_cast<float4*>(ocorr + h * kHeadDim + lane * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     __syncwarp();
 
-#pragma unroll 1
-    for (int blk = blk_lo; blk < blk_hi; ++blk) {
-      const bool buf_blk = blk >= a.n_blocks_c;
-      if (!buf_blk && (blk >= c_seg_hi || blk < c_seg_lo)) {
-        load_desc(sdc, blk);
-        c_seg_lo = sdc->blk_start;
-        c_seg_hi = c_seg_lo + sdc->nblk;
-        c_shape = sdc->shape_id;
-      }
-      auto body = [&](auto shape_tag) {
-      using S = decltype(shape_tag);
-      constexpr bool is_buf = S::kBuf;
-      constexpr int TU = HP == 1 ? S::tok_unroll : 1;     // unrolling of the per-token loops (latency, one head only)
-      // ---------------- block geometry
-      const int T = S::kDyn ? sdc->T : S::T;
-      const int r_pad = S::kDyn ? sdc->r_pad : S::r_pad;
-      const int k2k = S::kDyn ? 2 * sdc->k_k : S::k2k;
-      const int k2v = S::kDyn ? 2 * a.cc.k_v : S::k2v;
-      const int off_kscale = S::kDyn ? sdc->off_kscale : S::off_kscale;
-      const int off_koval = S::kDyn ? sdc->off_koval : S::off_koval;
-      const int off_koidx = S::kDyn ? sdc->off_koidx : S::off_koidx;
-      const int off_kcodes = S::kDyn ? sdc->off_kcodes : S::off_kcodes;
-      const int off_ak = S::kDyn ? sdc->off_ak : S::off_ak;
-      const int o_av = S::kDyn ? sdc->off_av - sdc->off_vpart : S::off_av;
-      const int o_vsz = S::kDyn ? sdc->off_vscale - sdc->off_vpart : S::off_vscale;
-      const int o_voval = S::kDyn ? sdc->off_voval - sdc->off_vpart : S::off_voval;
-      const int o_voidx = S::kDyn ? sdc->off_voidx - sdc->off_vpart : S::off_voidx;
-      int valid_tokens = T;
-      bool with_bk = false, with_bv = false;
-      if (!is_buf) {
-        with_bk = r_pad > 0 && (blk == c_seg_lo || blk == blk_lo);
-        with_bv = r_pad > 0 && (blk == c_seg_hi - 1 || blk == blk_hi - 1);
-      } else {
-        valid_tokens = min(kSlab, a.buf_len - (blk - a.n_blocks_c) * kSlab);
-      }
-      const int nslab = T / kSlab;
-
-      // ================================================================ key item
-      unsigned char* stK = acquire();
-      if (!alive) return;
-      const unsigned char* kp = stK + a.bregion;
-      float dmax_v = 0.f;
-      int sexp_k[HP];                                 // per head: exponent of the sparse key term's fixed-point scale
-      float c_zero[HP];                               // per head: sum over channels of q * zero-point
+    // scale everything accumulated in fp32 for head h by alpha[h] (the running maximum grew)
+    auto scale_ocorr = [&](const float (&alpha)[HP]) {
 #pragma unroll
-      for (int h = 0; h < HP; ++h) { sexp_k[h] = 0; c_zero[h] = 0.f; }
-
-      if (with_bk) {
-        // w = q B_K through the tensor cores, kept as the B operand of the low-rank key term
-        const __half* bk = reinterpret_cast<const __half*>(stK);     // [r_pad][128]
-        float wacc[NT][4];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-          for (int i = 0; i < 4; ++i) wacc[nt][i] = 0.f;
-#pragma unroll 2
-        for (int kc = 0; kc < 8; ++kc) {
-          uint32_t af[4] = {0u, 0u, 0u, 0u};
-          if (gid < r_pad) {
-            af[0] = *reinterpret_cast<const uint32_t*>(bk + gid * kHeadDim + 16 * kc + 2 * t);
-            af[2] = *reinterpret_cast<const uint32_t*>(bk + gid * kHeadDim + 16 * kc + 2 * t + 8);
-          }
-          if (gid + 8 < r_pad) {
-            af[1] = *reinterpret_cast<const uint32_t*>(bk + (gid + 8) * kHeadDim + 16 * kc + 2 * t);
-            af[3] = *reinterpret_cast<const uint32_t*>(bk + (gid + 8) * kHeadDim + 16 * kc + 2 * t + 8);
-          }
-#pragma unroll
-          for (int nt = 0; nt < NT; ++nt) {
-            uint32_t b0 = 0u, b1 = 0u;
-            const int h = (gid >> 1) + 4 * nt;
-            if ((gid & 1) == 0 && h < HPu) {
-              const __half* qrow = qs + h * kHeadDim + 16 * kc + 2 * t;
-              b0 = *reinterpret_cast<const uint32_t*>(qrow);
-              b1 = *reinterpret_cast<const uint32_t*>(qrow + 8);
-            }
-            mma16816(wacc[nt], af, b0, b1);
-          }
+      for (int h = 0; h < HP; ++h) {
+        if (h < HPu) {
+          float4* oc = reinterpret_cast<float4*>(ocorr + h * kHeadDim + lane * 4);
+          float4 v = *oc;
+          v.x *= alpha[h]; v.y *= alpha[h]; v.z *= alpha[h]; v.w *= alpha[h];
+          *oc = v;
         }
-        __syncwarp();
+      }
+    };
+
+    // ==================================================================== compressed blocks
+    if (blk_lo < c_hi) {
+      int O[8][NT][4];                                   // value sums: tile (16 channels) x column tile, 32-bit integers
+      float U[4], cm[HP][NGV];
+      uint32_t bw[NT][2];                                // low-rank key term: B operand (q B_K) of the current segment
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {       // D[rho][col 2t] = w[rho][head t + 4nt]
-          if (t + 4 * nt < HP) {
-            wl[gid * WLS + t + 4 * nt] = wacc[nt][0] * a.scale_log2;
-            wl[(gid + 8) * WLS + t + 4 * nt] = wacc[nt][2] * a.scale_log2;
-          }
-        }
+      for (int nt = 0; nt < NT; ++nt) {
+        bw[nt][0] = bw[nt][1] = 0u;
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) O[mt][nt][i] = 0;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) U[i] = 0.f;
+#pragma unroll
+      for (int h = 0; h < HP; ++h)
+#pragma unroll
+        for (int g = 0; g < NGV; ++g) cm[h][g] = 0.f;
+      bool u_pending = false;
+      int eV_cur = 1000;                                 // exponent of the value fixed-point scale the integer sums carry
+      int tok_acc = 0;                                   // tokens in the integer sums since they were last folded
+
+      // integer sums -> fp32 copy in shared memory, times alpha[h]; the integers start again from zero
+      auto fold_O = [&](const float (&alpha)[HP]) {
+        const float fs = pow2i(-eV_cur);
         __syncwarp();
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          const int h = (gid >> 1) + 4 * nt;
-          uint32_t hi0, lo0, hi1, lo1;
-          split_hi_lo(wl[(2 * t) * WLS + (h & HMASK)], wl[(2 * t + 1) * WLS + (h & HMASK)], hi0, lo0);
-          split_hi_lo(wl[(2 * t + 8) * WLS + (h & HMASK)], wl[(2 * t + 9) * WLS + (h & HMASK)], hi1, lo1);
-          bw[nt][0] = (gid & 1) ? lo0 : hi0;
-          bw[nt][1] = (gid & 1) ? lo1 : hi1;
+          const int hd = HP == 1 ? 0 : 2 * nt + (t >> 1);
+          float al = alpha[HP == 1 ? 0 : 2 * nt];
+          if (HP > 1 && (t >> 1)) al = alpha[HP == 1 ? 0 : 2 * nt + 1];
+          const float w1 = pair_hi ? 0.f : 256.f;            // the high pair's second column is no limb: dropped
+          const float w0 = pair_hi ? 65536.f * fs : fs;
+#pragma unroll
+          for (int mt = 0; mt < 8; ++mt) {
+            const float rs = w0 * (1.0f / (float)(1 << (BITS * (mt % F))));
+            float v0 = fmaf((float)O[mt][nt][1], w1, (float)O[mt][nt][0]) * rs;
+            float v1 = fmaf((float)O[mt][nt][3], w1, (float)O[mt][nt][2]) * rs;
+            v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
+            v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+            if (writer && hd < HPu) {
+              float* oc = ocorr + hd * kHeadDim + 16 * mt + gid;
+              oc[0] = (oc[0] + v0) * al;
+              oc[8] = (oc[8] + v1) * al;
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) O[mt][nt][i] = 0;
+          }
         }
         __syncwarp();
-      }
+      };
 
-      // ---------------- B operand of the key scores: q * scale per channel, split hi / lo;
-      //                  c_h = sum q * zero;  sparse key term scattered to its token
-      {
-        float sc4[4] = {1.f, 1.f, 1.f, 1.f}, zr4[4] = {0.f, 0.f, 0.f, 0.f};
-        int ed = 0;
-        if (!is_buf) {
-          const float dmax_k = reinterpret_cast<const float*>(kp)[0];
-          dmax_v = reinterpret_cast<const float*>(kp)[1];
-          ed = float_exponent(dmax_k);
-          const uint4 kz = reinterpret_cast<const uint4*>(kp + off_kscale)[lane];
-          const uint32_t w4[4] = {kz.x, kz.y, kz.z, kz.w};
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            sc4[j] = __low2float(u32_as_h2(w4[j])) * kfac;
-            zr4[j] = __high2float(u32_as_h2(w4[j]));
-          }
-        }
-        float qS[HP][4];
-        const int kc = lane >> 2, reg = (lane >> 1) & 1, tA = 2 * (lane & 1);
-#pragma unroll
-        for (int h = 0; h < HP; ++h) {
-          if (h < HPu) {
-            float4 qv;
-            if (HP == 1) {
-              qv = *reinterpret_cast<const float4*>(qf + h * kHeadDim + lane * 4);
-            } else {
-              const uint2 qh = *reinterpret_cast<const uint2*>(qs + h * kHeadDim + lane * 4);
-              const __half2 q01 = u32_as_h2(qh.x), q23 = u32_as_h2(qh.y);
-              qv = make_float4(__low2float(q01) * a.scale_log2, __high2float(q01) * a.scale_log2,
-                               __low2float(q23) * a.scale_log2, __high2float(q23) * a.scale_log2);
-            }
-            uint32_t hiA, loA, hiB, loB;
-            split_hi_lo(qv.x * sc4[0], qv.y * sc4[1], hiA, loA);
-            split_hi_lo(qv.z * sc4[2], qv.w * sc4[3], hiB, loB);
-            uint32_t* base = frag + ((h >> 2) * 8 + kc) * kFragStride + reg;
-            const int cl = 2 * (h & 3);
-            base[(4 * cl + tA) * 2] = hiA;
-            base[(4 * (cl + 1) + tA) * 2] = loA;
-            base[(4 * cl + tA + 1) * 2] = hiB;
-            base[(4 * (cl + 1) + tA + 1) * 2] = loB;
-            if (!is_buf) {
-              float c = fmaf(qv.x, zr4[0], fmaf(qv.y, zr4[1], fmaf(qv.z, zr4[2], qv.w * zr4[3])));   // this lane's part
-              if (HP != 4) {
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-              }
-              const int sexp = clamp60(21 - qexp_s[h] - ed);
-              const float S = pow2i(sexp);
-              qS[h][0] = qv.x * S; qS[h][1] = qv.y * S; qS[h][2] = qv.z * S; qS[h][3] = qv.w * S;
-              c_zero[h] = c; sexp_k[h] = sexp;
-            }
-          }
-        }
-        if (!is_buf && HP == 4) {            // c_zero of four heads: sums over the warp
-          {
-            // four sums at once: two exchange steps halve what a lane carries, a butterfly finishes the one value left
-            // (head 2 * bit4 + bit3 of the lane), four broadcasts hand the sums back: 10 shuffles instead of 20
-            float s0 = c_zero[0], s1 = c_zero[1];
-            {
-              const bool up = (lane & 16) != 0;
-              const float send0 = up ? c_zero[0] : c_zero[2], keep0 = up ? c_zero[2] : c_zero[0];
-              const float send1 = up ? c_zero[1] : c_zero[3], keep1 = up ? c_zero[3] : c_zero[1];
-              s0 = keep0 + __shfl_xor_sync(0xffffffffu, send0, 16);
-              s1 = keep1 + __shfl_xor_sync(0xffffffffu, send1, 16);
-            }
-            {
-              const bool up = (lane & 8) != 0;
-              const float send = up ? s0 : s1, keep = up ? s1 : s0;
-              s0 = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-            }
-#pragma unroll
-            for (int o = 4; o > 0; o >>= 1) s0 += __shfl_xor_sync(0xffffffffu, s0, o);
-#pragma unroll
-            for (int h = 0; h < HP; ++h) c_zero[h] = __shfl_sync(0xffffffffu, s0, 8 * h);
-          }
-        }
-        if (!is_buf && k2k > 0) {
-          auto k_entry = [&](int j, float val, int idx) {
-            const float d = val - zr4[j];
-#pragma unroll
-            for (int h = 0; h < HP; ++h)
-              if (h < HPu) atomicAdd(&corr_k[h * maxT + idx], __float2int_rn(qS[h][j] * d));
-          };
-          if (k2k == 2) {
-            const uint4 ov = reinterpret_cast<const uint4*>(kp + off_koval)[lane];
-            const uint2 oi = reinterpret_cast<const uint2*>(kp + off_koidx)[lane];
-            const uint32_t o4[4] = {ov.x, ov.y, ov.z, ov.w};
-            const uint32_t i2[2] = {oi.x, oi.y};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              k_entry(j, __low2float(u32_as_h2(o4[j])), (i2[j >> 1] >> (16 * (j & 1))) & 0xFFu);
-              k_entry(j, __high2float(u32_as_h2(o4[j])), (i2[j >> 1] >> (16 * (j & 1) + 8)) & 0xFFu);
-            }
-          } else if (k2k == 4) {
-            // this lane's 4 channels x 4 entries: 32 bytes of values, 16 bytes of token indices
-            const uint4 ova = reinterpret_cast<const uint4*>(kp + off_koval)[2 * lane];
-            const uint4 ovb = reinterpret_cast<const uint4*>(kp + off_koval)[2 * lane + 1];
-            const uint4 oi = reinterpret_cast<const uint4*>(kp + off_koidx)[lane];
-            const uint32_t o8[8] = {ova.x, ova.y, ova.z, ova.w, ovb.x, ovb.y, ovb.z, ovb.w};
-            const uint32_t i4[4] = {oi.x, oi.y, oi.z, oi.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              k_entry(j, __low2float(u32_as_h2(o8[2 * j])), i4[j] & 0xFFu);
-              k_entry(j, __high2float(u32_as_h2(o8[2 * j])), (i4[j] >> 8) & 0xFFu);
-              k_entry(j, __low2float(u32_as_h2(o8[2 * j + 1])), (i4[j] >> 16) & 0xFFu);
-              k_entry(j, __high2float(u32_as_h2(o8[2 * j + 1])), i4[j] >> 24);
-            }
-          } else {
-            const __half* ov = reinterpret_cast<const __half*>(kp + off_koval) + lane * 4 * k2k;
-            const unsigned char* oi = kp + off_koidx + lane * 4 * k2k;
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
 #pragma unroll 1
-              for (int e = 0; e < k2k; ++e) k_entry(j, __half2float(ov[j * k2k + e]), oi[j * k2k + e]);
-          }
+      for (int blk = blk_lo; blk < c_hi; ++blk) {
+        if (blk >= c_seg_hi || blk < c_seg_lo) {
+          load_desc(sdc, blk);
+          c_seg_lo = sdc->blk_start;
+          c_seg_hi = c_seg_lo + sdc->nblk;
+          c_shape = sdc->shape_id;
         }
-      }
-      __syncwarp();
-      uint32_t bq[NT][8][2];
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-        for (int kc = 0; kc < 8; ++kc) {
-          const uint2 v = *reinterpret_cast<const uint2*>(frag + (nt * 8 + kc) * kFragStride + ((gid & CMASK) * 4 + t) * 2);
-          bq[nt][kc][0] = v.x; bq[nt][kc][1] = v.y;
-        }
+        auto body = [&](auto shape_tag) {
+          using S = decltype(shape_tag);
+          // ---------------- block geometry
+          const int T = S::kDyn ? sdc->T : S::T;
+          const int r_pad = S::kDyn ? sdc->r_pad : S::r_pad;
+          const int k2k = S::kDyn ? 2 * sdc->k_k : S::k2k;
+          const int k2v = S::kDyn ? 2 * a.cc.k_v : S::k2v;
+          const int off_kscale = S::kDyn ? sdc->off_kscale : S::off_kscale;
+          const int off_koval = S::kDyn ? sdc->off_koval : S::off_koval;
+          const int off_koidx = S::kDyn ? sdc->off_koidx : S::off_koidx;
+          const int off_kcodes = S::kDyn ? sdc->off_kcodes : S::off_kcodes;
+          const int off_ak = S::kDyn ? sdc->off_ak : S::off_ak;
+          const int o_av = S::kDyn ? sdc->off_av - sdc->off_vpart : S::off_av;
+          const int o_vsz = S::kDyn ? sdc->off_vscale - sdc->off_vpart : S::off_vscale;
+          const int o_voval = S::kDyn ? sdc->off_voval - sdc->off_vpart : S::off_voval;
+          const int o_voidx = S::kDyn ? sdc->off_voidx - sdc->off_vpart : S::off_voidx;
+          const bool with_bk = r_pad > 0 && (blk == c_seg_lo || blk == blk_lo);
+          const bool with_bv = r_pad > 0 && (blk == c_seg_hi - 1 || blk == blk_hi - 1);
+          const int nslab = T / kSlab;
+          const int nchunk = (T + 31) / 32;
 
-      // ---------------- key scores, slab by slab; scores go to shared memory
-      {
-        int psoff[NT];                                  // this lane's first score slot (head t + 4 nt, token gid)
+          // ================================================================ key item
+          unsigned char* stK = acquire();
+          if (!alive) return;
+          const unsigned char* kp = stK + a.bregion;
+          const float dmax_k = reinterpret_cast<const float*>(kp)[0];
+          const float dmax_v = reinterpret_cast<const float*>(kp)[1];
+          const float smax_v = reinterpret_cast<const float*>(kp)[3];
+          int sexp_k[HP];                                 // per head: exponent of the sparse key term's fixed-point scale
+          float c_zero[HP];                               // per head: sum over channels of q * zero-point
+          float kscl[NT];                                 // per column tile: what turns this lane's integer sums into scores
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) psoff[nt] = (t + 4 * nt) * maxT + gid;
-        const bool pa0 = 2 * t < r_pad, pa1 = 2 * t + 8 < r_pad;
-        auto k_slabs = [&](auto buf_tag) {
-          constexpr bool kBuf = decltype(buf_tag)::value;
-          const uint4* cwp = reinterpret_cast<const uint4*>(kp + off_kcodes) + lane;
-          const __half* akp = reinterpret_cast<const __half*>(kp + off_ak) + gid * r_pad + 2 * t;
-          const int ak8 = 8 * r_pad, ak_step = kSlab * r_pad;
-          int tok0 = 0;
-#pragma unroll (S::unroll)
-          for (int slab = 0; slab < nslab; ++slab) {
-            float acc[2][NT][4];
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-              for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) acc[hf][nt][i] = 0.f;
-            uint4 w0 = make_uint4(0u, 0u, 0u, 0u), w1 = w0;
-            if (!kBuf) {
-              w0 = cwp[0];
-              if (BITS == 4) w1 = cwp[32];
-              cwp += SLABW;
+          for (int h = 0; h < HP; ++h) { sexp_k[h] = 0; c_zero[h] = 0.f; }
+
+          if (with_bk) {
+            // w = q B_K through the fp16 tensor cores, kept as the B operand of the low-rank key term
+            const __half* bk = reinterpret_cast<const __half*>(stK);     // [r_pad][128]
+            float wacc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 2
+            for (int kc = 0; kc < 8; ++kc) {
+              uint32_t af[4] = {0u, 0u, 0u, 0u};
+              if (gid < r_pad) {
+                af[0] = *reinterpret_cast<const uint32_t*>(bk + gid * kHeadDim + 16 * kc + 2 * t);
+                af[2] = *reinterpret_cast<const uint32_t*>(bk + gid * kHeadDim + 16 * kc + 2 * t + 8);
+              }
+              if (gid + 8 < r_pad) {
+                af[1] = *reinterpret_cast<const uint32_t*>(bk + (gid + 8) * kHeadDim + 16 * kc + 2 * t);
+                af[3] = *reinterpret_cast<const uint32_t*>(bk + (gid + 8) * kHeadDim + 16 * kc + 2 * t + 8);
+              }
+              uint32_t b0 = 0u, b1 = 0u;
+              const int h = gid >> 1;
+              if ((gid & 1) == 0 && h < HPu) {
+                const __half* qrow = qs + h * kHeadDim + 16 * kc + 2 * t;
+                b0 = *reinterpret_cast<const uint32_t*>(qrow);
+                b1 = *reinterpret_cast<const uint32_t*>(qrow + 8);
+              }
+              mma16816(wacc, af, b0, b1);
             }
+            __syncwarp();
+            if (t < HP) {                           // D[rho][col 2t] = w[rho][head t]
+              wl[gid * WLS + t] = wacc[0] * a.scale_log2;
+              wl[(gid + 8) * WLS + t] = wacc[2] * a.scale_log2;
+            }
+            __syncwarp();
+            // B operand of the low-rank key product, one per integer column tile: column 4u holds the high parts of
+            // head 2 nt + u, column 4u + 1 the remainders, the other columns are zero -- so that the lane that
+            // finishes the integer sum of a head also receives the head's low-rank term
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {            // channel chunks 4 hf .. 4 hf + 3
-              uint32_t af[4][4];
-              if (!kBuf) {
-                if (BITS == 2) {
-                  uint32_t r[8];
-                  unpack_word<2>(hf == 0 ? w0.x : w0.y, r);
+            for (int nt = 0; nt < NT; ++nt) {
+              const int h = HP == 1 ? 0 : 2 * nt + (gid >> 2);
+              uint32_t hi0, lo0, hi1, lo1;
+              split_hi_lo(wl[(2 * t) * WLS + h], wl[(2 * t + 1) * WLS + h], hi0, lo0);
+              split_hi_lo(wl[(2 * t + 8) * WLS + h], wl[(2 * t + 9) * WLS + h], hi1, lo1);
+              bw[nt][0] = limb_b == 0 ? hi0 : (limb_b == 1 ? lo0 : 0u);
+              bw[nt][1] = limb_b == 0 ? hi1 : (limb_b == 1 ? lo1 : 0u);
+            }
+            __syncwarp();
+          }
+
+          // ---------------- B operand of the key scores: the block-wide fixed-point image of q * scale per channel,
+          //                  as four signed base-256 digits; c_h = sum q * zero; sparse key term scattered to its token
+          {
+            const uint4 kz = reinterpret_cast<const uint4*>(kp + off_kscale)[lane];
+            const uint32_t w4[4] = {kz.x, kz.y, kz.z, kz.w};
+            float sc4[4], zr4[4];
 #pragma unroll
-                  for (int u2 = 0; u2 < 8; ++u2) af[u2 >> 1][(u2 & 1) * 2] = r[u2];
-                  unpack_word<2>(hf == 0 ? w0.z : w0.w, r);
+            for (int j = 0; j < 4; ++j) {
+              sc4[j] = __low2float(u32_as_h2(w4[j]));
+              zr4[j] = __high2float(u32_as_h2(w4[j]));
+            }
+            // this lane's four channels sit in 32-channel chunk lane / 8, i.e. in code field (lane / 8) % F: the digits
+            // carry the power of two that brings every field to the weight of the highest one
+            const int sh = BITS * (F - 1 - ((lane >> 3) % F));
+            const uint32_t mulc = 1u << sh, addc = 0x80808080u - (kMagicBits << sh);
+            const int ed = float_exponent(dmax_k);
+            float qS[HP][4];
+            int eK[HP];
 #pragma unroll
-                  for (int u2 = 0; u2 < 8; ++u2) af[u2 >> 1][(u2 & 1) * 2 + 1] = r[u2];
+            for (int h = 0; h < HP; ++h) {
+              eK[h] = 0;
+              if (h < HPu) {
+                float qv[4];
+                if (HP == 1) {
+                  qv[0] = qreg[0]; qv[1] = qreg[1]; qv[2] = qreg[2]; qv[3] = qreg[3];
                 } else {
+                  const uint2 qh = *reinterpret_cast<const uint2*>(qs + h * kHeadDim + lane * 4);
+                  const __half2 q01 = u32_as_h2(qh.x), q23 = u32_as_h2(qh.y);
+                  qv[0] = __low2float(q01) * a.scale_log2; qv[1] = __high2float(q01) * a.scale_log2;
+                  qv[2] = __low2float(q23) * a.scale_log2; qv[3] = __high2float(q23) * a.scale_log2;
+                }
+                float qd[4];
 #pragma unroll
-                  for (int th = 0; th < 2; ++th) {
-                    const uint4 w = th == 0 ? w0 : w1;
-                    uint32_t r[4];
-                    unpack_word<4>(hf == 0 ? w.x : w.z, r);
+                for (int j = 0; j < 4; ++j) qd[j] = qv[j] * sc4[j];
+                const float am = fmaxf(fmaxf(fabsf(qd[0]), fabsf(qd[1])), fmaxf(fabsf(qd[2]), fabsf(qd[3])));
+                const uint32_t mb = warp_max_u32(__float_as_uint(am));     // non-negative floats order like their bits
+                const int e = clamp60(21 - ((int)(mb >> 23) - 127));        // |q * scale| * 2^e < 2^22
+                eK[h] = e;
+                const float Sk = pow2i(e);
+                uint32_t z[4];
 #pragma unroll
-                    for (int u2 = 0; u2 < 4; ++u2) af[u2 >> 1][(u2 & 1) * 2 + th] = r[u2];
-                    unpack_word<4>(hf == 0 ? w.y : w.w, r);
+                for (int j = 0; j < 4; ++j)
+                  z[j] = (__float_as_uint(fmaf(qd[j], Sk, kMagic)) * mulc + addc) ^ 0x80808080u;    // balanced digits
+                // digits of four channels -> one register per limb (bytes = the lane's four channels in order)
+                const uint32_t p01l = __byte_perm(z[0], z[1], 0x5140), p23l = __byte_perm(z[2], z[3], 0x5140);
+                const uint32_t p01h = __byte_perm(z[0], z[1], 0x7362), p23h = __byte_perm(z[2], z[3], 0x7362);
+                uint32_t* row = xr + (h * 4) * kFragKRow + (lane >> 3) * 8 + (lane & 3) * 2 + ((lane >> 2) & 1);
+                row[0] = __byte_perm(p01l, p23l, 0x5410);
+                row[kFragKRow] = __byte_perm(p01l, p23l, 0x7632);
+                row[2 * kFragKRow] = __byte_perm(p01h, p23h, 0x5410);
+                row[3 * kFragKRow] = __byte_perm(p01h, p23h, 0x7632);
+
+                float c = fmaf(qv[0], zr4[0], fmaf(qv[1], zr4[1], fmaf(qv[2], zr4[2], qv[3] * zr4[3])));   // this lane's part
+                if (HP != 4) {
 #pragma unroll
-                    for (int u2 = 0; u2 < 4; ++u2) af[2 + (u2 >> 1)][(u2 & 1) * 2 + th] = r[u2];
-                  }
+                  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+                }
+                const int sexp = clamp60(21 - qexp_s[h] - ed);
+                const float Sx = pow2i(sexp);
+                qS[h][0] = qv[0] * Sx; qS[h][1] = qv[1] * Sx; qS[h][2] = qv[2] * Sx; qS[h][3] = qv[3] * Sx;
+                c_zero[h] = c; sexp_k[h] = sexp;
+              }
+            }
+            if (HP == 4) {            // c_zero of four heads: sums over the warp
+              // four sums at once: two exchange steps halve what a lane carries, a butterfly finishes the one value left
+              // (head 2 * bit4 + bit3 of the lane), four broadcasts hand the sums back: 10 shuffles instead of 20
+              float s0 = c_zero[0], s1 = c_zero[1 % HP];
+              {
+                const bool up = (lane & 16) != 0;
+                const float send0 = up ? c_zero[0] : c_zero[2 % HP], keep0 = up ? c_zero[2 % HP] : c_zero[0];
+                const float send1 = up ? c_zero[1 % HP] : c_zero[3 % HP], keep1 = up ? c_zero[3 % HP] : c_zero[1 % HP];
+                s0 = keep0 + __shfl_xor_sync(0xffffffffu, send0, 16);
+                s1 = keep1 + __shfl_xor_sync(0xffffffffu, send1, 16);
+              }
+              {
+                const bool up = (lane & 8) != 0;
+                const float send = up ? s0 : s1, keep = up ? s1 : s0;
+                s0 = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+              }
+#pragma unroll
+              for (int o = 4; o > 0; o >>= 1) s0 += __shfl_xor_sync(0xffffffffu, s0, o);
+#pragma unroll
+              for (int h = 0; h < HP; ++h) c_zero[h] = __shfl_sync(0xffffffffu, s0, 8 * h);
+            }
+            // what turns this lane's integer sums of column tile nt into scores: the inverse fixed-point scale of the
+            // head it serves, the weight of the highest field, and 2^16 for the high limb pair
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              int e = eK[HP == 1 ? 0 : 2 * nt];
+              if (HP > 1 && (t >> 1)) e = eK[HP == 1 ? 0 : 2 * nt + 1];
+              kscl[nt] = pow2i(-e - kTop + (pair_hi ? 16 : 0));
+            }
+            if (k2k > 0) {
+              auto k_entry = [&](int j, float val, int idx) {
+                const float d = val - zr4[j];
+#pragma unroll
+                for (int h = 0; h < HP; ++h)
+                  if (h < HPu) atomicAdd(&corr_k[h * maxT + idx], __float2int_rn(qS[h][j] * d));
+              };
+              if (k2k == 2) {
+                const uint4 ov = reinterpret_cast<const uint4*>(kp + off_koval)[lane];
+                const uint2 oi = reinterpret_cast<const uint2*>(kp + off_koidx)[lane];
+                const uint32_t o4[4] = {ov.x, ov.y, ov.z, ov.w};
+                const uint32_t i2[2] = {oi.x, oi.y};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  k_entry(j, __low2float(u32_as_h2(o4[j])), (i2[j >> 1] >> (16 * (j & 1))) & 0xFFu);
+                  k_entry(j, __high2float(u32_as_h2(o4[j])), (i2[j >> 1] >> (16 * (j & 1) + 8)) & 0xFFu);
+                }
+              } else if (k2k == 4) {
+                // this lane's 4 channels x 4 entries: 32 bytes of values, 16 bytes of token indices
+                const uint4 ova = reinterpret_cast<const uint4*>(kp + off_koval)[2 * lane];
+                const uint4 ovb = reinterpret_cast<const uint4*>(kp + off_koval)[2 * lane + 1];
+                const uint4 oi = reinterpret_cast<const uint4*>(kp + off_koidx)[lane];
+                const uint32_t o8[8] = {ova.x, ova.y, ova.z, ova.w, ovb.x, ovb.y, ovb.z, ovb.w};
+                const uint32_t i4[4] = {oi.x, oi.y, oi.z, oi.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  k_entry(j, __low2float(u32_as_h2(o8[2 * j])), i4[j] & 0xFFu);
+                  k_entry(j, __high2float(u32_as_h2(o8[2 * j])), (i4[j] >> 8) & 0xFFu);
+                  k_entry(j, __low2float(u32_as_h2(o8[2 * j + 1])), (i4[j] >> 16) & 0xFFu);
+                  k_entry(j, __high2float(u32_as_h2(o8[2 * j + 1])), i4[j] >> 24);
                 }
               } else {
+                const __half* ov = reinterpret_cast<const __half*>(kp + off_koval) + lane * 4 * k2k;
+                const unsigned char* oi = kp + off_koidx + lane * 4 * k2k;
 #pragma unroll
-                for (int k4 = 0; k4 < 4; ++k4)
-                  ldmatrix_x4(af[k4], stK + ((lane & 7) + 8 * ((lane >> 3) & 1)) * kBufPitch +
-                                          (16 * (4 * hf + k4) + 8 * (lane >> 4)) * 2);
+                for (int j = 0; j < 4; ++j)
+#pragma unroll 1
+                  for (int e = 0; e < k2k; ++e) k_entry(j, __half2float(ov[j * k2k + e]), oi[j * k2k + e]);
               }
-#pragma unroll
-              for (int k4 = 0; k4 < 4; ++k4)
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt)
-                  mma16816(acc[hf][nt], af[k4], bq[nt][4 * hf + k4][0], bq[nt][4 * hf + k4][1]);
             }
-            if (!kBuf) {                                // low-rank key term: A_K rows times w (zero rows when r = 0)
+          }
+          __syncwarp();
+          // this lane's B registers: limb gid % 4 of head hcol(nt) for the four 32-channel chunks
+          uint32_t bK[NT][4][2];
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            const int hcol = HP == 1 ? 0 : 2 * nt + (gid >> 2);
+            const uint32_t* row = xr + (hcol * 4 + limb_b) * kFragKRow + 2 * t;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const uint2 v = *reinterpret_cast<const uint2*>(row + c * 8);
+              bK[nt][c][0] = v.x; bK[nt][c][1] = v.y;
+            }
+          }
+
+          // ---------------- key scores, slab by slab; scores go to shared memory
+          {
+            const bool pa0 = 2 * t < r_pad, pa1 = 2 * t + 8 < r_pad;
+            const uint4* cwp = reinterpret_cast<const uint4*>(kp + off_kcodes) + lane;
+            const __half* akp = reinterpret_cast<const __half*>(kp + off_ak) + gid * r_pad + 2 * t;
+            const int ak8 = 8 * r_pad, ak_step = kSlab * r_pad;
+            int tok0 = gid;
+#pragma unroll (S::unroll)
+            for (int slab = 0; slab < nslab; ++slab) {
+              int acc[NT][4];
 #pragma unroll
               for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[1][nt][i] *= kKeyBack;
+                for (int i = 0; i < 4; ++i) acc[nt][i] = 0;
+#pragma unroll
+              for (int tau = 0; tau < KT; ++tau) {
+                const uint4 w = cwp[tau * 32];
+#pragma unroll
+                for (int j = 0; j < F; ++j) {
+                  constexpr uint32_t m0 = field_mask<BITS>(0);
+                  const uint32_t m = m0 << (BITS * j);
+                  const uint32_t af[4] = {w.x & m, w.y & m, w.z & m, w.w & m};
+#pragma unroll
+                  for (int nt = 0; nt < NT; ++nt) imma16832(acc[nt], af, bK[nt][F * tau + j][0], bK[nt][F * tau + j][1]);
+                }
+              }
+              cwp += KT * 32;
+              // low-rank key term: A_K rows times w (zero rows when r = 0)
               uint32_t aa[4] = {0u, 0u, 0u, 0u};
               if (pa0) {
                 aa[0] = *reinterpret_cast<const uint32_t*>(akp);
@@ -767,440 +776,491 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
               }
               akp += ak_step;
 #pragma unroll
-              for (int nt = 0; nt < NT; ++nt) mma16816(acc[1][nt], aa, bw[nt][0], bw[nt][1]);
-            }
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-              if (t + 4 * nt < HPu) {
-                // raw sums only: the zero-point constant and the sparse term are added in the softmax pass
-                const float back = kBuf ? 1.f : kKeyBack;
-                const float v0 = fmaf(acc[0][nt][0] + acc[0][nt][1], back, acc[1][nt][0] + acc[1][nt][1]);
-                const float v1 = fmaf(acc[0][nt][2] + acc[0][nt][3], back, acc[1][nt][2] + acc[1][nt][3]);
-                float* pr = ps + psoff[nt] + tok0;
-                pr[0] = v0; pr[8] = v1;
+              for (int nt = 0; nt < NT; ++nt) {
+                // low limb pair + 2^16 high limb pair, each lane converting its own pair; the partner adds the other
+                float f0 = (float)(acc[nt][0] + acc[nt][1] * 256) * kscl[nt];
+                float f1 = (float)(acc[nt][2] + acc[nt][3] * 256) * kscl[nt];
+                f0 += __shfl_xor_sync(0xffffffffu, f0, 1);
+                f1 += __shfl_xor_sync(0xffffffffu, f1, 1);
+                if (r_pad > 0) {
+                  float d[4];
+                  mma16816_z(d, aa, bw[nt][0], bw[nt][1]);
+                  f0 += d[0] + d[1];
+                  f1 += d[2] + d[3];
+                }
+                const int hd = HP == 1 ? 0 : 2 * nt + (t >> 1);
+                if (writer && hd < HPu) {
+                  // raw sums only: the zero-point constant and the sparse term are added in the softmax pass
+                  float* pr = ps + hd * maxT + tok0;
+                  pr[0] = f0; pr[8] = f1;
+                }
               }
+              tok0 += kSlab;
             }
-            tok0 += kSlab;
           }
-        };
-        k_slabs(std::integral_constant<bool, is_buf>{});
-      }
-      release();                                      // the key item is consumed
+          release();                                      // the key item is consumed
 
-      // after the running maximum grew: everything accumulated so far is scaled by alpha (per head)
-      auto apply_alpha = [&](const float (&alpha)[HP]) {                                      // warp-uniform: m_run is the same in every lane
-#pragma unroll
-          for (int nt = 0; nt < NT; ++nt) {
-            float al = alpha[4 * nt];
-#pragma unroll
-            for (int hh = 1; hh < 4; ++hh)
-              if (4 * nt + hh < HP && t == hh) al = alpha[4 * nt + hh];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) U[nt][i] *= al;
-#pragma unroll
-            for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-              for (int i = 0; i < 4; ++i) O[mt][nt][i] *= al;
-          }
+          // ================================================================ value item
+          unsigned char* stV = acquire();
+          if (!alive) return;
+          const unsigned char* vp = stV + a.bregion;          // value part of the record
+
+          // ---------------- softmax over the block, the B operands of the value products and the sparse value term in
+          //                  one pass over this lane's token pairs (pairs lane, lane + 32), probabilities in registers
+          constexpr int NPR = S::kDyn ? 2 : (S::T > 64 ? S::T / 64 : 1);
+          float2 sc[HP][NPR];
+          float alpha[HP], m_new[HP];
+          bool grew = false;
 #pragma unroll
           for (int h = 0; h < HP; ++h) {
+            alpha[h] = 1.f; m_new[h] = 0.f;
             if (h < HPu) {
+              const float Sik = pow2i(-sexp_k[h]);
+              float mx = -INFINITY;
 #pragma unroll
-              for (int g = 0; g < NGV; ++g) cm[h][g] *= alpha[h];
-              float4* oc = reinterpret_cast<float4*>(ocorr + h * kHeadDim + lane * 4);
-              float4 v = *oc;
-              v.x *= alpha[h]; v.y *= alpha[h]; v.z *= alpha[h]; v.w *= alpha[h];
-              *oc = v;
-            }
-          }
-              };
-      // Up to four query heads and a compile-time block shape: the softmax, the value operands and the value outliers
-      // run as one pass over this lane's token pairs with the probabilities in registers (the value item is waited
-      // for first, since its scales are needed).  Every other case takes the separate passes below.
-      constexpr bool kFuse = HP <= 4 && !S::kDyn && !is_buf;
-      unsigned char* stV = nullptr;
-      if (!kFuse) {
-      // ---------------- online softmax over the block: one rescale at most
-      {
-        float alpha[HP];
-        bool grew = false;
-#pragma unroll
-        for (int h = 0; h < HP; ++h) {
-          alpha[h] = 1.f;
-          if (h < HPu) {
-            float* row = ps + h * maxT;
-            int* crow = corr_k + h * maxT;
-            const float Sik = pow2i(-sexp_k[h]);
-            float mx = -INFINITY;
-#pragma unroll (TU)
-            for (int tk = lane; tk < valid_tokens; tk += 32) {
-              float v = row[tk] + c_zero[h];
-              if (!is_buf && k2k > 0) {
-                v = fmaf((float)crow[tk], Sik, v);
-                crow[tk] = 0;
+              for (int i = 0; i < NPR; ++i) {
+                const int tp = 2 * (lane + 32 * i);
+                float2 v = make_float2(-INFINITY, -INFINITY);
+                if (tp < T) {
+                  v = *reinterpret_cast<const float2*>(ps + h * maxT + tp);
+                  v.x += c_zero[h]; v.y += c_zero[h];
+                  if (k2k > 0) {
+                    const int2 c = *reinterpret_cast<const int2*>(corr_k + h * maxT + tp);
+                    v.x = fmaf((float)c.x, Sik, v.x);
+                    v.y = fmaf((float)c.y, Sik, v.y);
+                    *reinterpret_cast<int2*>(corr_k + h * maxT + tp) = make_int2(0, 0);
+                  }
+                }
+                sc[h][i] = v;
+                mx = fmaxf(mx, fmaxf(v.x, v.y));
               }
-              row[tk] = v;
-              mx = fmaxf(mx, v);
-            }
-            mx = warp_max(mx);
-            const float m_new = fmaxf(m_run[h], mx);       // finite: every block holds a valid token
-            if (m_new > m_run[h]) {
-              alpha[h] = exp2f(m_run[h] - m_new);
-              grew = true;
-              m_run[h] = m_new;
-            }
-            float l = 0.f;
-#pragma unroll (TU)
-            for (int tk = lane; tk < T; tk += 32) {
-              const float p = tk < valid_tokens ? exp2f(row[tk] - m_new) : 0.f;   // tokens past the end of the buffer
-              l += p;
-              row[tk] = p;
-            }
-            l_run[h] = fmaf(l_run[h], alpha[h], l);
-          }
-        }
-        if (grew) apply_alpha(alpha);
-      }
-      __syncwarp();
-      }
-
-      // ================================================================ value item
-      stV = acquire();
-      if (!alive) return;
-      const unsigned char* vp = stV + a.bregion;          // value part of the record
-      uint32_t* fragV = frag;                                         // [NT][NGV][nslab] rows of kFragStride words
-      uint32_t* fragP = frag + NT * NGV * nslab * kFragStride;        // [NT][nslab]
-      if (is_buf && valid_tokens < kSlab) {
-        // rows past the end of the buffer hold stale bytes: clear them (0 * garbage must stay 0)
-        for (int i = lane; i < (kSlab - valid_tokens) * (kBufPitch / 16); i += 32) {
-          const int r = valid_tokens + i / (kBufPitch / 16), cc = i % (kBufPitch / 16);
-          reinterpret_cast<uint4*>(stV + r * kBufPitch)[cc] = make_uint4(0u, 0u, 0u, 0u);
-        }
-        fence_async_smem();
-      }
-
-      if (kFuse) {
-        constexpr int NPR = S::T >= 64 ? S::T / 64 : 1;   // token pairs per lane
-        float2 sc[HP][NPR];
-        float alpha[HP], m_new[HP];
-        bool grew = false;
-#pragma unroll
-        for (int h = 0; h < HP; ++h) {
-          alpha[h] = 1.f; m_new[h] = 0.f;
-          if (h < HPu) {
-            const float Sik = pow2i(-sexp_k[h]);
-            float mx = -INFINITY;
-#pragma unroll
-            for (int i = 0; i < NPR; ++i) {
-              const int tp = 2 * (lane + 32 * i);
-              float2 v = *reinterpret_cast<const float2*>(ps + h * maxT + tp);
-              v.x += c_zero[h]; v.y += c_zero[h];
-              if (k2k > 0) {
-                const int2 c = *reinterpret_cast<const int2*>(corr_k + h * maxT + tp);
-                v.x = fmaf((float)c.x, Sik, v.x);
-                v.y = fmaf((float)c.y, Sik, v.y);
-                *reinterpret_cast<int2*>(corr_k + h * maxT + tp) = make_int2(0, 0);
-              }
-              sc[h][i] = v;
-              mx = fmaxf(mx, fmaxf(v.x, v.y));
-            }
-            mx = warp_max(mx);
-            m_new[h] = fmaxf(m_run[h], mx);
-            if (m_new[h] > m_run[h]) {                    // warp-uniform
-              alpha[h] = exp2f(m_run[h] - m_new[h]);
-              m_run[h] = m_new[h];
-              grew = true;
-            }
-          }
-        }
-        if (grew) apply_alpha(alpha);
-        const float Sv = pow2i(clamp60(21 - float_exponent(dmax_v)));
-        const __half2* vsz = reinterpret_cast<const __half2*>(vp + o_vsz);
-        float l[HP];
-#pragma unroll
-        for (int h = 0; h < HP; ++h) l[h] = 0.f;
-#pragma unroll
-        for (int i = 0; i < NPR; ++i) {
-          const int pr = lane + 32 * i, tp = 2 * pr;
-          const int s = pr >> 3, pi = pr & 7, tw = pi & 3, rg = pi >> 2;
-          float p[HP][2];
-          __half2 z[2][NGV];
-#pragma unroll
-          for (int g = 0; g < NGV; ++g) { z[0][g] = vsz[tp * NGV + g]; z[1][g] = vsz[(tp + 1) * NGV + g]; }
-#pragma unroll
-          for (int h = 0; h < HP; ++h) {
-            p[h][0] = p[h][1] = 0.f;
-            if (h < HPu) {
-              const float p0 = exp2f(sc[h][i].x - m_new[h]), p1 = exp2f(sc[h][i].y - m_new[h]);
-              p[h][0] = p0; p[h][1] = p1;
-              l[h] += p0 + p1;
-              const int col = 2 * (h & 3);
-              uint32_t hi, lo;
-              split_hi_lo(p0, p1, hi, lo);
-              uint32_t* bp = fragP + ((h >> 2) * nslab + s) * kFragStride + rg;
-              bp[(col * 4 + tw) * 2] = hi;
-              bp[((col + 1) * 4 + tw) * 2] = lo;
-#pragma unroll
-              for (int g = 0; g < NGV; ++g) {
-                split_hi_lo(p0 * __low2float(z[0][g]), p1 * __low2float(z[1][g]), hi, lo);
-                uint32_t* bv = fragV + (((h >> 2) * NGV + g) * nslab + s) * kFragStride + rg;
-                bv[(col * 4 + tw) * 2] = hi;
-                bv[((col + 1) * 4 + tw) * 2] = lo;
-                cm[h][g] = fmaf(p0, __high2float(z[0][g]), fmaf(p1, __high2float(z[1][g]), cm[h][g]));
+              mx = warp_max(mx);
+              m_new[h] = fmaxf(m_run[h], mx);
+              if (m_new[h] > m_run[h]) {                    // warp-uniform
+                alpha[h] = exp2f(m_run[h] - m_new[h]);
+                m_run[h] = m_new[h];
+                grew = true;
               }
             }
           }
-          if (k2v > 0) {                                  // sparse value term of the two tokens, scattered in fixed point
+          // The integer value sums carry the scale 2^eV_cur.  They are folded into the fp32 copy when the running
+          // maximum grew (everything so far shrinks by alpha), when this block's scales do not fit that exponent (too
+          // large: overflow of the 22-bit image; more than three bits too small: precision), or when the 32-bit range
+          // nears its end.
+          {
+            const int need = clamp60(21 - float_exponent(smax_v));      // p <= 1: p * scale * 2^need < 2^22
+            const bool exp_bad = eV_cur > need || eV_cur < need - 3;
+            const bool conv = tok_acc > 0 && (grew || exp_bad || tok_acc + T > kTokLimit);
+            if (conv) {
+              fold_O(alpha);
+              tok_acc = 0;
+            } else if (grew) {
+              scale_ocorr(alpha);
+            }
+            if (grew) {
 #pragma unroll
-            for (int e2 = 0; e2 < 2; ++e2) {
-              const int tk = tp + e2;
-              auto v_entry = [&](int g, float val, int idx) {
-                const float d = (val - __high2float(z[e2][g])) * Sv;
+              for (int i = 0; i < 4; ++i) {
+                float al = alpha[0];
 #pragma unroll
-                for (int h = 0; h < HP; ++h)
-                  if (h < HPu) atomicAdd(&corr_v[h * kHeadDim + g * GV + idx], __float2int_rn(p[h][e2] * d));
-              };
-              if (NGV * k2v == 4) {
-                const uint2 ov = reinterpret_cast<const uint2*>(vp + o_voval)[tk];
-                const uint32_t oi = reinterpret_cast<const uint32_t*>(vp + o_voidx)[tk];
-                v_entry(0, __low2float(u32_as_h2(ov.x)), oi & 0xFFu);
-                v_entry(0, __high2float(u32_as_h2(ov.x)), (oi >> 8) & 0xFFu);
-                v_entry(NGV == 2 ? 1 : 0, __low2float(u32_as_h2(ov.y)), (oi >> 16) & 0xFFu);
-                v_entry(NGV == 2 ? 1 : 0, __high2float(u32_as_h2(ov.y)), oi >> 24);
-              } else {
-                const __half* ov = reinterpret_cast<const __half*>(vp + o_voval) + (size_t)tk * NGV * k2v;
-                const unsigned char* oi = vp + o_voidx + (size_t)tk * NGV * k2v;
-#pragma unroll
-                for (int g = 0; g < NGV; ++g)
-#pragma unroll 1
-                  for (int e = 0; e < k2v; ++e) v_entry(g, __half2float(ov[g * k2v + e]), oi[g * k2v + e]);
+                for (int hh = 1; hh < HP; ++hh)
+                  if (t == hh) al = alpha[hh];
+                U[i] *= al;
               }
+#pragma unroll
+              for (int h = 0; h < HP; ++h)
+#pragma unroll
+                for (int g = 0; g < NGV; ++g) cm[h][g] *= alpha[h];
             }
+            if (tok_acc == 0 && exp_bad) eV_cur = need;
+            tok_acc += T;
           }
-        }
+          const float Sv = pow2i(eV_cur);
+          const float Sx = pow2i(clamp60(21 - float_exponent(dmax_v)));     // fixed-point scale of the sparse value term
+          const __half2* vsz = reinterpret_cast<const __half2*>(vp + o_vsz);
+          unsigned char* fragVb = reinterpret_cast<unsigned char*>(xr);
+          float l[HP];
 #pragma unroll
-        for (int h = 0; h < HP; ++h)
-          if (h < HPu) l_run[h] = fmaf(l_run[h], alpha[h], l[h]);
-      } else {
-      // ---------------- B operands of the value products: p * scale (per token and group) and p, split hi / lo;
-      //                  the zero-point term goes to the fp32 side sums cm
-#pragma unroll (TU)
-      for (int pr = lane; pr < T / 2; pr += 32) {      // this lane's token pairs
-        const int s = pr >> 3, pi = pr & 7, tw = pi & 3, rg = pi >> 2;
-        const int tp = 2 * pr;
+          for (int h = 0; h < HP; ++h) l[h] = 0.f;
 #pragma unroll
-        for (int h = 0; h < HP; ++h) {
-          if (h < HPu) {
-            const float2 pp = *reinterpret_cast<const float2*>(ps + h * maxT + tp);
-            const int col = 2 * (h & 3);
-            uint32_t hi, lo;
-            {
-              split_hi_lo(pp.x, pp.y, hi, lo);
-              uint32_t* bp = fragP + ((h >> 2) * nslab + s) * kFragStride + rg;
-              bp[(col * 4 + tw) * 2] = hi;
-              bp[((col + 1) * 4 + tw) * 2] = lo;
-            }
-            if (!is_buf) {
-              const __half2* vsz = reinterpret_cast<const __half2*>(vp + o_vsz) + tp * NGV;
+          for (int i = 0; i < NPR; ++i) {
+            const int pr = lane + 32 * i, tp = 2 * pr;
+            if (S::kDyn && tp >= T) break;
+            if (!S::kDyn && S::T < 64 && tp >= T) break;
+            const int s = pr >> 3, pi = pr & 7, tw = pi & 3, rg = pi >> 2;
+            // where this pair's two bytes go in a row of the value B operand: chunk, register (tokens 4t.. / 16+4t..),
+            // lane column, half word
+            const int vboff = (((pr >> 4) * 8 + ((pr & 7) >> 1) * 2 + ((pr & 15) >> 3)) << 2) + ((pr & 1) << 1);
+            float p[HP][2];
+            __half2 z[2][NGV];
 #pragma unroll
-              for (int g = 0; g < NGV; ++g) {
-                const __half2 z0 = vsz[g], z1 = vsz[NGV + g];
-                split_hi_lo(pp.x * __low2float(z0), pp.y * __low2float(z1), hi, lo);
-                uint32_t* bv = fragV + (((h >> 2) * NGV + g) * nslab + s) * kFragStride + rg;
-                bv[(col * 4 + tw) * 2] = hi;
-                bv[((col + 1) * 4 + tw) * 2] = lo;
-                cm[h][g] = fmaf(pp.x, __high2float(z0), fmaf(pp.y, __high2float(z1), cm[h][g]));
-              }
-            }
-          }
-        }
-      }
-      }
-      __syncwarp();
-
-      // ---------------- values: out += sum_tok (p * scale) * code on the tensor cores, low rank on the side
-      {
-        const bool pv0 = gid < r_pad, pv1 = gid + 8 < r_pad;
-        auto v_slabs = [&](auto buf_tag) {
-          constexpr bool kBuf = decltype(buf_tag)::value;
-          const uint4* cwp = reinterpret_cast<const uint4*>(vp) + lane;
-          const __half* avp = reinterpret_cast<const __half*>(vp + o_av) + gid * kSlab + 2 * t;
-          const uint32_t* fvp = fragV + ((gid & CMASK) * 4 + t) * 2;
-          const uint32_t* fpp = fragP + ((gid & CMASK) * 4 + t) * 2;
-          const int fstep = nslab * kFragStride, av_step = kSlab * r_pad;
-#pragma unroll (S::unroll)
-          for (int slab = 0; slab < nslab; ++slab) {
-            uint32_t bp[NT][2];
+            for (int g = 0; g < NGV; ++g) { z[0][g] = vsz[tp * NGV + g]; z[1][g] = vsz[(tp + 1) * NGV + g]; }
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-              const uint2 v = *reinterpret_cast<const uint2*>(fpp + nt * fstep);
-              bp[nt][0] = v.x; bp[nt][1] = v.y;
-            }
-            fpp += kFragStride;
-            if (!kBuf) {
-              uint32_t bv[NT][NGV][2];
-#pragma unroll
-              for (int nt = 0; nt < NT; ++nt)
+            for (int h = 0; h < HP; ++h) {
+              p[h][0] = p[h][1] = 0.f;
+              if (h < HPu) {
+                const float p0 = exp2f(sc[h][i].x - m_new[h]), p1 = exp2f(sc[h][i].y - m_new[h]);
+                p[h][0] = p0; p[h][1] = p1;
+                l[h] += p0 + p1;
+                if (r_pad > 0) {                              // fp16 fragments of p for the low-rank value term
+                  const int col = 2 * (h & 3);
+                  uint32_t hi, lo;
+                  split_hi_lo(p0, p1, hi, lo);
+                  uint32_t* bp = fragPc + s * kFragStride + rg;
+                  bp[(col * 4 + tw) * 2] = hi;
+                  bp[((col + 1) * 4 + tw) * 2] = lo;
+                }
 #pragma unroll
                 for (int g = 0; g < NGV; ++g) {
-                  const uint2 v = *reinterpret_cast<const uint2*>(fvp + (nt * NGV + g) * fstep);
-                  bv[nt][g][0] = v.x; bv[nt][g][1] = v.y;
+                  const uint32_t y0 = balanced_digits(__float_as_uint(fmaf(p0 * __low2float(z[0][g]), Sv, kMagic)) - kMagicBits);
+                  const uint32_t y1 = balanced_digits(__float_as_uint(fmaf(p1 * __low2float(z[1][g]), Sv, kMagic)) - kMagicBits);
+                  unsigned char* rowb = fragVb + ((g * HP + h) * 4) * RS * 4 + vboff;
+                  *reinterpret_cast<unsigned short*>(rowb) = (unsigned short)__byte_perm(y0, y1, 0x0040);
+                  *reinterpret_cast<unsigned short*>(rowb + RS * 4) = (unsigned short)__byte_perm(y0, y1, 0x0051);
+                  *reinterpret_cast<unsigned short*>(rowb + 2 * RS * 4) = (unsigned short)__byte_perm(y0, y1, 0x0062);
+                  cm[h][g] = fmaf(p0, __high2float(z[0][g]), fmaf(p1, __high2float(z[1][g]), cm[h][g]));
                 }
-              fvp += kFragStride;
-              constexpr int TPP = 8 / BITS;               // channel tiles per pair of words
+              }
+            }
+            if (k2v > 0) {                                  // sparse value term of the two tokens, scattered in fixed point
 #pragma unroll
-              for (int pl = 0; pl < BITS / 2; ++pl) {
-                const uint4 w = cwp[pl * 32];
-                const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
+              for (int e2 = 0; e2 < 2; ++e2) {
+                const int tk = tp + e2;
+                auto v_entry = [&](int g, float val, int idx) {
+                  const float d = (val - __high2float(z[e2][g])) * Sx;
 #pragma unroll
-                for (int wp = 0; wp < 2; ++wp) {
-                  uint32_t rA[16 / BITS], rB[16 / BITS];
-                  unpack_word<BITS>(wv[2 * wp], rA);
-                  unpack_word<BITS>(wv[2 * wp + 1], rB);
+                  for (int h = 0; h < HP; ++h)
+                    if (h < HPu) atomicAdd(&corr_v[h * kHeadDim + g * GV + idx], __float2int_rn(p[h][e2] * d));
+                };
+                if (NGV * k2v == 4) {
+                  const uint2 ov = reinterpret_cast<const uint2*>(vp + o_voval)[tk];
+                  const uint32_t oi = reinterpret_cast<const uint32_t*>(vp + o_voidx)[tk];
+                  v_entry(0, __low2float(u32_as_h2(ov.x)), oi & 0xFFu);
+                  v_entry(0, __high2float(u32_as_h2(ov.x)), (oi >> 8) & 0xFFu);
+                  v_entry(NGV == 2 ? 1 : 0, __low2float(u32_as_h2(ov.y)), (oi >> 16) & 0xFFu);
+                  v_entry(NGV == 2 ? 1 : 0, __high2float(u32_as_h2(ov.y)), oi >> 24);
+                } else {
+                  const __half* ov = reinterpret_cast<const __half*>(vp + o_voval) + (size_t)tk * NGV * k2v;
+                  const unsigned char* oi = vp + o_voidx + (size_t)tk * NGV * k2v;
 #pragma unroll
-                  for (int j = 0; j < TPP; ++j) {
-                    const int mt = TPP * (2 * pl + wp) + j, g = (mt * 16) / GV;
-                    const uint32_t av[4] = {rA[2 * j], rA[2 * j + 1], rB[2 * j], rB[2 * j + 1]};
+                  for (int g = 0; g < NGV; ++g)
+#pragma unroll 1
+                    for (int e = 0; e < k2v; ++e) v_entry(g, __half2float(ov[g * k2v + e]), oi[g * k2v + e]);
+                }
+              }
+            }
+          }
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) mma16816(O[mt][nt], av, bv[nt][g][0], bv[nt][g][1]);
+          for (int h = 0; h < HP; ++h)
+            if (h < HPu) l_run[h] = fmaf(l_run[h], alpha[h], l[h]);
+          __syncwarp();
+
+          // ---------------- values: out += sum_tok (p * scale) * code on the integer tensor cores, low rank on the side
+          {
+            const bool pv0 = gid < r_pad, pv1 = gid + 8 < r_pad;
+            const uint4* cwp = reinterpret_cast<const uint4*>(vp) + lane;
+            const __half* avp = reinterpret_cast<const __half*>(vp + o_av) + gid * kSlab + 2 * t;
+            const uint32_t* fpp = fragPc + ((gid & CMASK) * 4 + t) * 2;
+            const int av_step = kSlab * r_pad;
+#pragma unroll (S::unroll)
+            for (int ck = 0; ck < nchunk; ++ck) {
+              uint32_t bV[NGV][NT][2];
+#pragma unroll
+              for (int g = 0; g < NGV; ++g)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                  const int hcol = HP == 1 ? 0 : 2 * nt + (gid >> 2);
+                  const uint2 v = *reinterpret_cast<const uint2*>(xr + ((g * HP + hcol) * 4 + limb_b) * RS + ck * 8 + 2 * t);
+                  bV[g][nt][0] = v.x; bV[g][nt][1] = v.y;
+                }
+#pragma unroll
+              for (int tau = 0; tau < VT; ++tau) {
+                const uint4 w = cwp[tau * 32];
+#pragma unroll
+                for (int j = 0; j < F; ++j) {
+                  constexpr uint32_t m0 = field_mask<BITS>(0);
+                  const uint32_t m = m0 << (BITS * j);
+                  const int mt = F * tau + j, g = (mt * 16) / GV;
+                  const uint32_t af[4] = {w.x & m, w.y & m, w.z & m, w.w & m};
+#pragma unroll
+                  for (int nt = 0; nt < NT; ++nt) imma16832(O[mt][nt], af, bV[g][nt][0], bV[g][nt][1]);
+                }
+              }
+              cwp += VT * 32;
+              if (r_pad > 0) {
+                // low-rank value term, first product: U = A_V^T p, slab by slab
+#pragma unroll
+                for (int s2 = 0; s2 < 2; ++s2) {
+                  if (2 * ck + s2 < nslab) {
+                    const uint2 bpv = *reinterpret_cast<const uint2*>(fpp);
+                    fpp += kFragStride;
+                    uint32_t aa[4] = {0u, 0u, 0u, 0u};
+                    if (pv0) {
+                      aa[0] = *reinterpret_cast<const uint32_t*>(avp);
+                      aa[2] = *reinterpret_cast<const uint32_t*>(avp + 8);
+                    }
+                    if (pv1) {
+                      aa[1] = *reinterpret_cast<const uint32_t*>(avp + 8 * kSlab);
+                      aa[3] = *reinterpret_cast<const uint32_t*>(avp + 8 * kSlab + 8);
+                    }
+                    avp += av_step;
+                    mma16816(U, aa, bpv.x, bpv.y);
                   }
                 }
               }
-              cwp += SLABW;
-              // low-rank value term, first product: U = A_V^T p (zero rows when r = 0)
-              uint32_t aa[4] = {0u, 0u, 0u, 0u};
-              if (pv0) {
-                aa[0] = *reinterpret_cast<const uint32_t*>(avp);
-                aa[2] = *reinterpret_cast<const uint32_t*>(avp + 8);
-              }
-              if (pv1) {
-                aa[1] = *reinterpret_cast<const uint32_t*>(avp + 8 * kSlab);
-                aa[3] = *reinterpret_cast<const uint32_t*>(avp + 8 * kSlab + 8);
-              }
-              avp += av_step;
+            }
+            if (r_pad > 0) u_pending = true;
+          }
+
+          // ---------------- sparse value term: the fixed-point sums of this block join the fp32 copy
+          if (k2v > 0) {
+            const float Si = 1.0f / Sx;
 #pragma unroll
-              for (int nt = 0; nt < NT; ++nt) mma16816(U[nt], aa, bp[nt][0], bp[nt][1]);
-            } else {
-#pragma unroll
-              for (int mt = 0; mt < 8; ++mt) {
-                uint32_t av[4];
-                ldmatrix_x4_trans(av, stV + ((lane & 7) + 8 * (lane >> 4)) * kBufPitch + (16 * mt + 8 * ((lane >> 3) & 1)) * 2);
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                  if (o_plain) mma16816(O[mt][nt], av, bp[nt][0], bp[nt][1]);
-                  else add_scaled(O[mt][nt], mt, av, bp[nt][0], bp[nt][1]);
-                }
+            for (int h = 0; h < HP; ++h) {
+              if (h < HPu) {
+                int4* cv = reinterpret_cast<int4*>(corr_v + h * kHeadDim) + lane;
+                float4* oc = reinterpret_cast<float4*>(ocorr + h * kHeadDim) + lane;
+                const int4 v = *cv;
+                *cv = make_int4(0, 0, 0, 0);
+                float4 o = *oc;
+                o.x = fmaf((float)v.x, Si, o.x);
+                o.y = fmaf((float)v.y, Si, o.y);
+                o.z = fmaf((float)v.z, Si, o.z);
+                o.w = fmaf((float)v.w, Si, o.w);
+                *oc = o;
               }
             }
+            __syncwarp();
           }
-        };
-        v_slabs(std::integral_constant<bool, is_buf>{});
-        if (!is_buf && r_pad > 0) u_pending = true;
-      }
 
-      // ---------------- sparse value term: p[tok] * (x - zero[tok, g]) scattered to the outlier's channel
-      if (!is_buf && k2v > 0) {
-        const int sexp = clamp60(21 - float_exponent(dmax_v));
-        const float S = pow2i(sexp), Si = pow2i(-sexp);
-        const __half2* vsz = reinterpret_cast<const __half2*>(vp + o_vsz);
-        const unsigned char* voval = vp + o_voval;
-        const unsigned char* voidx = vp + o_voidx;
-#pragma unroll (TU)
-        for (int tk = lane; tk < (kFuse ? 0 : T); tk += 32) {      // the fused pass above has scattered them already
-          float pS[HP];
+          // ---------------- end of a segment (or of this warp's share of it): out += B_V U, into the fp32 copy
+          if (with_bv && u_pending) {
+            __syncwarp();
+            if (t < HP) {
+              wl[gid * WLS + t] = U[0] + U[1];
+              wl[(gid + 8) * WLS + t] = U[2] + U[3];
+            }
 #pragma unroll
-          for (int h = 0; h < HP; ++h) pS[h] = h < HPu ? ps[h * maxT + tk] * S : 0.f;
-          auto v_entry = [&](int g, float val, int idx) {
-            const float d = val - __high2float(vsz[tk * NGV + g]);
-            const int ch = g * GV + idx;
+            for (int i = 0; i < 4; ++i) U[i] = 0.f;
+            __syncwarp();
+            uint32_t bu[2];
+            {
+              const int h = (gid >> 1) & (HP - 1);
+              uint32_t hi0, lo0, hi1, lo1;
+              split_hi_lo(wl[(2 * t) * WLS + h], wl[(2 * t + 1) * WLS + h], hi0, lo0);
+              split_hi_lo(wl[(2 * t + 8) * WLS + h], wl[(2 * t + 9) * WLS + h], hi1, lo1);
+              bu[0] = (gid & 1) ? lo0 : hi0;
+              bu[1] = (gid & 1) ? lo1 : hi1;
+            }
+            const __half* bvf = reinterpret_cast<const __half*>(stV);      // B_V [128][r_pad]
 #pragma unroll
-            for (int h = 0; h < HP; ++h)
-              if (h < HPu) atomicAdd(&corr_v[h * kHeadDim + ch], __float2int_rn(pS[h] * d));
-          };
-          if (NGV * k2v == 4) {
-            const uint2 ov = reinterpret_cast<const uint2*>(voval)[tk];
-            const uint32_t oi = reinterpret_cast<const uint32_t*>(voidx)[tk];
-            v_entry(0, __low2float(u32_as_h2(ov.x)), oi & 0xFFu);
-            v_entry(0, __high2float(u32_as_h2(ov.x)), (oi >> 8) & 0xFFu);
-            v_entry(NGV == 2 ? 1 : 0, __low2float(u32_as_h2(ov.y)), (oi >> 16) & 0xFFu);
-            v_entry(NGV == 2 ? 1 : 0, __high2float(u32_as_h2(ov.y)), oi >> 24);
-          } else {
-            const __half* ov = reinterpret_cast<const __half*>(voval) + (size_t)tk * NGV * k2v;
-            const unsigned char* oi = voidx + (size_t)tk * NGV * k2v;
-#pragma unroll
-            for (int g = 0; g < NGV; ++g)
-#pragma unroll 1
-              for (int e = 0; e < k2v; ++e) v_entry(g, __half2float(ov[g * k2v + e]), oi[g * k2v + e]);
+            for (int mt = 0; mt < 8; ++mt) {
+              uint32_t aa[4] = {0u, 0u, 0u, 0u};
+              const __half* r0 = bvf + (16 * mt + gid) * r_pad, *r1 = bvf + (16 * mt + gid + 8) * r_pad;
+              if (2 * t < r_pad) {
+                aa[0] = *reinterpret_cast<const uint32_t*>(r0 + 2 * t);
+                aa[1] = *reinterpret_cast<const uint32_t*>(r1 + 2 * t);
+              }
+              if (2 * t + 8 < r_pad) {
+                aa[2] = *reinterpret_cast<const uint32_t*>(r0 + 2 * t + 8);
+                aa[3] = *reinterpret_cast<const uint32_t*>(r1 + 2 * t + 8);
+              }
+              float d[4];
+              mma16816_z(d, aa, bu[0], bu[1]);
+              if (t < HPu) {                              // columns 2t, 2t + 1: high and low part of head t
+                float* oc = ocorr + t * kHeadDim + 16 * mt + gid;
+                oc[0] += d[0] + d[1];
+                oc[8] += d[2] + d[3];
+              }
+            }
+            __syncwarp();
+            u_pending = false;
           }
-        }
+          release();                                      // the value item is consumed
+        };
+        if (NGV == 2 && c_shape == 1) body(ShapeA1<BITS>{});
+        else if (NGV == 2 && c_shape == 2) body(ShapeA2<BITS>{});
+        else if (NGV == 1 && c_shape == 3) body(ShapeB1<BITS>{});
+        else if (NGV == 1 && c_shape == 4) body(ShapeB2<BITS>{});
+        else body(DynShape{});
+        if (!alive) break;
+      }
+      if (!alive) break;
+      // the integer sums and the zero-point side sums join the fp32 copy
+      {
+        float one[HP];
+#pragma unroll
+        for (int h = 0; h < HP; ++h) one[h] = 1.f;
+        if (tok_acc > 0) fold_O(one);
         __syncwarp();
 #pragma unroll
         for (int h = 0; h < HP; ++h) {
           if (h < HPu) {
-            int4* cv = reinterpret_cast<int4*>(corr_v + h * kHeadDim) + lane;
+            float add = 0.f;
+#pragma unroll
+            for (int g = 0; g < NGV; ++g) {
+              float c = cm[h][g];
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+              if ((lane * 4) / GV == g) add = c;
+            }
             float4* oc = reinterpret_cast<float4*>(ocorr + h * kHeadDim) + lane;
-            const int4 v = *cv;
-            *cv = make_int4(0, 0, 0, 0);
-            float4 o = *oc;
-            o.x = fmaf((float)v.x, Si, o.x);
-            o.y = fmaf((float)v.y, Si, o.y);
-            o.z = fmaf((float)v.z, Si, o.z);
-            o.w = fmaf((float)v.w, Si, o.w);
-            *oc = o;
+            float4 v = *oc;
+            v.x += add; v.y += add; v.z += add; v.w += add;
+            *oc = v;
+          }
+        }
+        __syncwarp();
+      }
+    }
+
+    // ==================================================================== fp16 rows of the streaming buffer
+    if (blk_hi > a.n_blocks_c && alive) {
+      float Ob[8][4];
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) Ob[mt][i] = 0.f;
+      // B operand of the scores: q * scale * log2 e per channel, split into fp16 high and low parts (columns 2h, 2h + 1)
+      __syncwarp();
+      {
+        const int kc = lane >> 2, reg = (lane >> 1) & 1, tA = 2 * (lane & 1);
+#pragma unroll
+        for (int h = 0; h < HP; ++h) {
+          if (h < HPu) {
+            const uint2 qh = *reinterpret_cast<const uint2*>(qs + h * kHeadDim + lane * 4);
+            const __half2 q01 = u32_as_h2(qh.x), q23 = u32_as_h2(qh.y);
+            uint32_t hiA, loA, hiB, loB;
+            split_hi_lo(__low2float(q01) * a.scale_log2, __high2float(q01) * a.scale_log2, hiA, loA);
+            split_hi_lo(__low2float(q23) * a.scale_log2, __high2float(q23) * a.scale_log2, hiB, loB);
+            uint32_t* base = xr + kc * kFragStride + reg;
+            const int cl = 2 * (h & 3);
+            base[(4 * cl + tA) * 2] = hiA;
+            base[(4 * (cl + 1) + tA) * 2] = loA;
+            base[(4 * cl + tA + 1) * 2] = hiB;
+            base[(4 * (cl + 1) + tA + 1) * 2] = loB;
           }
         }
       }
-
-      // ---------------- end of a segment (or of this warp's share of it): out += B_V U
-      if (with_bv && u_pending) {
-        __syncwarp();
+      __syncwarp();
+      uint32_t bq[8][2];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          if (t + 4 * nt < HP) {
-            wl[gid * WLS + t + 4 * nt] = U[nt][0] + U[nt][1];
-            wl[(gid + 8) * WLS + t + 4 * nt] = U[nt][2] + U[nt][3];
+      for (int kc = 0; kc < 8; ++kc) {
+        const uint2 v = *reinterpret_cast<const uint2*>(xr + kc * kFragStride + ((gid & CMASK) * 4 + t) * 2);
+        bq[kc][0] = v.x; bq[kc][1] = v.y;
+      }
+#pragma unroll 1
+      for (int blk = max(blk_lo, a.n_blocks_c); blk < blk_hi; ++blk) {
+        const int valid_tokens = min(kSlab, a.buf_len - (blk - a.n_blocks_c) * kSlab);
+        // ---- key rows
+        unsigned char* stK = acquire();
+        if (!alive) break;
+        {
+          float acc[2][4];
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[hf][i] = 0.f;
+#pragma unroll
+          for (int kc = 0; kc < 8; ++kc) {
+            uint32_t af[4];
+            ldmatrix_x4(af, stK + ((lane & 7) + 8 * ((lane >> 3) & 1)) * kBufPitch + (16 * kc + 8 * (lane >> 4)) * 2);
+            mma16816(acc[kc & 1], af, bq[kc][0], bq[kc][1]);
           }
+          if (t < HPu) {
+            float* pr = ps + t * maxT + gid;
+            pr[0] = (acc[0][0] + acc[0][1]) + (acc[1][0] + acc[1][1]);
+            pr[8] = (acc[0][2] + acc[0][3]) + (acc[1][2] + acc[1][3]);
+          }
+        }
+        release();
+        __syncwarp();
+        // ---- online softmax over the slab: one rescale at most
+        {
+          float alpha[HP];
+          bool grew = false;
 #pragma unroll
-          for (int i = 0; i < 4; ++i) U[nt][i] = 0.f;
+          for (int h = 0; h < HP; ++h) {
+            alpha[h] = 1.f;
+            if (h < HPu) {
+              float* row = ps + h * maxT;
+              const float v = lane < valid_tokens ? row[lane & 15] : -INFINITY;
+              const float mx = warp_max(v);
+              const float m_new = fmaxf(m_run[h], mx);       // finite: every slab holds a valid token
+              if (m_new > m_run[h]) {
+                alpha[h] = exp2f(m_run[h] - m_new);
+                grew = true;
+                m_run[h] = m_new;
+              }
+              const float p = lane < valid_tokens ? exp2f(v - m_new) : 0.f;   // tokens past the end of the buffer
+              l_run[h] = fmaf(l_run[h], alpha[h], lane < kSlab ? p : 0.f);
+              __syncwarp();
+              if (lane < kSlab) row[lane] = p;
+            }
+          }
+          if (grew) {
+            float al = alpha[0];
+#pragma unroll
+            for (int hh = 1; hh < HP; ++hh)
+              if (t == hh) al = alpha[hh];
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+              for (int i = 0; i < 4; ++i) Ob[mt][i] *= al;
+            scale_ocorr(alpha);
+          }
         }
         __syncwarp();
-        uint32_t bu[NT][2];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          const int h = (gid >> 1) + 4 * nt;
-          uint32_t hi0, lo0, hi1, lo1;
-          split_hi_lo(wl[(2 * t) * WLS + (h & HMASK)], wl[(2 * t + 1) * WLS + (h & HMASK)], hi0, lo0);
-          split_hi_lo(wl[(2 * t + 8) * WLS + (h & HMASK)], wl[(2 * t + 9) * WLS + (h & HMASK)], hi1, lo1);
-          bu[nt][0] = (gid & 1) ? lo0 : hi0;
-          bu[nt][1] = (gid & 1) ? lo1 : hi1;
+        // ---- value rows
+        unsigned char* stV = acquire();
+        if (!alive) break;
+        if (valid_tokens < kSlab) {
+          // rows past the end of the buffer hold stale bytes: clear them (0 * garbage must stay 0)
+          for (int i = lane; i < (kSlab - valid_tokens) * (kBufPitch / 16); i += 32) {
+            const int r = valid_tokens + i / (kBufPitch / 16), cc = i % (kBufPitch / 16);
+            reinterpret_cast<uint4*>(stV + r * kBufPitch)[cc] = make_uint4(0u, 0u, 0u, 0u);
+          }
+          fence_async_smem();
         }
-        const __half* bvf = reinterpret_cast<const __half*>(stV);      // B_V [128][r_pad]
+        // probabilities -> fp16 high / low fragments
+        if (lane < kSlab / 2) {
+          const int pr = lane, pi = pr & 7, tw = pi & 3, rg = pi >> 2;
+#pragma unroll
+          for (int h = 0; h < HP; ++h) {
+            if (h < HPu) {
+              const float2 pp = *reinterpret_cast<const float2*>(ps + h * maxT + 2 * pr);
+              const int col = 2 * (h & 3);
+              uint32_t hi, lo;
+              split_hi_lo(pp.x, pp.y, hi, lo);
+              uint32_t* bp = fragPb + rg;
+              bp[(col * 4 + tw) * 2] = hi;
+              bp[((col + 1) * 4 + tw) * 2] = lo;
+            }
+          }
+        }
+        __syncwarp();
+        {
+          const uint2 bpv = *reinterpret_cast<const uint2*>(fragPb + ((gid & CMASK) * 4 + t) * 2);
+#pragma unroll
+          for (int mt = 0; mt < 8; ++mt) {
+            uint32_t av[4];
+            ldmatrix_x4_trans(av, stV + ((lane & 7) + 8 * (lane >> 4)) * kBufPitch + (16 * mt + 8 * ((lane >> 3) & 1)) * 2);
+            mma16816(Ob[mt], av, bpv.x, bpv.y);
+          }
+        }
+        release();
+      }
+      if (!alive) break;
+      // the tensor-core part of the buffer rows joins the fp32 copy
+      __syncwarp();
+      if (t < HPu) {
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt) {
-          uint32_t aa[4] = {0u, 0u, 0u, 0u};
-          const __half* r0 = bvf + (16 * mt + gid) * r_pad, *r1 = bvf + (16 * mt + gid + 8) * r_pad;
-          if (2 * t < r_pad) {
-            aa[0] = *reinterpret_cast<const uint32_t*>(r0 + 2 * t);
-            aa[1] = *reinterpret_cast<const uint32_t*>(r1 + 2 * t);
-          }
-          if (2 * t + 8 < r_pad) {
-            aa[2] = *reinterpret_cast<const uint32_t*>(r0 + 2 * t + 8);
-            aa[3] = *reinterpret_cast<const uint32_t*>(r1 + 2 * t + 8);
-          }
-#pragma unroll
-          for (int nt = 0; nt < NT; ++nt) add_scaled(O[mt][nt], mt, aa, bu[nt][0], bu[nt][1]);
+          float* oc = ocorr + t * kHeadDim + 16 * mt + gid;
+          oc[0] += Ob[mt][0] + Ob[mt][1];
+          oc[8] += Ob[mt][2] + Ob[mt][3];
         }
-        u_pending = false;
       }
-      release();                                      // the value item is consumed
-      };
-      if (buf_blk) body(BufShape{});
-      else if (NGV == 2 && c_shape == 1) body(ShapeA1<BITS>{});
-      else if (NGV == 2 && c_shape == 2) body(ShapeA2<BITS>{});
-      else if (NGV == 1 && c_shape == 3) body(ShapeB1<BITS>{});
-      else if (NGV == 1 && c_shape == 4) body(ShapeB2<BITS>{});
-      else body(DynShape{});
-      if (!alive) break;
+      __syncwarp();
     }
     if (!alive) break;
 
@@ -1210,58 +1270,25 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
       n_parts = parts_u;
       slot = part;
     } else {
-      const long long F = (long long)a.cc.BH * passes * NB, NW = gridDim.x;
+      const long long Fl = (long long)a.cc.BH * passes * NB, NW = gridDim.x;
       const long long bflat = (long long)u * NB, eflat = bflat + NB;
-      const long long w_first = ((bflat + 1) * NW + F - 1) / F - 1;
-      const long long w_last = (eflat * NW + F - 1) / F - 1;
+      const long long w_first = ((bflat + 1) * NW + Fl - 1) / Fl - 1;
+      const long long w_last = (eflat * NW + Fl - 1) / Fl - 1;
       n_parts = (int)(w_last - w_first + 1);
       slot = (int)(blockIdx.x - w_first);
     }
     float* part_base = a.partial + ((size_t)u * a.max_parts + slot) * (HP * kPartRow);
-    float cm_own[NT][NGV], m_own[NT], l_own[NT];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      m_own[nt] = 0.f; l_own[nt] = 0.f;
-#pragma unroll
-      for (int g = 0; g < NGV; ++g) cm_own[nt][g] = 0.f;
-    }
+    __syncwarp();
 #pragma unroll
     for (int h = 0; h < HP; ++h) {
-      float l = l_run[h];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-      if ((h & 3) == t) { m_own[h >> 2] = m_run[h]; l_own[h >> 2] = l; }
-#pragma unroll
-      for (int g = 0; g < NGV; ++g) {
-        float c = cm[h][g];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-        if ((h & 3) == t) cm_own[h >> 2][g] = c;
-      }
-    }
-    __syncwarp();
-    // the tensor-core part of the output joins the sparse part in shared memory, so that the partial goes out as
-    // one 16-byte store per lane and head
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const int h = t + 4 * nt;
       if (h < HPu) {
+        float l = l_run[h];
 #pragma unroll
-        for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            const int ch = 16 * mt + gid + 8 * half;
-            const float back = o_plain ? 1.f : (float)(1 << (24 - row_shift(mt, half)));
-            ocorr[h * kHeadDim + ch] += fmaf(O[mt][nt][2 * half] + O[mt][nt][2 * half + 1], back, cm_own[nt][(mt * 16) / GV]);
-          }
-        if (gid == 0) { part_base[h * kPartRow + 128] = m_own[nt]; part_base[h * kPartRow + 129] = l_own[nt]; }
+        for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+        if (lane == 0) { part_base[h * kPartRow + 128] = m_run[h]; part_base[h * kPartRow + 129] = l; }
+        reinterpret_cast<float4*>(part_base + h * kPartRow)[lane] = reinterpret_cast<const float4*>(ocorr + h * kHeadDim)[lane];
       }
     }
-    __syncwarp();
-#pragma unroll
-    for (int h = 0; h < HP; ++h)
-      if (h < HPu)
-        reinterpret_cast<float4*>(part_base + h * kPartRow)[lane] = reinterpret_cast<const float4*>(ocorr + h * kHeadDim)[lane];
     // The ticket is one acquire-release atomic at device scope: it publishes this warp's partial (the warp barrier
     // before it orders the other lanes' stores) and, for the warp that takes the last ticket, makes the others' visible.
     __syncwarp();
@@ -1272,6 +1299,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
       last = old == n_parts - 1;
     }
     last = __shfl_sync(0xffffffffu, last, 0);
+    __syncwarp();
     if (last) {
       const float* pb = a.partial + (size_t)u * a.max_parts * (HP * kPartRow);
       const size_t pstride = (size_t)HP * kPartRow;
@@ -1319,7 +1347,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
   // a warp that gave up still has copies in flight: let them land (bounded) before leaving
   if (!alive) {
     for (int i = 0; i < n_inflight; ++i) {
-      for (int k = 0; k < kSpinLimit && !mbar_try(&bar[c_stage], (uint32_t)c_par); ++k) {}
+      for (int k = 0; k < kDecodeSpinLimit && !mbar_try(&bar[c_stage], (uint32_t)c_par); ++k) {}
       if (++c_stage == NS) { c_stage = 0; c_par ^= 1; }
     }
   }
@@ -1328,10 +1356,10 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : (HEADS == 4 ? 8 : 6)) ge
 // ------------------------------------------------------------------ host side
 template <class Fn>
 static bool with_decode_kernel(int bits, int heads, int ngv, Fn fn) {
-  const int hp = heads == 1 ? 1 : (heads <= 4 ? 4 : 8);
+  const int hp = decode_heads_per_pass(heads);
 #define GEAR_DEC_CASE(B, N, V) \
   if (bits == B && hp == N && ngv == V) { fn(gear_decode_kernel<B, N, V>); return true; }
-#define GEAR_DEC_HEADS(B, V) GEAR_DEC_CASE(B, 1, V) GEAR_DEC_CASE(B, 4, V) GEAR_DEC_CASE(B, 8, V)
+#define GEAR_DEC_HEADS(B, V) GEAR_DEC_CASE(B, 1, V) GEAR_DEC_CASE(B, 4, V)
   GEAR_DEC_HEADS(2, 1) GEAR_DEC_HEADS(2, 2) GEAR_DEC_HEADS(2, 4) GEAR_DEC_HEADS(2, 8)
   GEAR_DEC_HEADS(4, 1) GEAR_DEC_HEADS(4, 2) GEAR_DEC_HEADS(4, 4) GEAR_DEC_HEADS(4, 8)
 #undef GEAR_DEC_HEADS

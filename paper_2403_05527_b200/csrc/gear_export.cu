@@ -12,31 +12,19 @@ __device__ __forceinline__ const unsigned char* record_of(const unsigned char* a
   return arena + sd.seg_base + (size_t)bh * sd.bh_stride + sd.bfac_bytes + (size_t)blk * sd.rec_bytes;
 }
 
-// inverse of code_coord_k / code_coord_v: where does the code of (token in slab, channel) sit?
+// the code of (token in block, channel): inverse of code_coord_k / code_coord_v
 __device__ __forceinline__ unsigned int load_code(const unsigned char* rec, const SegDesc& sd, int bits, int side,
-                                                  int slab, int ts, int ch) {
-  const int hpw = regs_per_word(bits);
-  int lane, q, u, e;
+                                                  int tib, int ch) {
+  int word, shift;
+  const unsigned int* words;
   if (side == 0) {
-    const int th = ts >> 3, gid = ts & 7, kc = ch >> 4, c16 = ch & 15;
-    const int hi = c16 >> 3, t = (c16 & 7) >> 1;
-    e = c16 & 1;
-    lane = gid * 4 + t;
-    const int kpw = hpw / 2, wpt = 16 / hpw;
-    q = th * wpt + kc / kpw;
-    u = 2 * (kc % kpw) + hi;
+    code_slot_k(bits, tib % kSlab, ch, word, shift);
+    words = reinterpret_cast<const unsigned int*>(rec + sd.off_kcodes + (tib / kSlab) * sd.slab_codes);
   } else {
-    const int mt = ch >> 4, c16 = ch & 15, gid = c16 & 7;
-    const int a = (c16 >> 3) | ((ts >> 3) << 1), t = (ts & 7) >> 1;
-    e = ts & 1;
-    lane = gid * 4 + t;
-    const int tpp = hpw / 2;
-    q = 2 * (mt / tpp) + (a >> 1);
-    u = 2 * (mt % tpp) + (a & 1);
+    code_slot_v(bits, tib % 32, ch, word, shift);
+    words = reinterpret_cast<const unsigned int*>(rec + sd.off_vcodes + (tib / 32) * 2 * sd.slab_codes);
   }
-  const unsigned int* words =
-      reinterpret_cast<const unsigned int*>(rec + (side == 0 ? sd.off_kcodes : sd.off_vcodes) + slab * sd.slab_codes);
-  return (words[word_index(lane, q)] >> (16 * e + bits * u)) & ((1u << bits) - 1u);
+  return (words[word] >> shift) & ((1u << bits) - 1u);
 }
 
 __global__ void export_kernel(const unsigned char* arena, SegDesc sd, CacheConst cc, int what, void* dst, size_t n) {
@@ -49,7 +37,7 @@ __global__ void export_kernel(const unsigned char* arena, SegDesc sd, CacheConst
       const int ch = i % d; const size_t r = i / d; const int tok = r % sd.n_c, bh = r / sd.n_c;
       const unsigned char* rec = record_of(arena, sd, bh, tok / T);
       const int tib = tok % T;
-      reinterpret_cast<unsigned char*>(dst)[i] = (unsigned char)load_code(rec, sd, cc.bits, side, tib / kSlab, tib % kSlab, ch);
+      reinterpret_cast<unsigned char*>(dst)[i] = (unsigned char)load_code(rec, sd, cc.bits, side, tib, ch);
       break;
     }
     case GEAR_EXP_K_SCALE: case GEAR_EXP_K_ZERO: {

@@ -25,7 +25,7 @@ cudaError_t launch_fp16_attn(const void* K, const void* V, const void* q, float*
                              int n_kv_heads, long long n, long long n_alloc, float scale, void* scratch,
                              size_t scratch_bytes, cudaStream_t st) {
   (void)scratch_bytes;
-  const int G = n_q_heads / n_kv_heads, hp = G <= 4 ? 4 : 8, passes = (G + hp - 1) / hp;
+  const int G = n_q_heads / n_kv_heads, passes = decode_passes(G);
   const size_t units = (size_t)batch * n_kv_heads * passes;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
@@ -102,13 +102,14 @@ extern "C" gear_status gear_fp16_decode_attn_static(const void* K, const void* V
   using namespace gear;
   if (!K || !V || !q || !out) return GEAR_ERR_ARG;
   if (batch < 1 || n_kv_heads < 1 || n_q_heads < 1 || n < 1 || n_alloc < n) return GEAR_ERR_ARG;
+  if (n_alloc > 0x7fffffffLL) return GEAR_ERR_ARG;                  // token counts travel as 32-bit integers
   if (head_dim != kHeadDim || n_q_heads % n_kv_heads) return GEAR_ERR_SHAPE;
   if (((uintptr_t)K | (uintptr_t)V | (uintptr_t)q | (uintptr_t)out) & 15) return GEAR_ERR_ALIGN;
   if ((long long)batch * n_q_heads > kStaticMaxQueryHeads) return GEAR_ERR_CAPACITY;
   cudaStream_t st = (cudaStream_t)stream;
   const int G = n_q_heads / n_kv_heads;
-  const int hp = G == 1 ? 1 : (G <= 4 ? 4 : 8);           // query heads per pass of the kernel that will run
-  const int passes = (G + hp - 1) / hp;
+  const int hp = decode_heads_per_pass(G);                // query heads per pass of the kernel that will run
+  const int passes = decode_passes(G);
   const size_t units = (size_t)batch * n_kv_heads * passes;
   // layout of the array: status word, tickets, then one partial slot per (unit, CTA touching it)
   const size_t header = 256 + ((units * 4 + 255) / 256) * 256;

@@ -63,7 +63,9 @@ cudaError_t launch_append(void* buf_k, void* buf_v, const void* k_new, const voi
 constexpr int kMaxStages = 4;
 constexpr int kPartRow = 132;     // floats per head of a partial result: 128 outputs, running max, denominator, padding to 16 bytes
 struct WarpSmem {      // byte offsets of a warp's (= a CTA's) shared-memory regions
-  int ring, sdp, sdc, qf, qs, frag, corr_k, ps, corr_v, ocorr, wl, misc, total;
+  int ring, sdc, qs, xr, ps, corr_k, corr_v, ocorr, wl, misc, total;
+  int fragv_stride;    // words per row of the value B-operand staging area
+  int fragp;           // byte offset of the fp16 probability fragments inside the xr region
 };
 struct DecodeArgs {
   const unsigned char* arena;
@@ -92,7 +94,9 @@ struct DecodeArgs {
   int stage_bytes;            // bytes of one ring stage
   int bregion;                // bytes at the front of a stage reserved for one B factor
   int max_T;                  // largest block length over the segments
-  int hpa;                    // query heads per pass that get shared-memory rows
+  int hpa;                    // query heads per pass (1 or 4)
+  int spin_limit;             // polls a consumer spends on one ring stage before it gives up
+  int test_dead_wait;         // test only: wait once on a barrier that nothing completes, with a short limit
   WarpSmem ws;
   float scale_log2;           // softmax scale * log2(e)
 };
@@ -102,6 +106,10 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
                  DecodeArgs* a);
 int decode_occupancy(int bits, int heads, int ngv, size_t smem);
 int static_shape_id(const SegDesc& s, const CacheConst& c);
+// query heads one pass of the kernel takes for G query heads per kv head, and the number of passes
+inline int decode_heads_per_pass(int G) { return G == 1 ? 1 : 4; }
+inline int decode_passes(int G) { return (G + decode_heads_per_pass(G) - 1) / decode_heads_per_pass(G); }
+constexpr int kDecodeSpinLimit = 4000000;
 
 // fp16-cache attention
 cudaError_t launch_fp16_attn(const void* K, const void* V, const void* q, float* out, int batch, int n_q_heads,

@@ -9,14 +9,15 @@
 // so that the decode kernel fetches a block (and, for block 0, the factors in
 // front of it) with one bulk copy.  A record holds, section by section:
 // key part (everything the score pass needs), then value part:
-//     header     16 B : fp32 max |x - zero| over the block's key / value outliers
+//     header     16 B : fp32 max |x - zero| over the block's key / value outliers, then the
+//                       largest key scale and the largest value scale of the block
 //     kscale     128 x (scale fp16, zero fp16)                 one pair per channel
 //     koval      128 x 2k_K fp16   outlier values, per channel, in-group index ascending
 //     koidx      128 x 2k_K u8     their token index inside the block
 //     kcodes     T/16 slabs x 16*128*b/8 bytes, in mma-fragment order (see code_coord_k)
 //     ak         T/16 slabs x [16 tokens][r_pad] fp16          rows of A_K
 //   -- off_vpart --
-//     vcodes     same size as kcodes (see code_coord_v)
+//     vcodes     ceil(T/32) chunks x 32*128*b/8 bytes (see code_coord_v; tokens past T hold code 0)
 //     av         T/16 slabs x [r_pad][16 tokens] fp16          rows of A_V, transposed per slab
 //     vscale     T x (d_H/g_V) x (scale fp16, zero fp16)
 //     voval      T x (d_H/g_V) x 2k_V fp16
@@ -76,6 +77,7 @@ __host__ __device__ inline int rank_pad(int r) {
 // Fill the size / offset fields of a descriptor from (T, n_c, rank, k_k) and the cache constants.
 __host__ __device__ inline void layout_segment(SegDesc& s, const CacheConst& c) {
   const int nslab = s.T / kSlab;
+  const int nchunk_v = (s.T + 31) / 32;
   s.r_pad = rank_pad(s.rank);
   s.nblk = s.n_c / s.T;
   s.slab_codes = kSlab * kHeadDim * c.bits / 8;
@@ -88,7 +90,7 @@ __host__ __device__ inline void layout_segment(SegDesc& s, const CacheConst& c) 
   s.off_kcodes = o;  o += nslab * s.slab_codes;
   s.off_ak = o;      o += round_up(nslab * s.slab_a, 16);
   s.off_vpart = o;
-  s.off_vcodes = o;  o += nslab * s.slab_codes;
+  s.off_vcodes = o;  o += nchunk_v * 2 * s.slab_codes;
   s.off_av = o;      o += round_up(nslab * s.slab_a, 16);
   s.off_vscale = o;  o += s.T * c.ngv * 4;
   s.off_voval = o;   o += round_up(s.T * c.ngv * 2 * c.k_v * 2, 16);
@@ -98,56 +100,57 @@ __host__ __device__ inline void layout_segment(SegDesc& s, const CacheConst& c) 
 }
 
 // ---------------------------------------------------------------------------
-// Where a code lives.  Per slab and side the codes are 32-bit words; lane `lane`
-// of a warp owns words q = 0 .. nq-1 (nq = 4 for 2-bit, 8 for 4-bit).  Word q of
-// lane `lane` sits at 32-bit index (q / 4) * 128 + lane * 4 + (q % 4) of the
-// slab, so one 128-bit shared-memory load per lane fetches four of them.
-// Inside a word, 16-bit half e (0 = low) holds, at bits [b*u, b*u + b), the code
-// that becomes half e of fragment register u of that word.
+// Where a code lives.  The decode kernel multiplies codes on the integer tensor
+// cores (mma.m16n8k32, u8 x s8): a byte of the A operand is one code, and a
+// b-bit field left where it sits in its byte is the code times 2^(b * field),
+// so a 32-bit word of packed codes becomes F = 8 / b fragment registers with one
+// AND each.  The power of two is absorbed where it is free: by the fixed-point
+// scale of the B operand (keys) or by the output row (values).
 //
-// Keys are the A operand (tokens x channels) of mma.m16n8k16: for channel
-// chunk kc (16 channels) lane (gid = lane/4, t = lane%4) needs
-//   a0 = {tok gid,   ch 2t, 2t+1}   a1 = {tok gid+8, ch 2t, 2t+1}
-//   a2 = {tok gid,   ch 2t+8, +9}   a3 = {tok gid+8, ch 2t+8, +9}
-// Values are the A operand (channels x tokens): for channel tile mt
-//   a0 = {ch gid,   tok 2t, 2t+1}   a1 = {ch gid+8, tok 2t, 2t+1}
-//   a2 = {ch gid,   tok 2t+8, +9}   a3 = {ch gid+8, tok 2t+8, +9}
-//
-// The decode kernel turns a word into fragment registers with one AND per
-// register: the masked field, left where it is, read as fp16 is the subnormal
-// code * 2^(b*u' - 24) (u' = u for the fields the 10-bit mantissa holds, after
-// one shift of the word for the others).  A power of two per register is
-// harmless only where the product can absorb it, which fixes who shares a field
-// position: for keys a0 and a1 (they meet the same B register: its q * scale is
-// pre-divided), for values a0 and a2 (they feed the same output row, which
-// carries the factor until the end).  Hence keys take (a0, a2) of a tile from
-// fields 2j, 2j+1 of one word and (a1, a3) from the same fields of a second
-// word; values take (a0, a1) from fields 2j, 2j+1 of one word and (a2, a3) from
-// a second word.
+// A "tuple" is four 32-bit words per lane -- the registers a0..a3 of one A
+// fragment (16 rows x 32 k) -- whose F fields are the same fragment of F
+// different tiles.  Lane (gid = lane / 4, t = lane % 4), word w = r + 2 * kh,
+// byte i, field j:
+//   keys   (rows = tokens of a 16-token slab, k = channels): tuple tau of the slab
+//          token   = gid + 8 r
+//          channel = 32 (F tau + j) + 16 kh + 4 t + i        field <-> 32-channel chunk
+//   values (rows = channels, k = tokens of a 32-token chunk): tuple tau of the chunk
+//          channel = 16 (F tau + j) + gid + 8 r              field <-> 16-channel tile
+//          token   = 16 kh + 4 t + i
+// The four words of a lane are one uint4: tuple number * 32 + lane in uint4 units
+// from the start of the slab (keys: 4 / F tuples per slab) or chunk (values:
+// 8 / F tuples per chunk).
 // ---------------------------------------------------------------------------
-__host__ __device__ inline int words_per_lane(int bits) { return bits == 2 ? 4 : 8; }
-__host__ __device__ inline int regs_per_word(int bits) { return bits == 2 ? 8 : 4; }   // half2 per word
+__host__ __device__ inline int fields_per_byte(int bits) { return 8 / bits; }
+__host__ __device__ inline int key_tuples_per_slab(int bits) { return 4 / fields_per_byte(bits); }
+__host__ __device__ inline int value_tuples_per_chunk(int bits) { return 8 / fields_per_byte(bits); }
 
-// key code at (lane, q, u, e) -> token in slab, channel
-__host__ __device__ inline void code_coord_k(int bits, int lane, int q, int u, int e, int& tok, int& ch) {
-  const int hpw = regs_per_word(bits);
-  const int wpt = 16 / hpw;                 // words per token half (2 or 4)
-  const int th = q / wpt, w = q % wpt;
-  const int kc = (hpw / 2) * w + (u >> 1);
-  const int hi = u & 1;                     // 0: a0/a1 columns, 1: a2/a3 columns (+8)
-  tok = 8 * th + (lane >> 2);
-  ch = 16 * kc + 8 * hi + 2 * (lane & 3) + e;
+// key code of (lane, tuple, word, byte, field) -> token in slab, channel
+__host__ __device__ inline void code_coord_k(int bits, int lane, int tau, int w, int i, int j, int& tok, int& ch) {
+  tok = (lane >> 2) + 8 * (w & 1);
+  ch = 32 * (fields_per_byte(bits) * tau + j) + 16 * (w >> 1) + 4 * (lane & 3) + i;
 }
-
-// value code at (lane, q, u, e) -> token in slab, channel
-__host__ __device__ inline void code_coord_v(int bits, int lane, int q, int u, int e, int& tok, int& ch) {
-  const int tpp = regs_per_word(bits) / 2;  // channel tiles per pair of words (4 or 2)
-  const int mt = tpp * (q >> 1) + (u >> 1);
-  const int a = (u & 1) + 2 * (q & 1);      // fragment register a0..a3
-  ch = 16 * mt + 8 * (a & 1) + (lane >> 2);
-  tok = 2 * (lane & 3) + 8 * (a >> 1) + e;
+// value code of (lane, tuple, word, byte, field) -> token in chunk, channel
+__host__ __device__ inline void code_coord_v(int bits, int lane, int tau, int w, int i, int j, int& tok, int& ch) {
+  ch = 16 * (fields_per_byte(bits) * tau + j) + (lane >> 2) + 8 * (w & 1);
+  tok = 16 * (w >> 1) + 4 * (lane & 3) + i;
 }
-
-__host__ __device__ inline int word_index(int lane, int q) { return (q >> 2) * 128 + lane * 4 + (q & 3); }
+// inverse maps: 32-bit word index inside the slab / chunk and bit position of the code
+__host__ __device__ inline void code_slot_k(int bits, int tok, int ch, int& word, int& shift) {
+  const int F = fields_per_byte(bits);
+  const int c32 = ch >> 5, c = ch & 31;
+  const int tau = c32 / F, j = c32 % F, kh = c >> 4, t = (c & 15) >> 2, i = c & 3;
+  const int gid = tok & 7, r = tok >> 3;
+  word = (tau * 32 + gid * 4 + t) * 4 + r + 2 * kh;
+  shift = 8 * i + bits * j;
+}
+__host__ __device__ inline void code_slot_v(int bits, int tok, int ch, int& word, int& shift) {
+  const int F = fields_per_byte(bits);
+  const int tile = ch >> 4, c = ch & 15;
+  const int tau = tile / F, j = tile % F, gid = c & 7, r = c >> 3;
+  const int kh = tok >> 4, t = (tok & 15) >> 2, i = tok & 3;
+  word = (tau * 32 + gid * 4 + t) * 4 + r + 2 * kh;
+  shift = 8 * i + bits * j;
+}
 
 }  // namespace gear
