@@ -349,6 +349,15 @@ extern "C" gear_status gear_append_buffer(gear_cache* c, const void* k_new, cons
 static gear_status plan_decode(gear_cache* c) {
   const int key = (int)c->segs.size();
   if (c->plan_key == key) return GEAR_OK;
+  // One-head passes: with four warps per scheduler the warps of a scheduler slow one another down by more than
+  // the fourth warp adds (measured: 3 warps finish 0.85 blocks per microsecond and scheduler, 4 warps 0.79), so
+  // long streams run with twelve resident warps.  Short streams (few blocks per warp) keep sixteen: there the
+  // fixed cost per warp and the granularity of the split weigh more.
+  int warps_cap = 0;
+  if (c->G == 1) {
+    const long long blocks = (long long)c->cc.BH * (c->n_blocks_c + (c->buf_len + 15) / 16);
+    if (blocks >= 24LL * 16 * c->sm_count) warps_cap = 12;
+  }
   int max_k = 0, max_v = 0, max_bfac = 0, max_T = 16;
   for (const SegDesc& s : c->segs) {
     if (s.off_vpart > max_k) max_k = s.off_vpart;
@@ -356,7 +365,8 @@ static gear_status plan_decode(gear_cache* c) {
     if (s.bfac_bytes > max_bfac) max_bfac = s.bfac_bytes;
     if (s.T > max_T) max_T = s.T;
   }
-  if (!decode_plan(c->cc.bits, c->G, c->cc.ngv, max_k, max_v, max_bfac, max_T, 227 * 1024, &c->plan)) return GEAR_ERR_SHAPE;
+  if (!decode_plan(c->cc.bits, c->G, c->cc.ngv, max_k, max_v, max_bfac, max_T, 227 * 1024, warps_cap, &c->plan))
+    return GEAR_ERR_SHAPE;
   const int occ = decode_occupancy(c->cc.bits, c->G, c->cc.ngv, (size_t)c->plan.ws.total);
   if (occ < 1) return GEAR_ERR_CUDA;
   c->plan_occ = occ;

@@ -140,13 +140,19 @@ __device__ __forceinline__ float warp_max(float x) {
 }
 __device__ __forceinline__ uint32_t warp_max_u32(uint32_t x) { return __reduce_max_sync(0xffffffffu, x); }
 __device__ __forceinline__ int float_exponent(float x) { return (int)((__float_as_uint(x) >> 23) & 0xFFu) - 127; }
+// 2^x for x <= 0 (scores minus a maximum): one instruction, relative error about 2^-22, flushes tiny results to zero
+__device__ __forceinline__ float exp2_fast(float x) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
 // 2^e for |e| <= 120
 __device__ __forceinline__ float pow2i(int e) { return __uint_as_float((uint32_t)(127 + e) << 23); }
 __device__ __forceinline__ int clamp60(int e) { return max(-60, min(60, e)); }
 
 // ------------------------------------------------------------------ shared memory plan (per warp)
 bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int max_bfac, int max_T, size_t smem_budget,
-                 DecodeArgs* a) {
+                 int warps_cap, DecodeArgs* a) {
   (void)bits;
   const int HP = decode_heads_per_pass(heads);
   const int frs = frag_row_words(HP);
@@ -182,13 +188,17 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
   w.fragp = fragv;
   // most resident warps (in steps of four: one per scheduler) whose ring still holds two stages; then as many
   // stages as fit
-  const int reg_limit = HP == 1 ? 16 : 8;
-  for (int warps = reg_limit; warps >= 1; warps -= (warps > 8 ? 4 : 1)) {
+  int reg_limit = HP == 1 ? 16 : 8;
+  const bool capped = warps_cap > 0 && warps_cap < reg_limit;
+  if (capped) reg_limit = warps_cap;
+  for (int warps = reg_limit; warps >= 1; warps -= (warps > 12 ? 4 : 1)) {
     const long long per = (long long)smem_budget / warps - 1024;     // the system reserves 1 KB per CTA
     long long ns = (per - w.ring) / stage;
     if (ns < 2) continue;
     if (ns > kMaxStages) ns = kMaxStages;
     w.total = w.ring + (int)ns * stage;
+    // a cap below what the registers allow is enforced through the shared-memory request
+    if (capped && warps == warps_cap) w.total = (int)(per & ~15LL);
     a->aligned = 0;
     a->nstage = (int)ns; a->stage_bytes = stage; a->bregion = bregion; a->max_T = max_T; a->hpa = HP; a->ws = w;
     a->spin_limit = kDecodeSpinLimit; a->test_dead_wait = 0;
@@ -408,7 +418,9 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
     const int blk_hi = min(NB, blk_lo + n_left);
     const int c_hi = min(blk_hi, a.n_blocks_c);          // end of the compressed blocks of this range
     const int bh = u / passes, pass = u - bh * passes;
-    const int HPu = HEADS == 1 ? 1 : min(HP, G - pass * HP);
+    const int HPu = HEADS == 1 ? 1 : min(HP, G - pass * HP);   // query heads this pass holds
+    constexpr int HC = HP;          // heads computed: a pass with fewer heads carries zero queries in the others, so that
+                                    // nothing in the block loop depends on the count; only the stores to global memory do
     const int hq0 = bh * G + pass * HP;                 // first query head of this pass
 
     // unit state
@@ -421,8 +433,9 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
     __syncwarp();
 #pragma unroll
     for (int h = 0; h < HP; ++h) {
-      if (h < HPu) {
-        const uint2 v = *reinterpret_cast<const uint2*>(a.q + (size_t)(hq0 + h) * kHeadDim + lane * 4);
+      {
+        const uint2 v = h < HPu ? *reinterpret_cast<const uint2*>(a.q + (size_t)(hq0 + h) * kHeadDim + lane * 4)
+                                : make_uint2(0u, 0u);
         *reinterpret_cast<uint2*>(qs + h * kHeadDim + lane * 4) = v;
         const __half2 q01 = u32_as_h2(v.x), q23 = u32_as_h2(v.y);
         const float4 qv = make_float4(__low2float(q01) * a.scale_log2, __high2float(q01) * a.scale_log2,
@@ -441,7 +454,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
     auto scale_ocorr = [&](const float (&alpha)[HP]) {
 #pragma unroll
       for (int h = 0; h < HP; ++h) {
-        if (h < HPu) {
+        if (h < HC) {
           float4* oc = reinterpret_cast<float4*>(ocorr + h * kHeadDim + lane * 4);
           float4 v = *oc;
           v.x *= alpha[h]; v.y *= alpha[h]; v.z *= alpha[h]; v.w *= alpha[h];
@@ -491,7 +504,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
             float v1 = fmaf((float)O[mt][nt][3], w1, (float)O[mt][nt][2]) * rs;
             v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
             v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
-            if (writer && hd < HPu) {
+            if (writer && hd < HC) {
               float* oc = ocorr + hd * kHeadDim + 16 * mt + gid;
               oc[0] = (oc[0] + v0) * al;
               oc[8] = (oc[8] + v1) * al;
@@ -562,7 +575,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
               }
               uint32_t b0 = 0u, b1 = 0u;
               const int h = gid >> 1;
-              if ((gid & 1) == 0 && h < HPu) {
+              if ((gid & 1) == 0 && h < HC) {
                 const __half* qrow = qs + h * kHeadDim + 16 * kc + 2 * t;
                 b0 = *reinterpret_cast<const uint32_t*>(qrow);
                 b1 = *reinterpret_cast<const uint32_t*>(qrow + 8);
@@ -611,7 +624,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
 #pragma unroll
             for (int h = 0; h < HP; ++h) {
               eK[h] = 0;
-              if (h < HPu) {
+              if (h < HC) {
                 float qv[4];
                 if (HP == 1) {
                   qv[0] = qreg[0]; qv[1] = qreg[1]; qv[2] = qreg[2]; qv[3] = qreg[3];
@@ -687,7 +700,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
                 const float d = val - zr4[j];
 #pragma unroll
                 for (int h = 0; h < HP; ++h)
-                  if (h < HPu) atomicAdd(&corr_k[h * maxT + idx], __float2int_rn(qS[h][j] * d));
+                  if (h < HC) atomicAdd(&corr_k[h * maxT + idx], __float2int_rn(qS[h][j] * d));
               };
               if (k2k == 2) {
                 const uint4 ov = reinterpret_cast<const uint4*>(kp + off_koval)[lane];
@@ -789,7 +802,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
                   f1 += d[2] + d[3];
                 }
                 const int hd = HP == 1 ? 0 : 2 * nt + (t >> 1);
-                if (writer && hd < HPu) {
+                if (writer && hd < HC) {
                   // raw sums only: the zero-point constant and the sparse term are added in the softmax pass
                   float* pr = ps + hd * maxT + tok0;
                   pr[0] = f0; pr[8] = f1;
@@ -814,7 +827,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
 #pragma unroll
           for (int h = 0; h < HP; ++h) {
             alpha[h] = 1.f; m_new[h] = 0.f;
-            if (h < HPu) {
+            if (h < HC) {
               const float Sik = pow2i(-sexp_k[h]);
               float mx = -INFINITY;
 #pragma unroll
@@ -897,8 +910,8 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
 #pragma unroll
             for (int h = 0; h < HP; ++h) {
               p[h][0] = p[h][1] = 0.f;
-              if (h < HPu) {
-                const float p0 = exp2f(sc[h][i].x - m_new[h]), p1 = exp2f(sc[h][i].y - m_new[h]);
+              if (h < HC) {
+                const float p0 = exp2_fast(sc[h][i].x - m_new[h]), p1 = exp2_fast(sc[h][i].y - m_new[h]);
                 p[h][0] = p0; p[h][1] = p1;
                 l[h] += p0 + p1;
                 if (r_pad > 0) {                              // fp16 fragments of p for the low-rank value term
@@ -929,7 +942,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
                   const float d = (val - __high2float(z[e2][g])) * Sx;
 #pragma unroll
                   for (int h = 0; h < HP; ++h)
-                    if (h < HPu) atomicAdd(&corr_v[h * kHeadDim + g * GV + idx], __float2int_rn(p[h][e2] * d));
+                    if (h < HC) atomicAdd(&corr_v[h * kHeadDim + g * GV + idx], __float2int_rn(p[h][e2] * d));
                 };
                 if (NGV * k2v == 4) {
                   const uint2 ov = reinterpret_cast<const uint2*>(vp + o_voval)[tk];
@@ -951,7 +964,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
           }
 #pragma unroll
           for (int h = 0; h < HP; ++h)
-            if (h < HPu) l_run[h] = fmaf(l_run[h], alpha[h], l[h]);
+            if (h < HC) l_run[h] = fmaf(l_run[h], alpha[h], l[h]);
           __syncwarp();
 
           // ---------------- values: out += sum_tok (p * scale) * code on the integer tensor cores, low rank on the side
@@ -1016,7 +1029,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
             const float Si = 1.0f / Sx;
 #pragma unroll
             for (int h = 0; h < HP; ++h) {
-              if (h < HPu) {
+              if (h < HC) {
                 int4* cv = reinterpret_cast<int4*>(corr_v + h * kHeadDim) + lane;
                 float4* oc = reinterpret_cast<float4*>(ocorr + h * kHeadDim) + lane;
                 const int4 v = *cv;
@@ -1066,7 +1079,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
               }
               float d[4];
               mma16816_z(d, aa, bu[0], bu[1]);
-              if (t < HPu) {                              // columns 2t, 2t + 1: high and low part of head t
+              if (t < HC) {                              // columns 2t, 2t + 1: high and low part of head t
                 float* oc = ocorr + t * kHeadDim + 16 * mt + gid;
                 oc[0] += d[0] + d[1];
                 oc[8] += d[2] + d[3];
@@ -1094,7 +1107,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
         __syncwarp();
 #pragma unroll
         for (int h = 0; h < HP; ++h) {
-          if (h < HPu) {
+          if (h < HC) {
             float add = 0.f;
 #pragma unroll
             for (int g = 0; g < NGV; ++g) {
@@ -1126,7 +1139,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
         const int kc = lane >> 2, reg = (lane >> 1) & 1, tA = 2 * (lane & 1);
 #pragma unroll
         for (int h = 0; h < HP; ++h) {
-          if (h < HPu) {
+          if (h < HC) {
             const uint2 qh = *reinterpret_cast<const uint2*>(qs + h * kHeadDim + lane * 4);
             const __half2 q01 = u32_as_h2(qh.x), q23 = u32_as_h2(qh.y);
             uint32_t hiA, loA, hiB, loB;
@@ -1166,7 +1179,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
             ldmatrix_x4(af, stK + ((lane & 7) + 8 * ((lane >> 3) & 1)) * kBufPitch + (16 * kc + 8 * (lane >> 4)) * 2);
             mma16816(acc[kc & 1], af, bq[kc][0], bq[kc][1]);
           }
-          if (t < HPu) {
+          if (t < HC) {
             float* pr = ps + t * maxT + gid;
             pr[0] = (acc[0][0] + acc[0][1]) + (acc[1][0] + acc[1][1]);
             pr[8] = (acc[0][2] + acc[0][3]) + (acc[1][2] + acc[1][3]);
@@ -1181,7 +1194,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
 #pragma unroll
           for (int h = 0; h < HP; ++h) {
             alpha[h] = 1.f;
-            if (h < HPu) {
+            if (h < HC) {
               float* row = ps + h * maxT;
               const float v = lane < valid_tokens ? row[lane & 15] : -INFINITY;
               const float mx = warp_max(v);
@@ -1226,7 +1239,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
           const int pr = lane, pi = pr & 7, tw = pi & 3, rg = pi >> 2;
 #pragma unroll
           for (int h = 0; h < HP; ++h) {
-            if (h < HPu) {
+            if (h < HC) {
               const float2 pp = *reinterpret_cast<const float2*>(ps + h * maxT + 2 * pr);
               const int col = 2 * (h & 3);
               uint32_t hi, lo;
@@ -1252,7 +1265,7 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
       if (!alive) break;
       // the tensor-core part of the buffer rows joins the fp32 copy
       __syncwarp();
-      if (t < HPu) {
+      if (t < HC) {
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt) {
           float* oc = ocorr + t * kHeadDim + 16 * mt + gid;

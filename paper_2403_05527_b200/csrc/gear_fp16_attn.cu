@@ -31,7 +31,7 @@ cudaError_t launch_fp16_attn(const void* K, const void* V, const void* q, float*
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   DecodeArgs a;
-  if (!decode_plan(2, G, 1, 0, 0, 0, 16, 227 * 1024, &a)) return cudaErrorInvalidConfiguration;
+  if (!decode_plan(2, G, 1, 0, 0, 0, 16, 227 * 1024, 0, &a)) return cudaErrorInvalidConfiguration;
   const int occ = decode_occupancy(2, G, 1, (size_t)a.ws.total);
   if (occ < 1) return cudaErrorInvalidConfiguration;
   long long grid = (long long)sms * occ;
@@ -128,7 +128,7 @@ extern "C" gear_status gear_fp16_decode_attn_static(const void* K, const void* V
     return GEAR_ERR_CUDA;
   }
   DecodeArgs a;
-  if (!decode_plan(2, G, 1, 0, 0, 0, 16, 227 * 1024, &a)) return GEAR_ERR_SHAPE;
+  if (!decode_plan(2, G, 1, 0, 0, 0, 16, 227 * 1024, 0, &a)) return GEAR_ERR_SHAPE;
   const int occ = decode_occupancy(2, G, 1, (size_t)a.ws.total);
   if (occ < 1) return GEAR_ERR_CUDA;
   long long grid = (long long)sms * occ;

@@ -102,8 +102,9 @@ struct DecodeArgs {
 };
 cudaError_t launch_decode(const DecodeArgs& a, int grid, cudaStream_t st);
 // Shared-memory plan of one warp; returns false if no stage count fits.  heads = G (query heads per kv head).
+// warps_cap > 0 limits the resident warps per SM below what registers and shared memory allow.
 bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int max_bfac, int max_T, size_t smem_budget,
-                 DecodeArgs* a);
+                 int warps_cap, DecodeArgs* a);
 int decode_occupancy(int bits, int heads, int ngv, size_t smem);
 int static_shape_id(const SegDesc& s, const CacheConst& c);
 // query heads one pass of the kernel takes for G query heads per kv head, and the number of passes
