@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the GEAR hot path on B200: decode steps over a compressed KV cache.
 
-Workload (configuration C2): one LLaMA-2-7B-shaped attention layer, batch 8, 32 heads, d_H = 128,
+Headline workload (configuration C2): one LLaMA-2-7B-shaped attention layer, batch 8, 32 heads, d_H = 128,
 context 4096, 2-bit codes with group 64, s = 2 % outliers, rank 4, streaming buffer n_b = 64.
 `--layers` independent layer caches are rotated so that the bytes touched between two uses of a cache
 exceed the 126 MB L2.
@@ -10,6 +10,9 @@ A step is one buffer cycle of every layer: n_b decode iterations, each = gear_ap
 fills the buffer compresses it: Filter, Quant, residual, power iteration, store) + gear_decode_attn over the
 whole compressed cache and the fp16 buffer.  `value` = batch / mean latency of one layer's decode iteration
 (append + its share of the flush + attention), summed over ranks.
+
+The line also carries, under `extra`, the decode and compress figures of the other configurations (LLaMA-2-13B
+shaped layer with 4- and 2-bit codes, Mistral-shaped grouped-query layer), each with its own roofline entry.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
 """
@@ -32,8 +35,11 @@ import numpy as np  # noqa: E402
 from paper_2403_05527_b200 import synth  # noqa: E402
 
 METRIC = "compressed-KV decode attn tokens/s"
-DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.015
 UNIT = "tokens/s"
+# dram__bytes_read + dram__bytes_write of one gear_decode_kernel launch per algorithmic byte, from an ncu capture of the
+# kernel on one C2 layer cache (137.5 MB of DRAM traffic for 134.3 MB); traffic grows in proportion to the cache
+DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {2: 1.0245}
+EXTRA_CONFIGS = (3, 32, 4)
 
 
 def workload_name(w, layers):
@@ -113,6 +119,32 @@ def oracle_unit_cycle(w, unit_seed, n_decode):
     return t_push / w.buffer_cap + t_attn / n_attn
 
 
+def _pool_unit(job):
+    """One oracle unit in a worker process, numeric libraries held to one thread."""
+    config_id, seed, n_decode = job
+    from threadpoolctl import threadpool_limits
+    with threadpool_limits(limits=1):
+        return oracle_unit_cycle(synth.WORKLOADS[config_id], seed, n_decode)
+
+
+def oracle_all_cores(w, units_per_core=8, max_workers=32):
+    """The oracle over independent (batch, head) units on every core the process may use: a pool of one-thread workers.
+    Returns (tokens/s of the whole layer, cores used, units timed, wall seconds)."""
+    import multiprocessing as mp
+    cores = min(len(os.sched_getaffinity(0)), max_workers)
+    jobs = [(w.config_id, 300 + i, 4) for i in range(cores * units_per_core)]
+    ctx = mp.get_context("spawn")
+    with ctx.Pool(cores) as pool:
+        pool.map(_pool_unit, jobs[:cores])            # start the workers (imports, page-in) outside the timed region
+        t0 = time.perf_counter()
+        per = pool.map(_pool_unit, jobs)
+        wall = time.perf_counter() - t0
+    units = w.batch * w.n_kv_heads
+    # `cores` units advance side by side: the layer's iteration takes units / cores rounds of the mean unit time
+    t_layer_iter = statistics.mean(per) * units / cores
+    return w.batch / t_layer_iter, cores, len(jobs), wall
+
+
 def run_reference(args, w):
     from threadpoolctl import threadpool_limits
     units = w.batch * w.n_kv_heads
@@ -128,8 +160,9 @@ def run_reference(args, w):
               f"4 of {w.buffer_cap} decode-attention calls timed; scaled by the unit count")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_layer_iter * w.buffer_cap * 1e3,
+            "extrapolated": "value and ms_per_step are the sampled unit's times scaled by the unit count",
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": workload_name(w, 1)},
+            "config": {"workload": workload_name(w, args.layers)},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -153,6 +186,46 @@ def whole_job_tokens_per_s(world, batch_per_rank, calls_per_rank, seconds):
     return world * batch_per_rank * calls_per_rank / seconds
 
 
+def rank_environment(rank, world, port):
+    """Environment of one spawned rank (the launcher below sets it before the rank's main runs)."""
+    return {"RANK": str(rank), "LOCAL_RANK": str(rank), "WORLD_SIZE": str(world), "MASTER_ADDR": "127.0.0.1",
+            "MASTER_PORT": str(port)}
+
+
+def _spawned_rank(rank, world, port, argv, main_name):
+    os.environ.update(rank_environment(rank, world, port))
+    sys.argv = list(argv)
+    globals()[main_name]()
+
+
+def spawn_ranks(world, argv, main_name="main", port=None):
+    """`python bench.py --gpus N` without a launcher: start N ranks of this file, one GPU each."""
+    import socket
+    import torch.multiprocessing as mp
+    if port is None:
+        with socket.socket() as s:
+            s.bind(("127.0.0.1", 0))
+            port = s.getsockname()[1]
+    mp.spawn(_spawned_rank, args=(world, port, argv, main_name), nprocs=world, join=True)
+
+
+def rank_probe():
+    """What a spawned rank sees, without a GPU: joins a gloo group from the environment the launcher set, reduces a
+    time with max_over_ranks and writes its view to the file named last on the command line (one line per rank)."""
+    import torch
+    import torch.distributed as dist
+    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        ms = max_over_ranks(10.0 + rank, dist, torch.device("cpu"))
+        with open(sys.argv[-1] + f".{rank}", "w") as f:
+            json.dump({"rank": rank, "world": world, "local_rank": int(os.environ["LOCAL_RANK"]), "ms": ms,
+                       "value": whole_job_tokens_per_s(world, 8, 10, ms * 1e-3)}, f)
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
 # --------------------------------------------------------------------------- our arm
 def device_kv(torch, w, dev, seed):
     """K, V fp16 [B, H, n, 128] drawn on the device with the distribution of synth.make_kv."""
@@ -167,25 +240,18 @@ def device_kv(torch, w, dev, seed):
     return k.contiguous(), v.contiguous()
 
 
-def run_ours(args, w):
-    import torch
-    from paper_2403_05527_b200 import binding as G
+def hbm_peak():
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        return float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the GEAR path has no CPU fallback")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    G.lib()
 
-    L, nb, B = args.layers, w.buffer_cap, w.batch
-    total_steps = args.warmup + args.steps + args.e2e_steps + 2
+def measure_config(torch, G, dev, w, layers, steps, warmup, rank, e2e_steps=0, dist=None, world=1, sampler_index=None):
+    """Build `layers` caches of workload w, run `warmup` + `steps` buffer cycles and time them.  Returns a dict of raw
+    measurements (CUDA events on the launching stream)."""
+    L, nb, B = layers, w.buffer_cap, w.batch
+    total_steps = warmup + steps + e2e_steps + 2
     max_tokens = w.n + total_steps * nb + nb
     cfg = G.make_config(B, w.n_q_heads, w.n_kv_heads, w.bits, w.group, w.s_pct, nb, w.rank, max_tokens,
                         rank_max=w.rank, power_iters=w.power_iters, seed=1234 + rank)
@@ -206,6 +272,7 @@ def run_ours(args, w):
         torch.cuda.synchronize()
         compress_ms.append(e0.elapsed_time(e1))
         del k, v
+    prefill_out_bytes = G.gear_cache_bytes(caches[0]).stored_total
     tok_shape = (B, w.n_kv_heads, 128)
     n_tok = 8
     g = torch.Generator(device=dev)
@@ -255,16 +322,16 @@ def run_ours(args, w):
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         step()
     barrier()
-    sampler = ClockSampler(local) if rank == 0 else None
+    sampler = ClockSampler(sampler_index) if sampler_index is not None else None
     launches0 = G.gear_kernel_launches()
     events, bytes_log, flush_events = [], [], []
     t_wall0 = time.time()
     s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s0.record()
-    for _ in range(args.steps):
+    for _ in range(steps):
         step(events, bytes_log, flush_events)
     s1.record()
     barrier()
@@ -278,83 +345,141 @@ def run_ours(args, w):
     if not all(torch.isfinite(o).all().item() for o in outs):
         raise SystemExit("non-finite attention output")
 
-    n_calls = args.steps * nb * L
-    value = whole_job_tokens_per_s(world, B, n_calls, ms_total * 1e-3)
     dec_ms = [a.elapsed_time(b) for a, b in events]       # one entry per group of L back-to-back decode launches
-    dec_launches = len(dec_ms) * L
-    dec_bytes = float(sum(bytes_log))
-    achieved = dec_bytes / (sum(dec_ms) * 1e-3) / 1e9
     flush_ms = [a.elapsed_time(b) for a, b in flush_events]
+    res = {"ms_total": ms_total, "n_calls": steps * nb * L, "dec_ms": sum(dec_ms), "dec_launches": len(dec_ms) * L,
+           "dec_bytes": float(sum(bytes_log)), "flush_ms": flush_ms, "compress_ms": compress_ms,
+           "prefill_out_bytes": prefill_out_bytes, "launches": int(launches), "clocks": clocks}
 
     # ---- end to end through the host-buffer entry points (pinned host memory, copies inside the timed region)
-    hk = torch.empty((n_tok, *tok_shape), dtype=torch.float16).pin_memory().copy_(new_k.cpu())
-    hv = torch.empty((n_tok, *tok_shape), dtype=torch.float16).pin_memory().copy_(new_v.cpu())
-    hq = torch.empty((B, w.n_q_heads, 128), dtype=torch.float16).pin_memory().copy_(q.cpu())
-    hout = torch.empty((B, w.n_q_heads, 128), dtype=torch.float32).pin_memory()
-    hk_np, hv_np, hq_np, hout_np = hk.numpy(), hv.numpy(), hq.numpy(), hout.numpy()
+    if e2e_steps > 0:
+        hk = torch.empty((n_tok, *tok_shape), dtype=torch.float16).pin_memory().copy_(new_k.cpu())
+        hv = torch.empty((n_tok, *tok_shape), dtype=torch.float16).pin_memory().copy_(new_v.cpu())
+        hq = torch.empty((B, w.n_q_heads, 128), dtype=torch.float16).pin_memory().copy_(q.cpu())
+        hout = torch.empty((B, w.n_q_heads, 128), dtype=torch.float32).pin_memory()
+        hk_np, hv_np, hq_np, hout_np = hk.numpy(), hv.numpy(), hq.numpy(), hout.numpy()
 
-    def step_e2e():
-        for i in range(nb):
-            for c in caches:
-                G.gear_append_buffer_host(c, hk_np[i % n_tok], hv_np[i % n_tok])
-                G.gear_decode_attn_host(c, hq_np, hout_np)
-    if args.e2e_steps > 0:
+        def step_e2e():
+            for i in range(nb):
+                for c in caches:
+                    G.gear_append_buffer_host(c, hk_np[i % n_tok], hv_np[i % n_tok])
+                    G.gear_decode_attn_host(c, hq_np, hout_np)
         step_e2e()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(args.e2e_steps):
-        step_e2e()
-    barrier()
-    e2e_s = max_over_ranks(max(time.perf_counter() - t0, 1e-9), dist, dev)
-    e2e_value = whole_job_tokens_per_s(world, B, args.e2e_steps * nb * L, e2e_s)
-    h2d = nb * L * (2 * hk_np[0].nbytes + hq_np.nbytes)
-    d2h = nb * L * hout_np.nbytes
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            step_e2e()
+        barrier()
+        e2e_s = max_over_ranks(max(time.perf_counter() - t0, 1e-9), dist, dev)
+        res["e2e_value"] = whole_job_tokens_per_s(world, B, e2e_steps * nb * L, e2e_s)
+        res["h2d"] = nb * L * (2 * hk_np[0].nbytes + hq_np.nbytes)
+        res["d2h"] = nb * L * hout_np.nbytes
+    for c in caches:
+        G.gear_free(c)
+    G.gear_release_workspace()
+    torch.cuda.empty_cache()
+    return res
+
+
+def decode_roofline(w, res, peak, peak_src):
+    achieved = res["dec_bytes"] / (res["dec_ms"] * 1e-3) / 1e9
+    per_launch = res["dec_bytes"] / res["dec_launches"]
+    ratio = DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE.get(w.config_id)
+    return {"bound": "hbm", "kernel": "gear_decode_kernel", "achieved": achieved, "peak": peak,
+            "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak, "frac_of_8000_nominal": achieved / 8000.0,
+            "traffic": ratio * per_launch if ratio else None,
+            "traffic_source": "ncu capture of one launch on one layer cache, scaled by the algorithmic bytes" if ratio else None,
+            "algorithmic_bytes_per_launch": per_launch, "us_per_launch": 1e3 * res["dec_ms"] / res["dec_launches"]}
+
+
+def compress_roofline(w, res, peak):
+    """Prefill: fp16 K and V in, the packed segment out.  Flush: one full buffer of every (batch, head) in, its segment
+    out.  Both against the HBM peak: what they must move is small next to what the kernels do per byte."""
+    B, H, nb = w.batch, w.n_kv_heads, w.buffer_cap
+    in_bytes = 2 * B * H * w.n * 128 * 2
+    pre_ms = statistics.median(res["compress_ms"])
+    pre_alg = in_bytes + res["prefill_out_bytes"]
+    out = {"prefill": {"bound": "hbm", "kernel": "quant_pack_kernel + pi_pass_kernel (dominant)", "ms": pre_ms,
+                       "input_gbs": in_bytes / (pre_ms * 1e-3) / 1e9, "algorithmic_bytes": pre_alg,
+                       "achieved": pre_alg / (pre_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                       "frac": pre_alg / (pre_ms * 1e-3) / 1e9 / peak}}
+    if res["flush_ms"]:
+        f_ms = statistics.median(res["flush_ms"])
+        f_in = 2 * B * H * nb * 128 * 2
+        f_alg = f_in + res["prefill_out_bytes"] * nb // w.n
+        out["flush"] = {"bound": "latency (one launch, less than one wave of tiles)", "kernel": "compress_tile_kernel",
+                        "us": 1e3 * f_ms, "input_gbs": f_in / (f_ms * 1e-3) / 1e9, "algorithmic_bytes": f_alg,
+                        "achieved": f_alg / (f_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                        "frac": f_alg / (f_ms * 1e-3) / 1e9 / peak}
+    return out
+
+
+def run_ours(args, w):
+    import torch
+    from paper_2403_05527_b200 import binding as G
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the GEAR path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    G.lib()
+
+    res = measure_config(torch, G, dev, w, args.layers, args.steps, args.warmup, rank, args.e2e_steps, dist, world,
+                         sampler_index=local if rank == 0 else None)
+    value = whole_job_tokens_per_s(world, w.batch, res["n_calls"], res["ms_total"] * 1e-3)
 
     line = None
     if rank == 0:
-        peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-        if os.path.exists(peaks_path):
-            peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
-        else:
-            peak, peak_src = 6650.0, "fallback"
-        # dram__bytes_read + dram__bytes_write of gear_decode_kernel<2,1,2> per algorithmic byte, from the ncu capture
-        # summarised in profiles/gear_decode_kernel_C2.md (one layer cache; traffic grows in proportion to the cache)
-        traffic = DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE * dec_bytes / dec_launches if w.config_id == 2 else None
-        in_bytes = 2 * B * w.n_kv_heads * w.n * 128 * 2
+        peak, peak_src = hbm_peak()
+        roof = decode_roofline(w, res, peak, peak_src)
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                "warmup": args.warmup, "ms_per_step": res["ms_total"] / args.steps, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "s32 (codes x fixed-point query on the integer tensor cores), f32 elsewhere",
                 "data": "synthetic",
-                "config": {"workload": workload_name(w, L), "batch_per_gpu": B, "layers_rotated": L,
-                           "l2": "rotating caches: %.0f MB touched between reuses" % (dec_bytes / dec_launches * L / 1e6)},
-                "roofline": {"bound": "hbm", "kernel": "gear_decode_kernel", "achieved": achieved, "peak": peak,
-                             "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                             "frac_of_8000_nominal": achieved / 8000.0, "traffic": traffic,
-                             "algorithmic_bytes_per_launch": dec_bytes / dec_launches,
-                             "us_per_launch": 1e3 * sum(dec_ms) / dec_launches},
-                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-                "gpu_launches": int(launches),
-                "clocks": clocks,
-                "compress": {"prefill_gbs": in_bytes / (statistics.median(compress_ms) * 1e-3) / 1e9,
-                             "prefill_ms": statistics.median(compress_ms),
-                             "flush_us": 1e3 * statistics.median(flush_ms) if flush_ms else None,
-                             "flush_gbs": (2 * B * w.n_kv_heads * nb * 128 * 2) / (statistics.median(flush_ms) * 1e-3) / 1e9
-                             if flush_ms else None},
-                "decode_attn_tokens_per_s_kernel_only": B / (1e-3 * sum(dec_ms) / dec_launches)}
-        if not args.no_cpu and world == 1:
-            from threadpoolctl import threadpool_limits
-            with threadpool_limits(limits=1):
-                t0 = time.perf_counter()
-                per = [oracle_unit_cycle(w, 100 + s, n_decode=8) for s in range(args.cpu_units)]
-                spent = time.perf_counter() - t0
-            units = B * w.n_kv_heads
-            line["cpu_baseline"] = {"value": B / (statistics.mean(per) * units), "unit": UNIT, "cores": 1,
-                                    "kind": "oracle",
-                                    "sample": f"{args.cpu_units} of {units} (batch, head) units, one buffer cycle each "
-                                              f"(64 pushes incl. the flush, 8 decode-attention calls timed), scaled by "
-                                              f"the unit count; {spent:.1f} s of CPU work incl. the untimed prefill compress"}
-    for c in caches:
-        G.gear_free(c)
+                "config": {"workload": workload_name(w, args.layers), "batch_per_gpu": w.batch, "layers_rotated": args.layers,
+                           "l2": "rotating caches: %.0f MB touched between reuses" % (roof["algorithmic_bytes_per_launch"] * args.layers / 1e6)},
+                "roofline": roof,
+                "e2e": {"value": res.get("e2e_value"), "unit": UNIT, "h2d_bytes_per_step": res.get("h2d"),
+                        "d2h_bytes_per_step": res.get("d2h")},
+                "gpu_launches": res["launches"],
+                "clocks": res["clocks"],
+                "compress": compress_roofline(w, res, peak),
+                "decode_attn_tokens_per_s_kernel_only": w.batch / (1e-3 * res["dec_ms"] / res["dec_launches"])}
+    # ---- the other configurations, a few steps each (rank 0's GPU at N = 1 only: they are context, not the headline)
+    if rank == 0 and world == 1 and not args.no_extra and w.config_id == 2:
+        extra = {}
+        for cid in EXTRA_CONFIGS:
+            we = synth.WORKLOADS[cid]
+            r = measure_config(torch, G, dev, we, 2, 1, 3, rank)
+            extra[f"C{cid}"] = {"workload": workload_name(we, 2), "steps": 1, "warmup": 3,
+                                "decode_attn_tokens_per_s_kernel_only": we.batch / (1e-3 * r["dec_ms"] / r["dec_launches"]),
+                                "roofline": decode_roofline(we, r, peak, peak_src),
+                                "compress": compress_roofline(we, r, peak)}
+        line["extra"] = extra
+    if rank == 0 and not args.no_cpu and world == 1:
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            t0 = time.perf_counter()
+            per = [oracle_unit_cycle(w, 100 + s, n_decode=8) for s in range(args.cpu_units)]
+            spent = time.perf_counter() - t0
+        units = w.batch * w.n_kv_heads
+        line["cpu_baseline"] = {"value": w.batch / (statistics.mean(per) * units), "unit": UNIT, "cores": 1,
+                                "kind": "oracle",
+                                "sample": f"{args.cpu_units} of {units} (batch, head) units, one buffer cycle each "
+                                          f"({w.buffer_cap} pushes incl. the flush, 8 decode-attention calls timed), scaled by "
+                                          f"the unit count; {spent:.1f} s of CPU work incl. the untimed prefill compress"}
+        v_all, cores, n_units, wall = oracle_all_cores(w)
+        line["cpu_baseline_all_cores"] = {"value": v_all, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                          "sample": f"{n_units} of {units} units over a pool of {cores} one-thread workers "
+                                                    f"(4 decode-attention calls timed per unit), scaled by the unit count; "
+                                                    f"{wall:.1f} s wall"}
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
@@ -373,11 +498,15 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-units", type=int, default=128)
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-extra", action="store_true")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.config]
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) == 0:
             run_reference(args, w)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(args.gpus, sys.argv)                  # no launcher: start the ranks here, one GPU each
         return
     run_ours(args, w)
 

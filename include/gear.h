@@ -21,6 +21,9 @@
  *  - Not thread-safe per cache: calls on one cache must be issued from one
  *    thread at a time and on one stream (or streams ordered by the caller).
  *  - Inputs are assumed finite; NaN / Inf give unspecified results, no error.
+ *  - Range of the decode kernel's fixed-point operands: per block it scales q * scale_K (per
+ *    channel) and p * scale_V (per token and group) by a power of two taken from their largest
+ *    magnitude, clamped to 2^+-60.  Every finite fp16 input stays inside that range.
  */
 #ifndef GEAR_H_
 #define GEAR_H_
@@ -50,6 +53,13 @@ enum {
   GEAR_FLAG_KEEP_FP32_FACTORS = 1u  /* also keep A, B in fp32 (before the fp16 rounding) for gear_export */
 };
 
+/* Device memory of the caches.  By default gear_create uses cudaMalloc / cudaFree.  A caller that owns the
+ * device heap installs its own pair here (process-wide; NULL, NULL restores the default): alloc returns a
+ * device pointer aligned to 256 bytes or NULL, which gear_create reports as GEAR_ERR_ALLOC after handing back
+ * what it had taken.  A cache frees through the pair it was created with. */
+typedef void* (*gear_alloc_fn)(size_t bytes, void* ctx);
+typedef void (*gear_free_fn)(void* ptr, void* ctx);
+
 /* Hyper-parameters in the paper's notation (Section 2 and 3; Algorithm 1, 2). */
 typedef struct gear_config {
   int32_t batch;        /* sequences in the batch                                              */
@@ -74,6 +84,8 @@ typedef struct gear_config {
 } gear_config;
 
 typedef struct gear_cache gear_cache;   /* opaque */
+
+gear_status gear_set_allocator(gear_alloc_fn alloc_fn, gear_free_fn free_fn, void* ctx);
 
 /* Create an empty cache (no segment, empty buffer) on the current device.
  * Allocates everything the cache will ever use.  *cache must be NULL. */
@@ -233,9 +245,19 @@ typedef struct gear_bytes {
 } gear_bytes;
 gear_status gear_cache_bytes(const gear_cache* cache, gear_bytes* out);
 
-/* Read (and clear) the device status word: 0, or a GEAR_ERR_* a kernel recorded
- * (a bounded wait that gave up, a range check that failed).  Synchronises. */
+/* Read (and clear) the device status word: 0, or the GEAR_ERR_* a kernel recorded (GEAR_ERR_TIMEOUT: a bounded
+ * wait on a copy gave up; the outputs of the calls since the last read are then undefined).  Synchronises the
+ * device.  When the word was set, the call also resets the cache's merge counters, so that the next
+ * gear_decode_attn on the cache starts clean. */
 gear_status gear_last_device_status(gear_cache* cache, int32_t* code);
+/* The same word for gear_fp16_decode_attn (it lives at the start of the caller's scratch buffer) and for
+ * gear_fp16_decode_attn_static (it lives in the library's array on the current device). */
+gear_status gear_fp16_attn_status(void* scratch, int32_t* code);
+gear_status gear_fp16_attn_static_status(int32_t* code);
+/* Test only: while `on`, every decode call on the cache first waits, with a limit of a few dozen polls, on a
+ * barrier that nothing completes, so that the give-up path runs: the kernel drains its copies, records
+ * GEAR_ERR_TIMEOUT and returns.  Nothing faults, traps or hangs. */
+gear_status gear_test_dead_wait(gear_cache* cache, int32_t on);
 
 const char* gear_strerror(gear_status s);
 

@@ -74,6 +74,10 @@ _SIGNATURES = {
     "gear_segment_info_get": (C.c_int32, [C.c_void_p, C.c_int32, C.POINTER(GearSegmentInfo)]),
     "gear_cache_bytes": (C.c_int32, [C.c_void_p, C.POINTER(GearBytes)]),
     "gear_last_device_status": (C.c_int32, [C.c_void_p, C.POINTER(C.c_int32)]),
+    "gear_fp16_attn_status": (C.c_int32, [C.c_void_p, C.POINTER(C.c_int32)]),
+    "gear_fp16_attn_static_status": (C.c_int32, [C.POINTER(C.c_int32)]),
+    "gear_test_dead_wait": (C.c_int32, [C.c_void_p, C.c_int32]),
+    "gear_set_allocator": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "gear_strerror": (C.c_char_p, [C.c_int32]),
     "gear_kernel_launches": (C.c_uint64, []),
 }
@@ -215,6 +219,34 @@ def gear_last_device_status(cache) -> int:
     code = C.c_int32()
     _check(lib().gear_last_device_status(cache, C.byref(code)), "gear_last_device_status")
     return code.value
+
+
+def gear_fp16_attn_status(scratch) -> int:
+    code = C.c_int32()
+    _check(lib().gear_fp16_attn_status(_ptr(scratch), C.byref(code)), "gear_fp16_attn_status")
+    return code.value
+
+
+def gear_fp16_attn_static_status() -> int:
+    code = C.c_int32()
+    _check(lib().gear_fp16_attn_static_status(C.byref(code)), "gear_fp16_attn_static_status")
+    return code.value
+
+
+def gear_test_dead_wait(cache, on: bool) -> None:
+    _check(lib().gear_test_dead_wait(cache, 1 if on else 0), "gear_test_dead_wait")
+
+
+ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_size_t, C.c_void_p)
+FREE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p)
+
+
+def gear_set_allocator(alloc_fn, free_fn) -> None:
+    """Install a device allocator pair (ctypes callbacks of type ALLOC_FN / FREE_FN, kept alive by the caller), or
+    None, None for cudaMalloc / cudaFree."""
+    a = C.cast(alloc_fn, C.c_void_p) if alloc_fn is not None else None
+    f = C.cast(free_fn, C.c_void_p) if free_fn is not None else None
+    _check(lib().gear_set_allocator(a, f, None), "gear_set_allocator")
 
 
 def gear_kernel_launches() -> int:

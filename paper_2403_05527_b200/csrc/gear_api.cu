@@ -54,7 +54,35 @@ extern "C" gear_status gear_release_workspace(void) {
   return GEAR_OK;
 }
 
+// Device memory of the caches comes from cudaMalloc unless the caller installed a pair of its own (gear_set_allocator).
+static std::mutex g_alloc_mutex;
+static gear_alloc_fn g_alloc = nullptr;
+static gear_free_fn g_free = nullptr;
+static void* g_alloc_ctx = nullptr;
+
+extern "C" gear_status gear_set_allocator(gear_alloc_fn alloc_fn, gear_free_fn free_fn, void* ctx) {
+  if ((alloc_fn == nullptr) != (free_fn == nullptr)) return GEAR_ERR_ARG;
+  std::lock_guard<std::mutex> lock(g_alloc_mutex);
+  g_alloc = alloc_fn; g_free = free_fn; g_alloc_ctx = ctx;
+  return GEAR_OK;
+}
+
+struct DeviceAllocator {       // the pair a cache was created with (it frees through the same pair)
+  gear_alloc_fn alloc; gear_free_fn free; void* ctx;
+  void* get(size_t bytes) const {
+    if (alloc) return alloc(bytes, ctx);
+    void* p = nullptr;
+    if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return p;
+  }
+  void put(void* p) const {
+    if (!p) return;
+    if (free) free(p, ctx); else cudaFree(p);
+  }
+};
+
 struct gear_cache {
+  DeviceAllocator mem;
   gear_config cfg;
   CacheConst cc;
   int device;
@@ -84,6 +112,7 @@ struct gear_cache {
   // cached launch plan of the decode kernel (depends on the segments' shapes)
   int plan_key, plan_occ;
   DecodeArgs plan;
+  int test_dead_wait;            // gear_test_dead_wait: the next decode calls wait on a barrier nothing completes
 };
 
 static int outlier_count(float s_pct, int len) {
@@ -129,9 +158,10 @@ static SegDesc shape_segment(const gear_cache* c, int n_c, int rank) {
 
 extern "C" void gear_free(gear_cache* c) {
   if (!c) return;
-  cudaFree(c->arena); cudaFree(c->dbg); cudaFree(c->table_dev); cudaFree(c->blk2seg); cudaFree(c->buf_k); cudaFree(c->buf_v);
-  cudaFree(c->flush_ws); cudaFree(c->partial); cudaFree(c->tickets); cudaFree(c->status);
-  cudaFree(c->stage_k); cudaFree(c->stage_q); cudaFree(c->stage_out); cudaFree(c->stage_b0);
+  const DeviceAllocator& m = c->mem;
+  m.put(c->arena); m.put(c->dbg); m.put(c->table_dev); m.put(c->blk2seg); m.put(c->buf_k); m.put(c->buf_v);
+  m.put(c->flush_ws); m.put(c->partial); m.put(c->tickets); m.put(c->status);
+  m.put(c->stage_k); m.put(c->stage_q); m.put(c->stage_out); m.put(c->stage_b0);
   for (int i = 0; i < gear_cache::kHostSlots; ++i) {
     if (c->host_ring[i]) cudaFreeHost(c->host_ring[i]);
     if (c->host_ev[i]) cudaEventDestroy(c->host_ev[i]);
@@ -141,8 +171,8 @@ extern "C" void gear_free(gear_cache* c) {
 
 #define GEAR_TRY_ALLOC(ptr, bytes)                                                   \
   do {                                                                               \
-    if (cudaMalloc((void**)&(ptr), (bytes)) != cudaSuccess) {                        \
-      cudaGetLastError();                                                            \
+    *reinterpret_cast<void**>(&(ptr)) = c->mem.get(bytes);                           \
+    if ((ptr) == nullptr) {                                                          \
       gear_free(c);                                                                  \
       return GEAR_ERR_ALLOC;                                                         \
     }                                                                                \
@@ -155,6 +185,11 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   gear_cache* c = new (std::nothrow) gear_cache();
   if (!c) return GEAR_ERR_ALLOC;
   c->cfg = *cfg;
+  {
+    std::lock_guard<std::mutex> lock(g_alloc_mutex);
+    c->mem.alloc = g_alloc; c->mem.free = g_free; c->mem.ctx = g_alloc_ctx;
+  }
+  c->test_dead_wait = 0;
   c->arena = nullptr; c->dbg = nullptr; c->table_dev = nullptr; c->blk2seg = nullptr; c->buf_k = c->buf_v = nullptr; c->flush_ws = nullptr;
   c->partial = nullptr; c->tickets = nullptr; c->status = nullptr;
   c->stage_k = c->stage_v = c->stage_q = nullptr; c->stage_out = nullptr; c->stage_b0 = nullptr;
@@ -388,6 +423,7 @@ extern "C" gear_status gear_decode_attn(gear_cache* c, const void* q, float* out
   a.n_kv_heads = c->cfg.n_kv_heads; a.group_heads = c->G; a.max_parts = c->max_parts;
   const float sc = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)kHeadDim);
   a.scale_log2 = sc * 1.4426950408889634f;
+  a.test_dead_wait = c->test_dead_wait;
   // one warp per CTA; never more warps than blocks of work
   const int passes = decode_passes(c->G);
   const long long work = (long long)c->cc.BH * passes * (c->n_blocks_c + (c->buf_len + 15) / 16);
@@ -615,6 +651,29 @@ extern "C" gear_status gear_last_device_status(gear_cache* c, int32_t* code) {
   int v = 0;
   if (cudaDeviceSynchronize() != cudaSuccess || cudaMemcpy(&v, c->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
       cudaMemset(c->status, 0, 4) != cudaSuccess) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  if (v != 0) {
+    // a warp that gave up left without taking its tickets: start the next call from a clean count
+    const size_t units = (size_t)c->cc.BH * decode_passes(c->G);
+    if (cudaMemset(c->tickets, 0, units * 4) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
+  }
+  *code = v;
+  return GEAR_OK;
+}
+
+extern "C" gear_status gear_test_dead_wait(gear_cache* c, int32_t on) {
+  if (!c) return GEAR_ERR_ARG;
+  c->test_dead_wait = on ? 1 : 0;
+  return GEAR_OK;
+}
+
+extern "C" gear_status gear_fp16_attn_status(void* scratch, int32_t* code) {
+  if (!scratch || !code) return GEAR_ERR_ARG;
+  int v = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess || cudaMemcpy(&v, scratch, 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemset(scratch, 0, 4) != cudaSuccess) {
     cudaGetLastError();
     return GEAR_ERR_CUDA;
   }

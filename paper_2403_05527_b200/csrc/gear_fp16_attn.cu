@@ -156,3 +156,9 @@ extern "C" gear_status gear_fp16_decode_attn_static(const void* K, const void* V
   return GEAR_OK;
 }
 
+extern "C" gear_status gear_fp16_attn_static_status(int32_t* code) {
+  if (!code) return GEAR_ERR_ARG;
+  void* scratch = nullptr;
+  if (static_scratch_address(&scratch) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
+  return gear_fp16_attn_status(scratch, code);
+}

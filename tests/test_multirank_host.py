@@ -60,3 +60,20 @@ def test_reference_arm_runs_on_rank_zero_only(monkeypatch, capsys):
     monkeypatch.setattr(sys, "argv", ["bench.py", "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0"])
     bench.main()
     assert capsys.readouterr().out == ""                   # other ranks exit without work or output
+
+
+def test_launcher_starts_the_ranks_itself_when_no_launcher_did(tmp_path):
+    """`bench.py --gpus N` without torchrun: the ranks are spawned by bench.py, each with its own RANK / LOCAL_RANK /
+    WORLD_SIZE and a common rendezvous on 127.0.0.1.  Checked with two CPU ranks on gloo."""
+    import json
+    sys.path.insert(0, ROOT)
+    import bench
+    env = bench.rank_environment(1, 2, 12345)
+    assert env == {"RANK": "1", "LOCAL_RANK": "1", "WORLD_SIZE": "2", "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": "12345"}
+    out = str(tmp_path / "probe")
+    bench.spawn_ranks(2, ["bench.py", "--gpus", "2", out], main_name="rank_probe", port=_free_port())
+    views = [json.load(open(f"{out}.{r}")) for r in (0, 1)]
+    for r, v in enumerate(views):
+        assert (v["rank"], v["local_rank"], v["world"]) == (r, r, 2)
+        assert v["ms"] == pytest.approx(11.0)                       # every rank sees the slowest rank's time
+        assert v["value"] == pytest.approx(2 * 8 * 10 / 11e-3)
