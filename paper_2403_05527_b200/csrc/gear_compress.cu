@@ -613,23 +613,33 @@ __global__ void __launch_bounds__(256) pi_gram2_kernel(PiArgs p, int identity) {
     for (int q = 0; q < kMaxRank; ++q) a0[q] = (row < row1 && q < r) ? A0[(size_t)row * kMaxRank + q] : 0.f;
 #pragma unroll
     for (int c = 0; c < kMaxRank; ++c) {
-      float s = 0.f;
+      if (c < r) {                               // uniform over the block: only the rank's columns exist
+        float s = 0.f;
 #pragma unroll
-      for (int q = 0; q < kMaxRank; ++q) s = fmaf(a0[q], Wm[q * kMaxRank + c], s);
-      rows[warp][lane][c] = s;
+        for (int q = 0; q < kMaxRank; ++q) s = fmaf(a0[q], Wm[q * kMaxRank + c], s);
+        rows[warp][lane][c] = s;
+      }
     }
     __syncwarp();
+    // entry (u, v) of the Gram matrix, u, v < r: pair number i * 32 + lane, so that a small rank takes one round
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const int pr = lane * 8 + i, u = pr / kMaxRank, v = pr % kMaxRank;
-      float s = g[i];
-      for (int t = 0; t < 32; ++t) s = fmaf(rows[warp][t][u], rows[warp][t][v], s);
-      g[i] = s;
+      if (i * 32 < r * r) {
+        const int pr = i * 32 + lane, u = min(pr / r, kMaxRank - 1), v = pr % r;
+        float s = g[i];
+        for (int t = 0; t < 32; ++t) s = fmaf(rows[warp][t][u], rows[warp][t][v], s);
+        g[i] = s;
+      }
     }
     __syncwarp();
   }
+  for (int i = threadIdx.x; i < 8 * 256; i += blockDim.x) (&red[0][0])[i] = 0.f;
+  __syncthreads();
 #pragma unroll
-  for (int i = 0; i < 8; ++i) red[warp][lane * 8 + i] = g[i];
+  for (int i = 0; i < 8; ++i) {
+    const int pr = i * 32 + lane;
+    if (pr < r * r) red[warp][(pr / r) * kMaxRank + pr % r] = g[i];
+  }
   __syncthreads();
   for (int i = threadIdx.x; i < 256; i += blockDim.x) {
     float s = 0.f;
