@@ -80,7 +80,7 @@ typedef struct gear_config {
   int64_t max_tokens;   /* capacity in compressed tokens per sequence (arena is sized from it)   */
   uint64_t seed;        /* start vectors when the caller passes no B0                           */
   uint32_t flags;       /* GEAR_FLAG_*                                                           */
-  uint32_t reserved;
+  uint32_t max_queries; /* most query rows per head a gear_decode_attn_multi call will bring (0 or 1: one) */
 } gear_config;
 
 typedef struct gear_cache gear_cache;   /* opaque */
@@ -127,6 +127,15 @@ gear_status gear_append_buffer(gear_cache* cache, const void* k_new, const void*
  * The cache must hold at least one token (GEAR_ERR_STATE otherwise). */
 gear_status gear_decode_attn(gear_cache* cache, const void* q, float* out,
                              float softmax_scale, void* stream);
+
+/* Eq. 1 for n_queries query rows per sequence and head at once (several positions scored against the same
+ * cache, as in speculative or chunked decoding): every row attends to every cached token, no mask among the rows.
+ *   q     device fp16 [batch, n_q_heads, n_queries, head_dim];  out device fp32, same shape.
+ *   n_queries  1 .. cfg.max_queries.
+ * The rows of a kv head share each read of its compressed blocks four at a time: G * n_queries rows take
+ * ceil(G * n_queries / 4) passes over the cache. */
+gear_status gear_decode_attn_multi(gear_cache* cache, const void* q, float* out, int32_t n_queries,
+                                   float softmax_scale, void* stream);
 
 /* Release the cache and everything it owns.  NULL is allowed. */
 void gear_free(gear_cache* cache);

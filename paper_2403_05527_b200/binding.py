@@ -27,7 +27,7 @@ class GearConfig(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("bits", C.c_int32), ("group", C.c_int32), ("outlier_pct", C.c_float), ("buffer_cap", C.c_int32),
                 ("rank_flush", C.c_int32), ("rank_max", C.c_int32), ("power_iters", C.c_int32),
-                ("max_tokens", C.c_int64), ("seed", C.c_uint64), ("flags", C.c_uint32), ("reserved", C.c_uint32)]
+                ("max_tokens", C.c_int64), ("seed", C.c_uint64), ("flags", C.c_uint32), ("max_queries", C.c_uint32)]
 
 
 class GearInfo(C.Structure):
@@ -59,6 +59,7 @@ _SIGNATURES = {
                                   C.c_int32, C.c_void_p, C.c_void_p]),
     "gear_append_buffer": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "gear_decode_attn": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
+    "gear_decode_attn_multi": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_float, C.c_void_p]),
     "gear_free": (None, [C.c_void_p]),
     "gear_release_workspace": (C.c_int32, []),
     "gear_append_buffer_host": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -123,9 +124,9 @@ def _stream(stream):
 
 
 def make_config(batch, n_q_heads, n_kv_heads, bits, group, outlier_pct, buffer_cap, rank_flush, max_tokens,
-                rank_max=None, power_iters=3, head_dim=128, seed=0, flags=0) -> GearConfig:
+                rank_max=None, power_iters=3, head_dim=128, seed=0, flags=0, max_queries=1) -> GearConfig:
     return GearConfig(batch, n_q_heads, n_kv_heads, head_dim, bits, group, float(outlier_pct), buffer_cap, rank_flush,
-                      rank_flush if rank_max is None else rank_max, power_iters, int(max_tokens), seed, flags, 0)
+                      rank_flush if rank_max is None else rank_max, power_iters, int(max_tokens), seed, flags, max_queries)
 
 
 def _check(status: int, where: str) -> int:
@@ -155,6 +156,12 @@ def gear_append_buffer(cache, k_new, v_new, B0_flush=None, stream=None) -> int:
 
 def gear_decode_attn(cache, q, out, softmax_scale: float = 0.0, stream=None) -> int:
     return _check(lib().gear_decode_attn(cache, _ptr(q), _ptr(out), softmax_scale, _stream(stream)), "gear_decode_attn")
+
+
+def gear_decode_attn_multi(cache, q, out, n_queries: int, softmax_scale: float = 0.0, stream=None) -> int:
+    """q, out: [B, H_q, n_queries, d_H]; every query row attends to the whole cache."""
+    return _check(lib().gear_decode_attn_multi(cache, _ptr(q), _ptr(out), n_queries, softmax_scale, _stream(stream)),
+                  "gear_decode_attn_multi")
 
 
 def gear_append_buffer_host(cache, k_new_host, v_new_host, B0_flush_host=None, stream=None) -> int:

@@ -113,6 +113,7 @@ struct gear_cache {
   int plan_key, plan_occ;
   DecodeArgs plan;
   int test_dead_wait;            // gear_test_dead_wait: the next decode calls wait on a barrier nothing completes
+  int max_queries, units_alloc;  // query rows per head the scratch was sized for; units of that size
 };
 
 static int outlier_count(float s_pct, int len) {
@@ -135,6 +136,7 @@ static gear_status check_config(const gear_config* c) {
   if (c->rank_flush < 0 || c->rank_flush > kMaxRank || c->rank_max < 0 || c->rank_max > kMaxRank) return GEAR_ERR_ARG;
   if (c->rank_flush > c->rank_max) return GEAR_ERR_ARG;
   if (c->rank_flush > c->buffer_cap) return GEAR_ERR_SHAPE;
+  if (c->max_queries > 64) return GEAR_ERR_ARG;
   if (c->power_iters < 1 || c->power_iters > 64) return GEAR_ERR_ARG;
   const int gv = c->group < kHeadDim ? c->group : kHeadDim;
   const int kv = outlier_count(c->outlier_pct, gv);
@@ -237,8 +239,11 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
     GEAR_TRY_ALLOC(c->dbg, c->dbg_bytes);
   }
   // decode scratch: one partial per (unit, warp touching it); upper bound of warps in a launch
-  const int hp = decode_heads_per_pass(c->G);
-  const int passes = decode_passes(c->G);
+  // scratch for the largest group of query rows a call may bring: G query heads x max_queries rows per kv head
+  c->max_queries = cfg->max_queries > 1 ? (int)cfg->max_queries : 1;
+  const int hp = decode_heads_per_pass(c->G * c->max_queries);
+  const int passes = decode_passes(c->G * c->max_queries);
+  c->units_alloc = (int)(BH * passes);
   const size_t units = BH * passes;
   const size_t nw_max = (size_t)c->sm_count * 32;        // one warp per CTA, at most 32 CTAs per SM
   c->max_parts = (int)(nw_max / units + 3);
@@ -381,15 +386,15 @@ extern "C" gear_status gear_append_buffer(gear_cache* c, const void* k_new, cons
   return GEAR_FLUSHED;
 }
 
-static gear_status plan_decode(gear_cache* c) {
-  const int key = (int)c->segs.size();
+static gear_status plan_decode(gear_cache* c, int Gq) {
+  const int key = (int)c->segs.size() * 4096 + Gq;
   if (c->plan_key == key) return GEAR_OK;
   // One-head passes: with four warps per scheduler the warps of a scheduler slow one another down by more than
   // the fourth warp adds (measured: 3 warps finish 0.85 blocks per microsecond and scheduler, 4 warps 0.79), so
   // long streams run with twelve resident warps.  Short streams (few blocks per warp) keep sixteen: there the
   // fixed cost per warp and the granularity of the split weigh more.
   int warps_cap = 0;
-  if (c->G == 1) {
+  if (Gq == 1) {
     const long long blocks = (long long)c->cc.BH * (c->n_blocks_c + (c->buf_len + 15) / 16);
     if (blocks >= 24LL * 16 * c->sm_count) warps_cap = 12;
   }
@@ -400,32 +405,39 @@ static gear_status plan_decode(gear_cache* c) {
     if (s.bfac_bytes > max_bfac) max_bfac = s.bfac_bytes;
     if (s.T > max_T) max_T = s.T;
   }
-  if (!decode_plan(c->cc.bits, c->G, c->cc.ngv, max_k, max_v, max_bfac, max_T, 227 * 1024, warps_cap, &c->plan))
+  if (!decode_plan(c->cc.bits, Gq, c->cc.ngv, max_k, max_v, max_bfac, max_T, 227 * 1024, warps_cap, &c->plan))
     return GEAR_ERR_SHAPE;
-  const int occ = decode_occupancy(c->cc.bits, c->G, c->cc.ngv, (size_t)c->plan.ws.total);
+  const int occ = decode_occupancy(c->cc.bits, Gq, c->cc.ngv, (size_t)c->plan.ws.total);
   if (occ < 1) return GEAR_ERR_CUDA;
   c->plan_occ = occ;
   c->plan_key = key;
   return GEAR_OK;
 }
 
-extern "C" gear_status gear_decode_attn(gear_cache* c, const void* q, float* out, float softmax_scale, void* stream) {
+// Decode attention for Gq query rows per kv head: q, out [B][H][Gq][128] (Gq = G for one query per head).
+static gear_status decode_rows(gear_cache* c, const void* q, float* out, int Gq, float softmax_scale, void* stream) {
   if (!c || !q || !out) return GEAR_ERR_ARG;
   if (((uintptr_t)q | (uintptr_t)out) & 15) return GEAR_ERR_ALIGN;
   if (c->n_compressed == 0 && c->buf_len == 0) return GEAR_ERR_STATE;
-  gear_status s = plan_decode(c);
+  gear_status s = plan_decode(c, Gq);
   if (s != GEAR_OK) return s;
   DecodeArgs a = c->plan;
   a.arena = c->arena; a.table = c->table_dev; a.blk2seg = c->blk2seg;
   a.buf_k = (const __half*)c->buf_k; a.buf_v = (const __half*)c->buf_v;
   a.q = (const __half*)q; a.out = out; a.partial = c->partial; a.tickets = c->tickets; a.status = c->status;
   a.cc = c->cc; a.n_blocks_c = c->n_blocks_c; a.buf_len = c->buf_len;
-  a.n_kv_heads = c->cfg.n_kv_heads; a.group_heads = c->G; a.max_parts = c->max_parts;
+  a.n_kv_heads = c->cfg.n_kv_heads; a.group_heads = Gq;
   const float sc = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)kHeadDim);
   a.scale_log2 = sc * 1.4426950408889634f;
   a.test_dead_wait = c->test_dead_wait;
   // one warp per CTA; never more warps than blocks of work
-  const int passes = decode_passes(c->G);
+  const int passes = decode_passes(Gq);
+  if ((long long)c->cc.BH * passes > c->units_alloc) return GEAR_ERR_CAPACITY;
+  // partial slots per unit for this call's unit count (the scratch was sized for the most units: fewer units get more
+  // slots each out of the same memory)
+  a.max_parts = (int)((size_t)c->sm_count * 32 / ((size_t)c->cc.BH * passes) + 3);
+  if ((size_t)c->cc.BH * passes * a.max_parts * decode_heads_per_pass(Gq) * kPartRow * 4 > c->partial_bytes)
+    return GEAR_ERR_CAPACITY;
   const long long work = (long long)c->cc.BH * passes * (c->n_blocks_c + (c->buf_len + 15) / 16);
   long long grid = (long long)c->sm_count * c->plan_occ;
   if (grid > work) grid = work;
@@ -437,7 +449,7 @@ extern "C" gear_status gear_decode_attn(gear_cache* c, const void* q, float* out
   {
     const long long units = (long long)c->cc.BH * passes, nb = work / units;
     const long long pb = grid / units, ua = grid - pb * units;         // ua units get pb + 1 ranges
-    if (pb >= 6 && pb + 1 <= nb && pb + 1 < c->max_parts) {
+    if (pb >= 6 && pb + 1 <= nb && pb + 1 < a.max_parts) {
       a.aligned = 1;
       a.units_a = (int)ua; a.parts_a = (int)pb + 1; a.parts_b = (int)pb;
       struct Cls { int len, u0, nu, p0, n; } cls[4];
@@ -463,6 +475,20 @@ extern "C" gear_status gear_decode_attn(gear_cache* c, const void* q, float* out
     return GEAR_ERR_CUDA;
   }
   return GEAR_OK;
+}
+
+extern "C" gear_status gear_decode_attn(gear_cache* c, const void* q, float* out, float softmax_scale, void* stream) {
+  if (!c) return GEAR_ERR_ARG;
+  return decode_rows(c, q, out, c->G, softmax_scale, stream);
+}
+
+extern "C" gear_status gear_decode_attn_multi(gear_cache* c, const void* q, float* out, int32_t n_queries,
+                                              float softmax_scale, void* stream) {
+  if (!c) return GEAR_ERR_ARG;
+  if (n_queries < 1 || n_queries > c->max_queries) return GEAR_ERR_ARG;
+  // The rows of one kv head -- its G query heads times n_queries positions -- are consecutive in q and out, and every
+  // row attends to the whole cache: to the kernel they are G * n_queries query heads of that kv head.
+  return decode_rows(c, q, out, c->G * n_queries, softmax_scale, stream);
 }
 
 extern "C" gear_status gear_append_buffer_host(gear_cache* c, const void* k_host, const void* v_host,
@@ -656,7 +682,7 @@ extern "C" gear_status gear_last_device_status(gear_cache* c, int32_t* code) {
   }
   if (v != 0) {
     // a warp that gave up left without taking its tickets: start the next call from a clean count
-    const size_t units = (size_t)c->cc.BH * decode_passes(c->G);
+    const size_t units = (size_t)c->units_alloc;
     if (cudaMemset(c->tickets, 0, units * 4) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
   }
   *code = v;

@@ -22,13 +22,19 @@ from . import binding as G
 
 
 def _kv(shape, n_heads, dev, seed):
+    """K, V fp16 of `shape` = (B, H, n, 128), drawn in slices of 16 sequences so that the fp32 temporaries stay small."""
     g = torch.Generator(device=dev)
     g.manual_seed(seed)
     c = torch.exp(torch.randn(n_heads, 128, generator=g, device=dev))[None, :, None, :]
-    k = torch.randn(shape, generator=g, device=dev) * c
-    k = torch.where(torch.rand(shape, generator=g, device=dev) < 0.01, k * 20.0, k).half().contiguous()
-    v = torch.randn(shape, generator=g, device=dev)
-    v = torch.where(torch.rand(shape, generator=g, device=dev) < 0.01, v * 20.0, v).half().contiguous()
+    k = torch.empty(shape, dtype=torch.float16, device=dev)
+    v = torch.empty(shape, dtype=torch.float16, device=dev)
+    for b0 in range(0, shape[0], 16):
+        part = (min(16, shape[0] - b0), *shape[1:])
+        x = torch.randn(part, generator=g, device=dev) * c
+        k[b0:b0 + part[0]] = torch.where(torch.rand(part, generator=g, device=dev) < 0.01, x * 20.0, x).half()
+        x = torch.randn(part, generator=g, device=dev)
+        v[b0:b0 + part[0]] = torch.where(torch.rand(part, generator=g, device=dev) < 0.01, x * 20.0, x).half()
+        del x
     return k, v
 
 
