@@ -185,9 +185,27 @@ def svd_solver(r_h: np.ndarray, b0: np.ndarray, rank: int, iters: int):
 # one tile: Filter -> Quant -> residual -> SVDSolver   (Algorithm 1, prefill body)
 # --------------------------------------------------------------------------
 def compress_tile(x16: np.ndarray, kind: str, bits: int, g: int, s_pct: float,
-                  rank: int, iters: int, b0: np.ndarray | None):
+                  rank: int, iters: int, b0: np.ndarray | None,
+                  filter_len: int | None = None, literal_eq5: bool = False):
     """Compress one (batch, head) tile X [n_c, d_H] (fp16) of keys ('K') or
-    values ('V').  Returns a dict with the canonical (unpacked) pieces:
+    values ('V').
+
+    Two switches select the other readings of Section 3 (defaults: the readings
+    listed in the module header):
+      filter_len   length of the vectors Filter_s acts on, along the grouping
+                   axis (tokens of a channel for keys, channels of a token for
+                   values).  None: the quantization group.  n_c for keys / d_H
+                   for values is Eq. 4 read literally: s/2 % of the largest and
+                   of the smallest entries of each whole channel / token vector.
+                   Must be a multiple of the group length.
+      literal_eq5  Eq. 5 read literally: the zeros that X - S holds at the
+                   outlier positions take part in min / max and receive a code
+                   like every other entry, so D^ is not 0 there and the residual
+                   at an outlier position is -D^.
+    With g at least the vector length the groups are the whole vectors (the
+    per-vector grouping, KCVT, of Section 2).
+
+    Returns a dict with the canonical (unpacked) pieces:
       codes u8 [n_c, d_H]; scale, zero fp16 ('K': [n_c/g_K, d_H]; 'V': [n_c, d_H/g_V]);
       mask bool [n_c, d_H] (support of S); S float64 (exact fp16 values on the mask);
       out_idx u8 / out_val fp16 [n_groups, 2k] (in-group index ascending);
@@ -200,9 +218,23 @@ def compress_tile(x16: np.ndarray, kind: str, bits: int, g: int, s_pct: float,
     x = x16.astype(F64)
 
     gr = tile_to_groups(x, kind, g_len)
-    gmask = filter_groups(gr, k)                                   # Eq. 4
-    codes_g, scale16, zero16 = quantize_groups(gr.astype(F16), gmask, bits)   # Eq. 5
-    d_g = dequantize_groups(codes_g, scale16, zero16, gmask)
+    if filter_len is None or filter_len == g_len:
+        gmask = filter_groups(gr, k)                               # Eq. 4, per quantization group
+        kf = k
+    else:
+        vec_len = n_c if kind == "K" else d_h
+        if filter_len % g_len or vec_len % filter_len:
+            raise ValueError("filter length must be a multiple of the group length and divide the vector")
+        kf = outlier_count(s_pct, filter_len)
+        fmask = filter_groups(tile_to_groups(x, kind, filter_len), kf)          # Eq. 4 on longer vectors
+        gmask = tile_to_groups(groups_to_tile(fmask, kind, n_c, d_h), kind, g_len)
+    if literal_eq5:
+        none = np.zeros_like(gmask)
+        codes_g, scale16, zero16 = quantize_groups(np.where(gmask, 0.0, gr).astype(F16), none, bits)   # Quant_b(X - S)
+        d_g = dequantize_groups(codes_g, scale16, zero16, none)
+    else:
+        codes_g, scale16, zero16 = quantize_groups(gr.astype(F16), gmask, bits)   # Eq. 5, outliers masked out
+        d_g = dequantize_groups(codes_g, scale16, zero16, gmask)
 
     mask = groups_to_tile(gmask, kind, n_c, d_h)
     codes = groups_to_tile(codes_g, kind, n_c, d_h)
@@ -210,10 +242,10 @@ def compress_tile(x16: np.ndarray, kind: str, bits: int, g: int, s_pct: float,
     s_mat = np.where(mask, x, 0.0)
     resid = x - d_hat - s_mat                                      # R = X - (D^ + S)
 
-    if k:
+    if k and (filter_len is None or filter_len == g_len):
         out_idx = np.nonzero(gmask)[1].reshape(-1, 2 * k).astype(np.uint8)   # ascending per group
         out_val = gr[gmask].reshape(-1, 2 * k).astype(F16)
-    else:
+    else:                                        # none, or a varying number per group: the mask and S carry them
         out_idx = np.zeros((gr.shape[0], 0), np.uint8)
         out_val = np.zeros((gr.shape[0], 0), F16)
 

@@ -257,3 +257,80 @@ def test_exact_half_steps_round_to_even():
     codes, sc, ze = O.quantize_groups(x16, np.zeros(x16.shape, bool), 2)
     assert float(sc[0]) == 1.0 and float(ze[0]) == 0.0
     assert codes[0].tolist() == [0, 3, 0, 2, 2, 1, 2, 1]
+
+
+# --------------------------------------------------------------------------- the other readings of Section 3
+def _vec_brute_force(vec, k):
+    """k largest then k smallest of what is left, value first, lower index on ties: plain loops."""
+    chosen = []
+    for sign in (-1.0, 1.0):
+        order = sorted((i for i in range(len(vec)) if i not in chosen), key=lambda i: (sign * float(vec[i]), i))
+        chosen += order[:k]
+    return sorted(chosen)
+
+
+def test_per_vector_filter_is_eq4_on_whole_channels_and_tokens():
+    """filter_len = the vector length: s/2 % of the largest and smallest entries of every key channel over all tokens
+    and of every value token over all channels (Eq. 4 as printed), while the quantization groups keep length g."""
+    rng = np.random.default_rng(21)
+    n_c, d, g = 64, 128, 16
+    x = rng.standard_normal((n_c, d)).astype(np.float16)
+    x[rng.random((n_c, d)) < 0.02] *= 12
+    tk = O.compress_tile(x, "K", 4, g, 8.0, 0, 3, None, filter_len=n_c)
+    tv = O.compress_tile(x, "V", 4, g, 8.0, 0, 3, None, filter_len=d)
+    kk, kv = O.outlier_count(8.0, n_c), O.outlier_count(8.0, d)
+    for j in range(0, d, 17):
+        assert sorted(np.nonzero(tk["mask"][:, j])[0]) == _vec_brute_force(x[:, j], kk)
+    for i in range(0, n_c, 9):
+        assert sorted(np.nonzero(tv["mask"][i])[0]) == _vec_brute_force(x[i], kv)
+    for t in (tk, tv):
+        assert np.array_equal(t["S"][t["mask"]], x.astype(np.float64)[t["mask"]])     # outliers kept exactly
+        assert np.all(t["D"][t["mask"]] == 0) and np.all(t["R"][t["mask"]] == 0)
+        keep = ~t["mask"]
+        scale = np.repeat(t["scale"].astype(np.float64), g, axis=0 if t["kind"] == "K" else 1)
+        assert np.all(np.abs(t["R"][keep]) <= scale[keep] * (0.5 + 2.0 ** -10))
+
+
+def test_filter_length_equal_to_the_group_is_the_default_and_whole_vector_groups_are_kcvt():
+    rng = np.random.default_rng(22)
+    x = (rng.standard_normal((128, 128)) * np.exp(rng.standard_normal(128))).astype(np.float16)
+    for kind, g in (("K", 32), ("V", 64)):
+        a = O.compress_tile(x, kind, 2, g, 4.0, 2, 3, rng.standard_normal((128, 2)))
+        b = O.compress_tile(x, kind, 2, g, 4.0, 2, 3, rng.standard_normal((128, 2)), filter_len=g)
+        for key in ("codes", "mask", "D"):
+            assert np.array_equal(a[key], b[key])
+    # groups as long as the vectors: one (scale, zero) per key channel over all tokens, one per value token
+    tk = O.compress_tile(x, "K", 4, 10 ** 6, 2.0, 0, 3, None)
+    tv = O.compress_tile(x, "V", 4, 10 ** 6, 2.0, 0, 3, None)
+    assert tk["scale"].shape == (1, 128) and tv["scale"].shape == (128, 1)
+    j = 5
+    keep = ~tk["mask"][:, j]
+    col = x[:, j].astype(np.float64)
+    assert tk["zero"][0, j] == np.float16(col[keep].min())
+    d32 = np.float32(np.float32(col[keep].max() - col[keep].min()) / np.float32(15))
+    assert tk["scale"][0, j] == np.float16(d32)
+    assert tk["mask"][:, j].sum() == 2 * O.outlier_count(2.0, 128)
+
+
+def test_literal_eq5_codes_the_zeros_left_by_the_outliers():
+    """Quant_b(X - S) with the zeros in the range: an all-positive group's minimum becomes 0, its range widens, and the
+    outlier positions carry D^ = dequant(code of 0), R = -D^ there; X^ = D^ + S + R still equals X everywhere."""
+    rng = np.random.default_rng(23)
+    x = (np.abs(rng.standard_normal((64, 128))) + 3.0).astype(np.float16)        # every group is strictly positive
+    lit = O.compress_tile(x, "V", 4, 64, 4.0, 0, 3, None, literal_eq5=True)
+    msk = O.compress_tile(x, "V", 4, 64, 4.0, 0, 3, None)
+    assert np.array_equal(lit["mask"], msk["mask"])
+    assert np.all(lit["zero"] == 0) and np.all(msk["zero"].astype(np.float64) >= 3.0)
+    assert np.all(lit["scale"].astype(np.float64) > msk["scale"].astype(np.float64))
+    m = lit["mask"]
+    assert np.all(lit["D"][m] == 0.0) and np.all(lit["codes"][m] == 0)           # quant(0) with zero-point 0 is code 0
+    x64 = x.astype(np.float64)
+    assert np.allclose(lit["D"] + lit["S"] + lit["R"], x64, atol=0, rtol=0)
+    # a group that straddles zero: the zero entries land on a grid point near 0, not on 0
+    y = rng.standard_normal((64, 128)).astype(np.float16)
+    lit2 = O.compress_tile(y, "K", 2, 64, 4.0, 0, 3, None, literal_eq5=True)
+    m2 = lit2["mask"]
+    scale = np.repeat(lit2["scale"].astype(np.float64), 64, axis=0)
+    assert np.all(np.abs(lit2["D"][m2]) <= scale[m2] * (0.5 + 2.0 ** -10))
+    assert np.any(lit2["D"][m2] != 0.0)
+    assert np.array_equal(lit2["R"][m2], -lit2["D"][m2])
