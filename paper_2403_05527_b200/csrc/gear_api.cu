@@ -407,7 +407,7 @@ static gear_status plan_decode(gear_cache* c, int Gq) {
   }
   if (!decode_plan(c->cc.bits, Gq, c->cc.ngv, max_k, max_v, max_bfac, max_T, 227 * 1024, warps_cap, &c->plan))
     return GEAR_ERR_SHAPE;
-  const int occ = decode_occupancy(c->cc.bits, Gq, c->cc.ngv, (size_t)c->plan.ws.total);
+  const int occ = decode_occupancy(c->cc.bits, Gq, c->cc.ngv, c->plan.wide, (size_t)c->plan.ws.total);
   if (occ < 1) return GEAR_ERR_CUDA;
   c->plan_occ = occ;
   c->plan_key = key;

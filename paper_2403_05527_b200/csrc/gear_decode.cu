@@ -202,6 +202,7 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
     a->aligned = 0;
     a->nstage = (int)ns; a->stage_bytes = stage; a->bregion = bregion; a->max_T = max_T; a->hpa = HP; a->ws = w;
     a->spin_limit = kDecodeSpinLimit; a->test_dead_wait = 0;
+    a->wide = (HP == 1 && warps <= 12) ? 1 : 0;          // twelve warps or fewer: the 168-register build
     return true;
   }
   return false;
@@ -258,8 +259,10 @@ int static_shape_id(const SegDesc& s, const CacheConst& c) {
 
 // ------------------------------------------------------------------ the kernel
 // HEADS = query heads handled per pass: 1 (multi-head attention) or 4 (grouped queries; a pass may hold fewer).
-template <int BITS, int HEADS, int NGV>
-__global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(const __grid_constant__ DecodeArgs a) {
+// MINB = resident warps per SM the registers are budgeted for: 16 (128 registers) or 12 (168 registers: about a tenth
+// fewer instructions, for long streams where twelve warps are enough) with one head per pass, 8 with four.
+template <int BITS, int HEADS, int NGV, int MINB>
+__global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_constant__ DecodeArgs a) {
   constexpr int HP = HEADS;
   constexpr int NT = HP == 1 ? 1 : 2;             // 8-column tiles of the integer B operands: four limb columns per head
   constexpr int F = 8 / BITS;                     // code fields per byte
@@ -1368,11 +1371,12 @@ __global__ void __launch_bounds__(32, HEADS == 1 ? 16 : 8) gear_decode_kernel(co
 
 // ------------------------------------------------------------------ host side
 template <class Fn>
-static bool with_decode_kernel(int bits, int heads, int ngv, Fn fn) {
+static bool with_decode_kernel(int bits, int heads, int ngv, int wide, Fn fn) {
   const int hp = decode_heads_per_pass(heads);
-#define GEAR_DEC_CASE(B, N, V) \
-  if (bits == B && hp == N && ngv == V) { fn(gear_decode_kernel<B, N, V>); return true; }
-#define GEAR_DEC_HEADS(B, V) GEAR_DEC_CASE(B, 1, V) GEAR_DEC_CASE(B, 4, V)
+  const int minb = hp == 1 ? (wide ? 12 : 16) : 8;
+#define GEAR_DEC_CASE(B, N, V, M) \
+  if (bits == B && hp == N && ngv == V && minb == M) { fn(gear_decode_kernel<B, N, V, M>); return true; }
+#define GEAR_DEC_HEADS(B, V) GEAR_DEC_CASE(B, 1, V, 16) GEAR_DEC_CASE(B, 1, V, 12) GEAR_DEC_CASE(B, 4, V, 8)
   GEAR_DEC_HEADS(2, 1) GEAR_DEC_HEADS(2, 2) GEAR_DEC_HEADS(2, 4) GEAR_DEC_HEADS(2, 8)
   GEAR_DEC_HEADS(4, 1) GEAR_DEC_HEADS(4, 2) GEAR_DEC_HEADS(4, 4) GEAR_DEC_HEADS(4, 8)
 #undef GEAR_DEC_HEADS
@@ -1383,7 +1387,7 @@ static bool with_decode_kernel(int bits, int heads, int ngv, Fn fn) {
 cudaError_t launch_decode(const DecodeArgs& a, int grid, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
   const size_t smem = (size_t)a.ws.total;
-  const bool ok = with_decode_kernel(a.cc.bits, a.group_heads, a.cc.ngv, [&](auto kern) {
+  const bool ok = with_decode_kernel(a.cc.bits, a.group_heads, a.cc.ngv, a.wide, [&](auto kern) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return;
     kern<<<grid, 32, smem, st>>>(a);
@@ -1394,10 +1398,10 @@ cudaError_t launch_decode(const DecodeArgs& a, int grid, cudaStream_t st) {
   return e;
 }
 
-int decode_occupancy(int bits, int heads, int ngv, size_t smem) {
+int decode_occupancy(int bits, int heads, int ngv, int wide, size_t smem) {
   int occ = 0;
   cudaError_t e = cudaErrorInvalidValue;
-  with_decode_kernel(bits, heads, ngv, [&](auto kern) {
+  with_decode_kernel(bits, heads, ngv, wide, [&](auto kern) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, 32, smem);
   });

@@ -32,7 +32,7 @@ cudaError_t launch_fp16_attn(const void* K, const void* V, const void* q, float*
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   DecodeArgs a;
   if (!decode_plan(2, G, 1, 0, 0, 0, 16, 227 * 1024, 0, &a)) return cudaErrorInvalidConfiguration;
-  const int occ = decode_occupancy(2, G, 1, (size_t)a.ws.total);
+  const int occ = decode_occupancy(2, G, 1, a.wide, (size_t)a.ws.total);
   if (occ < 1) return cudaErrorInvalidConfiguration;
   long long grid = (long long)sms * occ;
   const long long work = (long long)units * ((n + 15) / 16);
@@ -129,7 +129,7 @@ extern "C" gear_status gear_fp16_decode_attn_static(const void* K, const void* V
   }
   DecodeArgs a;
   if (!decode_plan(2, G, 1, 0, 0, 0, 16, 227 * 1024, 0, &a)) return GEAR_ERR_SHAPE;
-  const int occ = decode_occupancy(2, G, 1, (size_t)a.ws.total);
+  const int occ = decode_occupancy(2, G, 1, a.wide, (size_t)a.ws.total);
   if (occ < 1) return GEAR_ERR_CUDA;
   long long grid = (long long)sms * occ;
   const long long work = (long long)units * ((n + 15) / 16);

@@ -97,6 +97,7 @@ struct DecodeArgs {
   int hpa;                    // query heads per pass (1 or 4)
   int spin_limit;             // polls a consumer spends on one ring stage before it gives up
   int test_dead_wait;         // test only: wait once on a barrier that nothing completes, with a short limit
+  int wide;                   // one head per pass: use the kernel built for twelve resident warps (more registers)
   WarpSmem ws;
   float scale_log2;           // softmax scale * log2(e)
 };
@@ -105,7 +106,7 @@ cudaError_t launch_decode(const DecodeArgs& a, int grid, cudaStream_t st);
 // warps_cap > 0 limits the resident warps per SM below what registers and shared memory allow.
 bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int max_bfac, int max_T, size_t smem_budget,
                  int warps_cap, DecodeArgs* a);
-int decode_occupancy(int bits, int heads, int ngv, size_t smem);
+int decode_occupancy(int bits, int heads, int ngv, int wide, size_t smem);
 int static_shape_id(const SegDesc& s, const CacheConst& c);
 // query heads one pass of the kernel takes for G query heads per kv head, and the number of passes
 inline int decode_heads_per_pass(int G) { return G == 1 ? 1 : 4; }
