@@ -30,6 +30,7 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <math.h>
+#include <string.h>
 
 #include <type_traits>
 
@@ -334,6 +335,11 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
     u = (int)(f0 / NB);
     blk_lo = (int)(f0 - (long long)u * NB);
   }
+
+  // Everything above used kernel parameters and shared memory only.  Let the launch after this one start its own
+  // prologue, and wait until the launches before this one have completed and their writes are visible.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   auto load_desc = [&](SegDesc* dst, int blk) {
     const int* src = reinterpret_cast<const int*>(a.table + a.blk2seg[blk]);
@@ -1390,8 +1396,17 @@ cudaError_t launch_decode(const DecodeArgs& a, int grid, cudaStream_t st) {
   const bool ok = with_decode_kernel(a.cc.bits, a.group_heads, a.cc.ngv, a.wide, [&](auto kern) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return;
-    kern<<<grid, 32, smem, st>>>(a);
-    e = cudaGetLastError();
+    // Programmatic dependent launch: the CTAs of this launch may become resident while the kernel before it on the
+    // stream drains (the kernel below announces that at once, and waits for its predecessor before its first read of
+    // global memory), so that back-to-back decode calls do not pay the launch ramp one after the other.
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(32); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kern, a);
   });
   if (!ok) return cudaErrorInvalidValue;
   if (e == cudaSuccess) count_launches(1);
