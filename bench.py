@@ -37,8 +37,9 @@ from paper_2403_05527_b200 import synth  # noqa: E402
 METRIC = "compressed-KV decode attn tokens/s"
 UNIT = "tokens/s"
 # dram__bytes_read + dram__bytes_write of one gear_decode_kernel launch per algorithmic byte, from an ncu capture of the
-# kernel on one C2 layer cache (137.5 MB of DRAM traffic for 134.3 MB); traffic grows in proportion to the cache
-DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {2: 1.0245}
+# kernel on one layer cache (C2: 137.65 MB of DRAM traffic for 134.26 MB; C4: 125.65 MB for 118.48 MB); traffic grows in
+# proportion to the cache
+DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {2: 1.0253, 4: 1.0605}
 EXTRA_CONFIGS = (3, 32, 4)
 
 
