@@ -64,6 +64,8 @@ _SIGNATURES = {
     "gear_release_workspace": (C.c_int32, []),
     "gear_append_buffer_host": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "gear_decode_attn_host": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
+    "gear_decode_attn_host_async": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
+    "gear_stream_wait": (C.c_int32, [C.c_void_p]),
     "gear_fp16_decode_attn": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                           C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_float, C.c_void_p,
                                           C.c_size_t, C.c_void_p]),
@@ -172,6 +174,15 @@ def gear_append_buffer_host(cache, k_new_host, v_new_host, B0_flush_host=None, s
 def gear_decode_attn_host(cache, q_host, out_host, softmax_scale: float = 0.0, stream=None) -> int:
     return _check(lib().gear_decode_attn_host(cache, _ptr(q_host), _ptr(out_host), softmax_scale, _stream(stream)),
                   "gear_decode_attn_host")
+
+
+def gear_decode_attn_host_async(cache, q_host, out_host, softmax_scale: float = 0.0, stream=None) -> int:
+    return _check(lib().gear_decode_attn_host_async(cache, _ptr(q_host), _ptr(out_host), softmax_scale,
+                                                    _stream(stream)), "gear_decode_attn_host_async")
+
+
+def gear_stream_wait(stream=None) -> int:
+    return _check(lib().gear_stream_wait(_stream(stream)), "gear_stream_wait")
 
 
 def gear_fp16_attn_scratch_bytes(batch, n_q_heads, head_dim=128) -> int:

@@ -526,8 +526,8 @@ extern "C" gear_status gear_append_buffer_host(gear_cache* c, const void* k_host
   return s;
 }
 
-extern "C" gear_status gear_decode_attn_host(gear_cache* c, const void* q_host, float* out_host, float softmax_scale,
-                                             void* stream) {
+static gear_status decode_host(gear_cache* c, const void* q_host, float* out_host, float softmax_scale, void* stream,
+                               bool wait) {
   if (!c || !q_host || !out_host) return GEAR_ERR_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t nq = (size_t)c->cfg.batch * c->cfg.n_q_heads * kHeadDim;
@@ -538,7 +538,25 @@ extern "C" gear_status gear_decode_attn_host(gear_cache* c, const void* q_host, 
   gear_status s = gear_decode_attn(c, c->stage_q, c->stage_out, softmax_scale, stream);
   if (s != GEAR_OK) return s;
   if (cudaMemcpyAsync(out_host, c->stage_out, nq * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-      cudaStreamSynchronize(st) != cudaSuccess) {
+      (wait && cudaStreamSynchronize(st) != cudaSuccess)) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  return GEAR_OK;
+}
+
+extern "C" gear_status gear_decode_attn_host(gear_cache* c, const void* q_host, float* out_host, float softmax_scale,
+                                             void* stream) {
+  return decode_host(c, q_host, out_host, softmax_scale, stream, true);
+}
+
+extern "C" gear_status gear_decode_attn_host_async(gear_cache* c, const void* q_host, float* out_host,
+                                                   float softmax_scale, void* stream) {
+  return decode_host(c, q_host, out_host, softmax_scale, stream, false);
+}
+
+extern "C" gear_status gear_stream_wait(void* stream) {
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) {
     cudaGetLastError();
     return GEAR_ERR_CUDA;
   }

@@ -156,6 +156,11 @@ def test_host_buffer_entry_points(pair_factory):
     G.gear_decode_attn_host(p.cache, q, out)
     ref = p.oracle.decode_attn(q)
     assert np.abs(out - ref).max() / np.abs(ref).max() <= 1e-3
+    # the queued form: nothing is valid before the wait, the same bits after it
+    out2 = np.zeros((1, 2, 128), np.float32)
+    G.gear_decode_attn_host_async(p.cache, q, out2)
+    G.gear_stream_wait()
+    assert np.array_equal(out, out2)
 
 
 def test_fp16_cache_attention_against_textbook():
