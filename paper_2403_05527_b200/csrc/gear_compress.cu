@@ -254,7 +254,16 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
   // residual tile -> workspace (only needed when a low-rank part is fitted)
   if (p.R != nullptr) {
     float* R = p.R + (((size_t)bhl * 2 + side) * sd.n_c + (size_t)blk * T) * kHeadDim;
-    for (int i = tid; i < T * kHeadDim; i += 128) R[i] = rs[(i >> 7) * kRPitch + (i & 127)];
+    float rmax = 0.f;
+    for (int i = tid; i < T * kHeadDim; i += 128) {
+      const float v = rs[(i >> 7) * kRPitch + (i & 127)];
+      R[i] = v;
+      rmax = fmaxf(rmax, fabsf(v));
+    }
+    // the largest residual magnitude of the (batch, head, side) tile: the power iteration scales by it
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
+    if ((tid & 31) == 0) atomicMax(p.Rmax + bhl * 2 + side, __float_as_uint(rmax));
   }
 }
 
@@ -263,8 +272,40 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
 // R_h [n_c, 128] in the workspace.  Factor buffers are [128][16] fp32, zero
 // beyond the rank.
 // ---------------------------------------------------------------------------
+// ---- helpers of the tensor-core pass
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// transpose of an 8 x 8 tile of 16-bit elements held one row pair per lane (the ldmatrix distribution)
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+// floor(log2 |x|) for a finite x > 0 (0 for x == 0): the power of two that brings x into [1, 2)
+__device__ __forceinline__ int pow2_exponent(float x) { return x > 0.f ? ilogbf(x) : 0; }
+__device__ __forceinline__ float exp2_int(int e) { return scalbnf(1.0f, e); }
+// (x0, x1) -> packed fp16 heads and packed fp16 remainders (x - head, exact in fp32 before its own rounding)
+__device__ __forceinline__ void split_pair(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  const __half2 h = __floats2half2_rn(x0, x1);
+  const float2 hf = __half22float2(h);
+  const __half2 l = __floats2half2_rn(x0 - hf.x, x1 - hf.y);
+  hi = *reinterpret_cast<const uint32_t*>(&h);
+  lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+// x -> (head, remainder) packed in one register, head in the low half
+__device__ __forceinline__ void split_pair_hl(float x, uint32_t& hl) {
+  const __half h = __float2half_rn(x);
+  const __half l = __float2half_rn(x - __half2float(h));
+  const __half2 v = __halves2half2(h, l);
+  hl = *reinterpret_cast<const uint32_t*>(&v);
+}
+
 constexpr int kChunkRows = 512;
-constexpr int kPassWarps = 8;
+constexpr int kPassWarps = 4;
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -303,110 +344,132 @@ __global__ void pi_init_kernel(PiArgs p, const float* B0, int bh0, int BH_total_
   (void)BH_total_rank_stride;
 }
 
-// Sums over the warp of RP values per lane, every lane getting all RP sums.  The first log2(RP) exchange steps
-// halve the number of values a lane carries (each lane hands the half it drops to its partner), the remaining steps are
-// a butterfly on the single value left, and a broadcast per value returns the sums: RP - 1 + (5 - log2 RP) + RP
-// shuffles instead of 5 RP.  The order of the additions is fixed, so results are reproducible.
-template <int RP>
-__device__ __forceinline__ void warp_sum_all(float (&s)[RP], int lane) {
-  constexpr int LOG = RP == 4 ? 2 : (RP == 8 ? 3 : 4);
-  static_assert(RP == 4 || RP == 8 || RP == 16, "rank padding");
-  int cnt = RP;
-#pragma unroll
-  for (int step = 0; step < 5; ++step) {
-    const int o = 16 >> step;
-    if (step < LOG) {
-      const bool upper = (lane & o) != 0;
-      cnt >>= 1;
-#pragma unroll
-      for (int i = 0; i < RP / 2; ++i) {
-        if (i < cnt) {
-          const float send = upper ? s[i] : s[i + cnt];
-          const float keep = upper ? s[i + cnt] : s[i];
-          s[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
-        }
-      }
-    } else {
-      s[0] += __shfl_xor_sync(0xffffffffu, s[0], o);
-    }
-  }
-  const float mine = s[0];                    // the sum of value (lane >> (5 - LOG)) % RP
-#pragma unroll
-  for (int r = 0; r < RP; ++r) s[r] = __shfl_sync(0xffffffffu, mine, r << (5 - LOG));
-}
-
 // One pass over the residual: a = R b for every row, and this chunk's partial of R^T a.
 // mode 0: loops before the last.
 // mode 1: last loop: the rows a are also stored (A0).  Its Gram matrix and the orthonormalising factor W come from
 //         the small kernels below, and since R^T (A0 W) = (R^T A0) W, with W only 16 x 16, R is not read again.
-template <int RP, int MODE>
-__global__ void __launch_bounds__(kPassWarps * 32) pi_pass_kernel(PiArgs p) {
-  __shared__ float red[kHeadDim * RP];            // cross-warp sum, accumulated warp by warp
+//
+// Both products run on the tensor cores (mma.sync.m16n8k16, fp16 operands, fp32 accumulation) with every fp32
+// operand cut into an fp16 head and an fp16 remainder, the four cross products summed in fp32: 22 bits of each
+// operand survive.  Powers of two bring the operands into fp16's range first (R by the tile's largest magnitude, each
+// column of b by its own, a by the bound that follows) and are divided out of the results, so the scaling itself is
+// exact.  A warp owns 16 rows at a time.  A lane loads, for rows gid and gid + 8, the four channels 16c + 4t .. + 3 of
+// each 16-channel step c as one 128-bit load; since a contraction does not care about the order of its index, these
+// four channels serve as the step's k indices 2t, 2t+1, 2t+8, 2t+9 of the A fragment.  For R^T a the same registers,
+// transposed 8 x 8 by movmatrix, are the A fragment of R^T (rows: channels 4j, 4j+1 | 4j+2, 4j+3 of the step).
+template <int MODE>
+__global__ void __launch_bounds__(kPassWarps * 32, 3) pi_pass_kernel(PiArgs p) {
+  constexpr int RP = 4;                            // rank columns per CTA: 4 x (head, remainder) = the 8 columns of n
+  __shared__ float red[kHeadDim * RP];             // cross-warp sum, accumulated warp by warp
+  __shared__ __align__(16) __half bsplit[2 * RP][kHeadDim];   // [2 rho + (0: head, 1: remainder)][channel]
+  __shared__ float colmax[kPassWarps][RP];
   const int tile = blockIdx.y, chunk = blockIdx.x;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, t = lane & 3;
   const int row0 = chunk * kChunkRows;
   const int row1 = min(p.n_c, row0 + kChunkRows);
-  const int rho0 = blockIdx.z * RP;               // this CTA's rank columns [rho0, rho0 + RP)
+  const int rho0 = blockIdx.z * RP;                // this CTA's rank columns [rho0, rho0 + RP)
   const float* R = p.R + (size_t)tile * p.n_c * kHeadDim;
   float* A0 = p.A0 + (size_t)tile * p.n_c * kMaxRank + rho0;
 
-  float b[4][RP];
+  // ---- the scaled, split factor columns
+  const int er = pow2_exponent(__uint_as_float(p.Rmax[tile]));
+  const float sr = exp2_int(-er);
+  int eb[RP];
+  {
+    const int j = threadIdx.x;                     // one channel per thread (kPassWarps * 32 == kHeadDim)
+    float bj[RP];
 #pragma unroll
-  for (int j = 0; j < 4; ++j)
+    for (int r = 0; r < RP; ++r) {
+      bj[r] = p.Bcur[((size_t)tile * kHeadDim + j) * kMaxRank + rho0 + r];
+      float m = fabsf(bj[r]);
 #pragma unroll
-    for (int r = 0; r < RP; ++r) b[j][r] = p.Bcur[((size_t)tile * kHeadDim + lane * 4 + j) * kMaxRank + rho0 + r];
-  float acc[4][RP];       // this lane's 4 channels of R^T a
-#pragma unroll
-  for (int j = 0; j < 4; ++j)
-#pragma unroll
-    for (int r = 0; r < RP; ++r) acc[j][r] = 0.f;
-
-  // U rows of a warp are requested before the first is used: with one row in flight per warp the pass is bound by
-  // the latency of that load, not by bandwidth
-  constexpr int U = RP <= 8 ? 4 : 2;
-  for (int rowu = row0 + warp; rowu < row1; rowu += kPassWarps * U) {
-    float4 xs[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int r = rowu + u * kPassWarps;
-      xs[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (r < row1) xs[u] = *reinterpret_cast<const float4*>(R + (size_t)r * kHeadDim + lane * 4);
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      if (lane == 0) colmax[warp][r] = m;
     }
+    __syncthreads();
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int row = rowu + u * kPassWarps;
-      if (row >= row1) break;                      // uniform over the warp
-      const float x[4] = {xs[u].x, xs[u].y, xs[u].z, xs[u].w};
-      float a[RP];
+    for (int r = 0; r < RP; ++r) {
+      float m = 0.f;
 #pragma unroll
-      for (int r = 0; r < RP; ++r) {
-        float s = 0.f;
+      for (int w = 0; w < kPassWarps; ++w) m = fmaxf(m, colmax[w][r]);
+      eb[r] = pow2_exponent(m);
+      const float v = bj[r] * exp2_int(-eb[r]);
+      const __half h = __float2half_rn(v);
+      bsplit[2 * r][j] = h;
+      bsplit[2 * r + 1][j] = __float2half_rn(v - __half2float(h));
+    }
+    for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x) red[i] = 0.f;
+    __syncthreads();
+  }
+  // B fragments of a = R b: column n = gid is (rho = gid >> 1, head | remainder), k as described above
+  uint32_t bf[8][2];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) s = fmaf(x[j], b[j][r], s);
-        a[r] = s;
-      }
-      warp_sum_all<RP>(a, lane);
-      if (MODE == 1) {
-        float mine = 0.f;
+  for (int c = 0; c < 8; ++c) {
+    const uint2 v = *reinterpret_cast<const uint2*>(&bsplit[gid][16 * c + 4 * t]);
+    bf[c][0] = v.x; bf[c][1] = v.y;
+  }
+  // |R sr| < 2 and |b 2^-eb| < 2, so |a| < 512 in these units: a 2^-10 stays below one half
+  constexpr float kScaleA = 1.0f / 1024.0f;
+  const int ebt = t == 0 ? eb[0] : (t == 1 ? eb[1] : (t == 2 ? eb[2] : eb[3]));
+  const float inv_a = exp2_int(er + ebt);                   // back to a = R b for column rho = t
+  const float inv_acc = exp2_int(2 * er + ebt + 10);        // back to R^T a
+
+  float acc[8][4];        // R^T a: [step c][(channel 4 gid/2 + gid%2 of the step | the same + 2) x (head, remainder) of rho = t]
 #pragma unroll
-        for (int r = 0; r < RP; ++r) if (r == lane) mine = a[r];
-        if (lane < RP) A0[(size_t)row * kMaxRank + lane] = mine;
-      }
+  for (int c = 0; c < 8; ++c)
 #pragma unroll
-      for (int j = 0; j < 4; ++j)
+    for (int i = 0; i < 4; ++i) acc[c][i] = 0.f;
+
+  for (int rb = row0 + warp * 16; rb < row1; rb += kPassWarps * 16) {
+    const int ra = rb + gid, rc = rb + gid + 8;
+    const bool va = ra < row1, vc = rc < row1;
+    float4 xa[8], xc[8];
 #pragma unroll
-        for (int r = 0; r < RP; ++r) acc[j][r] = fmaf(x[j], a[r], acc[j][r]);
+    for (int c = 0; c < 8; ++c) {
+      xa[c] = va ? *reinterpret_cast<const float4*>(R + (size_t)ra * kHeadDim + 16 * c + 4 * t) : make_float4(0.f, 0.f, 0.f, 0.f);
+      xc[c] = vc ? *reinterpret_cast<const float4*>(R + (size_t)rc * kHeadDim + 16 * c + 4 * t) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    uint32_t fh[8][4], fl[8][4];
+    float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      split_pair(xa[c].x * sr, xa[c].y * sr, fh[c][0], fl[c][0]);
+      split_pair(xc[c].x * sr, xc[c].y * sr, fh[c][1], fl[c][1]);
+      split_pair(xa[c].z * sr, xa[c].w * sr, fh[c][2], fl[c][2]);
+      split_pair(xc[c].z * sr, xc[c].w * sr, fh[c][3], fl[c][3]);
+      mma16816(d, fh[c], bf[c][0], bf[c][1]);
+      mma16816(d, fl[c], bf[c][0], bf[c][1]);
+    }
+    const float a_lo_rows = d[0] + d[1], a_hi_rows = d[2] + d[3];   // a[row gid][rho t], a[row gid + 8][rho t] (scaled)
+    if (MODE == 1) {
+      if (va) A0[(size_t)ra * kMaxRank + t] = a_lo_rows * inv_a;
+      if (vc) A0[(size_t)rc * kMaxRank + t] = a_hi_rows * inv_a;
+    }
+    // B fragment of R^T a: k = row, n = (rho, head | remainder): the 8 x 8 tiles [row][2 rho + part], transposed
+    uint32_t m0, m1;
+    split_pair_hl(a_lo_rows * kScaleA, m0);
+    split_pair_hl(a_hi_rows * kScaleA, m1);
+    const uint32_t ab0 = movmatrix_trans(m0), ab1 = movmatrix_trans(m1);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      uint32_t th[4], tl[4];
+      th[0] = movmatrix_trans(fh[c][0]); th[1] = movmatrix_trans(fh[c][2]);
+      th[2] = movmatrix_trans(fh[c][1]); th[3] = movmatrix_trans(fh[c][3]);
+      tl[0] = movmatrix_trans(fl[c][0]); tl[1] = movmatrix_trans(fl[c][2]);
+      tl[2] = movmatrix_trans(fl[c][1]); tl[3] = movmatrix_trans(fl[c][3]);
+      mma16816(acc[c], th, ab0, ab1);
+      mma16816(acc[c], tl, ab0, ab1);
     }
   }
   // combine the warps of this block in a fixed order, write the chunk's partial
-  for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x) red[i] = 0.f;
-  __syncthreads();
   for (int w = 0; w < kPassWarps; ++w) {
     if (warp == w) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j)
-#pragma unroll
-        for (int r = 0; r < RP; ++r) red[(lane * 4 + j) * RP + r] += acc[j][r];
+      for (int c = 0; c < 8; ++c) {
+        const int ch = 16 * c + 4 * (gid >> 1) + (gid & 1);
+        red[ch * RP + t] += (acc[c][0] + acc[c][1]) * inv_acc;
+        red[(ch + 2) * RP + t] += (acc[c][2] + acc[c][3]) * inv_acc;
+      }
     }
     __syncthreads();
   }
@@ -1034,10 +1097,9 @@ static cudaError_t launch_quant(const CompressArgs& a, int nbh, int kmax_needed,
 template <int MODE>
 static void launch_pass(const PiArgs& p, cudaStream_t st) {
   // Four rank columns per CTA; a higher rank is spread over gridDim.z CTAs that read the same chunk of R (the second
-  // reader finds it in L2).  With eight or sixteen columns per CTA the registers allow half the resident warps and
-  // the pass runs three times slower per byte.
+  // reader finds it in L2).
   dim3 grid(p.nchunk, p.ntiles, p.rank <= 4 ? 1 : (p.rank <= 8 ? 2 : 4));
-  pi_pass_kernel<4, MODE><<<grid, kPassWarps * 32, 0, st>>>(p);
+  pi_pass_kernel<MODE><<<grid, kPassWarps * 32, 0, st>>>(p);
 }
 
 size_t compress_workspace_bytes(int nbh, int n_c, int rank) {
@@ -1051,6 +1113,7 @@ size_t compress_workspace_bytes(int nbh, int n_c, int rank) {
   b += ntiles * n_c * kMaxRank * 4;               // A0
   b += ntiles * nchunk * 256 * 4;                 // Gp
   b += ntiles * 256 * 4;                          // W
+  b += ntiles * 4;                                // Rmax
   return b + 1024;
 }
 
@@ -1062,7 +1125,7 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
   PiArgs pa;
   pa.seg = sd; pa.arena = job.arena; pa.bh0 = bh0; pa.ntiles = (int)ntiles; pa.n_c = sd.n_c; pa.rank = sd.rank;
   pa.nchunk = nchunk;
-  pa.R = nullptr; pa.Bcur = nullptr; pa.Bp = nullptr; pa.A0 = nullptr; pa.Gp = nullptr; pa.W = nullptr;
+  pa.R = nullptr; pa.Rmax = nullptr; pa.Bcur = nullptr; pa.Bp = nullptr; pa.A0 = nullptr; pa.Gp = nullptr; pa.W = nullptr;
   pa.dbgA = job.dbgA; pa.dbgB = job.dbgB;
   if (sd.rank > 0) {
     pa.R = wsf;       wsf += ntiles * sd.n_c * kHeadDim;
@@ -1070,13 +1133,15 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
     pa.Bp = wsf;      wsf += ntiles * nchunk * kHeadDim * kMaxRank;
     pa.A0 = wsf;      wsf += ntiles * sd.n_c * kMaxRank;
     pa.Gp = wsf;      wsf += ntiles * nchunk * 256;
-    pa.W = wsf;
+    pa.W = wsf;       wsf += ntiles * 256;
+    pa.Rmax = reinterpret_cast<unsigned int*>(wsf);
+    if (cudaMemsetAsync(pa.Rmax, 0, ntiles * 4, st) != cudaSuccess) return cudaGetLastError();
   }
   CompressArgs ca;
   ca.seg = sd; ca.cc = job.cc; ca.arena = job.arena; ca.bh0 = bh0;
   ca.K = job.K + (size_t)bh0 * sd.n_c * kHeadDim;
   ca.V = job.V + (size_t)bh0 * sd.n_c * kHeadDim;
-  ca.R = pa.R;
+  ca.R = pa.R; ca.Rmax = pa.Rmax;
   const int kneed = sd.k_k > job.cc.k_v ? sd.k_k : job.cc.k_v;
   cudaError_t e = job.cc.bits == 2 ? launch_quant<2>(ca, nbh, kneed, st) : launch_quant<4>(ca, nbh, kneed, st);
   if (e != cudaSuccess) return e;

@@ -19,6 +19,7 @@ struct CompressArgs {
   const __half* K;      // [nbh][n_c][128], already offset to the first (batch, head) of the range
   const __half* V;
   float* R;             // residual workspace [nbh][2][n_c][128] or nullptr (rank 0)
+  unsigned int* Rmax;   // [nbh][2] bit patterns of max |R| per tile (zeroed before the launch), with R
   int bh0;              // first (batch, head) of the range, for addressing the records
 };
 
@@ -26,6 +27,7 @@ struct PiArgs {
   SegDesc seg;
   unsigned char* arena;
   float* R;             // [ntiles][n_c][128]
+  unsigned int* Rmax;   // [ntiles] bit pattern of the tile's largest |R|
   float* Bcur;          // [ntiles][128][16]
   float* Bp;            // [ntiles][nchunk][128][16]
   float* A0;            // [ntiles][n_c][16]
