@@ -268,6 +268,174 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
 }
 
 // ---------------------------------------------------------------------------
+// The same step for the common shape -- blocks of 64 tokens, value groups of 64 channels, one outlier per side and
+// group (s <= 3.1 %) -- with the group in registers: a thread owns one group (keys: a channel's 64 tokens, read as a
+// column; values: 64 consecutive channels of a token), walks it in fully unrolled loops, stores the residual itself and
+// leaves only the codes in shared memory, one byte each, transposed so that the packing step fetches the four codes
+// of an output byte row with one 32-bit load.  Every code, scale, outlier and residual is bit-identical to
+// quant_pack_kernel: the operations on a group are the same binary32 sequence.
+// ---------------------------------------------------------------------------
+constexpr int kFastLen = 64;
+constexpr int kCodePitchK = kHeadDim + 4;   // bytes per token row of the key codes  [token][channel]
+constexpr int kCodePitchV = kFastLen + 4;   // bytes per channel row of the value codes [channel][token]
+
+template <int BITS>
+__global__ void __launch_bounds__(128) quant_fast_kernel(CompressArgs p) {
+  constexpr int L = kFastLen, F = 8 / BITS;
+  __shared__ __align__(16) unsigned char codes[kHeadDim * kCodePitchV > L * kCodePitchK ? kHeadDim * kCodePitchV
+                                                                                      : L * kCodePitchK];
+  __shared__ unsigned int dmax_bits, smax_bits, rmax_bits;
+  const SegDesc& sd = p.seg;
+  const int side = blockIdx.z, bhl = blockIdx.y, blk = blockIdx.x, tid = threadIdx.x;
+  if (tid == 0) { dmax_bits = 0u; smax_bits = 0u; rmax_bits = 0u; }
+  const __half* X = (side == 0 ? p.K : p.V) + ((size_t)bhl * sd.n_c + (size_t)blk * L) * kHeadDim;
+  float* R = p.R ? p.R + (((size_t)bhl * 2 + side) * sd.n_c + (size_t)blk * L) * kHeadDim : nullptr;
+  unsigned char* rec = p.arena + sd.seg_base + (size_t)(p.bh0 + bhl) * sd.bh_stride + sd.bfac_bytes +
+                       (size_t)blk * sd.rec_bytes;
+  // element e of this thread's group sits at X[first + e * step]
+  const int first = side == 0 ? tid : (tid >> 1) * kHeadDim + (tid & 1) * L;
+  const int step = side == 0 ? kHeadDim : 1;
+
+  float x[L];
+  if (side == 0) {
+#pragma unroll
+    for (int e = 0; e < L; ++e) x[e] = __half2float(X[first + e * kHeadDim]);
+  } else {
+    const uint4* src = reinterpret_cast<const uint4*>(X + first);
+#pragma unroll
+    for (int q = 0; q < L / 8; ++q) {
+      const uint4 v = src[q];
+      const unsigned int w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+        x[8 * q + 2 * i] = f.x;
+        x[8 * q + 2 * i + 1] = f.y;
+      }
+    }
+  }
+  // Filter_s (Eq. 4), one entry per side: the largest and the smallest entry leave the group, the second largest and
+  // second smallest instances bound what is kept; ties go to the lower index
+  float max1 = -INFINITY, max2 = -INFINITY, min1 = INFINITY, min2 = INFINITY;
+#pragma unroll
+  for (int e = 0; e < L; ++e) {
+    max2 = fmaxf(max2, fminf(x[e], max1));
+    max1 = fmaxf(max1, x[e]);
+    min2 = fminf(min2, fmaxf(x[e], min1));
+    min1 = fminf(min1, x[e]);
+  }
+  int imax = 0, imin = 0;
+#pragma unroll
+  for (int e = L - 1; e >= 0; --e) {
+    imax = x[e] == max1 ? e : imax;
+    imin = x[e] == min1 ? e : imin;
+  }
+  if (imin == imax) imin = 1;               // all entries equal: the bottom entry is the next index
+  const float mn = min2, mx = max2;
+  // Eq. 2 on the kept entries: binary32, one rounding per operation
+  const float levels = (float)((1 << BITS) - 1);
+  const float range = __fsub_rn(mx, mn);
+  const float d32 = __fdiv_rn(range, levels);
+  const __half d16 = __float2half_rn(d32);
+  const float d = __half2float(d16);
+  const float inv = d != 0.f ? __fdiv_rn(1.0f, d) : 0.f;
+  float rmax = 0.f;
+  if (side == 0) {
+#pragma unroll
+    for (int e = 0; e < L; ++e) {
+      const bool out = e == imax || e == imin;
+      const float t = __fmul_rn(__fsub_rn(x[e], mn), inv);
+      float cf = fminf(fmaxf(rintf(t), 0.f), levels);
+      float resid = x[e] - fmaf(cf, d, mn);
+      if (out) { cf = 0.f; resid = 0.f; }
+      codes[e * kCodePitchK + tid] = (unsigned char)(int)cf;
+      if (R != nullptr) R[e * kHeadDim + tid] = resid;
+      rmax = fmaxf(rmax, fabsf(resid));
+    }
+  } else {
+    const int tok = tid >> 1, c0 = (tid & 1) * L;
+#pragma unroll
+    for (int q = 0; q < L / 4; ++q) {
+      float rr[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int e = 4 * q + i;
+        const bool out = e == imax || e == imin;
+        const float t = __fmul_rn(__fsub_rn(x[e], mn), inv);
+        float cf = fminf(fmaxf(rintf(t), 0.f), levels);
+        float resid = x[e] - fmaf(cf, d, mn);
+        if (out) { cf = 0.f; resid = 0.f; }
+        codes[(c0 + e) * kCodePitchV + tok] = (unsigned char)(int)cf;
+        rr[i] = resid;
+        rmax = fmaxf(rmax, fabsf(resid));
+      }
+      if (R != nullptr) *reinterpret_cast<float4*>(R + first + 4 * q) = make_float4(rr[0], rr[1], rr[2], rr[3]);
+    }
+  }
+  // the group's scale, zero point and its two outliers (in-group index ascending)
+  {
+    const __half vmax = X[first + imax * step], vmin = X[first + imin * step];
+    const bool max_first = imax < imin;
+    const __half2 ov = max_first ? __halves2half2(vmax, vmin) : __halves2half2(vmin, vmax);
+    const uchar2 oi = max_first ? make_uchar2((unsigned char)imax, (unsigned char)imin)
+                                : make_uchar2((unsigned char)imin, (unsigned char)imax);
+    reinterpret_cast<__half2*>(rec + (side == 0 ? sd.off_koval : sd.off_voval))[tid] = ov;
+    reinterpret_cast<uchar2*>(rec + (side == 0 ? sd.off_koidx : sd.off_voidx))[tid] = oi;
+    reinterpret_cast<__half2*>(rec + (side == 0 ? sd.off_kscale : sd.off_vscale))[tid] =
+        __halves2half2(d16, __float2half_rn(mn));
+    float dm = fmaxf(fabsf(__half2float(vmax) - mn), fabsf(__half2float(vmin) - mn));
+    float sm = d;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      dm = fmaxf(dm, __shfl_xor_sync(0xffffffffu, dm, o));
+      sm = fmaxf(sm, __shfl_xor_sync(0xffffffffu, sm, o));
+      rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
+    }
+    if ((tid & 31) == 0) {                   // non-negative floats order like their bit patterns
+      atomicMax(&dmax_bits, __float_as_uint(dm));
+      atomicMax(&smax_bits, __float_as_uint(sm));
+      atomicMax(&rmax_bits, __float_as_uint(rmax));
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    reinterpret_cast<float*>(rec)[side] = __uint_as_float(dmax_bits);
+    reinterpret_cast<float*>(rec)[2 + side] = __uint_as_float(smax_bits);
+    if (R != nullptr) atomicMax(p.Rmax + bhl * 2 + side, rmax_bits);
+  }
+  // pack the codes into mma-fragment order (code_coord_k / code_coord_v): the four codes of a byte row are neighbours
+  // in shared memory, a field of the word is one 32-bit load shifted into place
+  unsigned int* dst = reinterpret_cast<unsigned int*>(rec + (side == 0 ? sd.off_kcodes : sd.off_vcodes));
+  if (side == 0) {
+    constexpr int kWords = kSlab * kHeadDim * BITS / 32;            // words per slab
+    for (int li = tid; li < (L / kSlab) * kWords; li += 128) {
+      const int slab = li / kWords, wl = li % kWords;
+      const int w = wl & 3, lane = (wl >> 2) & 31, tau = wl >> 7;
+      const int tok = slab * kSlab + (lane >> 2) + 8 * (w & 1);
+      const int ch = 32 * F * tau + 16 * (w >> 1) + 4 * (lane & 3);
+      unsigned int word = 0;
+#pragma unroll
+      for (int j = 0; j < F; ++j)
+        word |= *reinterpret_cast<const unsigned int*>(&codes[tok * kCodePitchK + ch + 32 * j]) << (BITS * j);
+      dst[li] = word;
+    }
+  } else {
+    constexpr int kWords = 32 * kHeadDim * BITS / 32;               // words per 32-token chunk
+    for (int li = tid; li < (L / 32) * kWords; li += 128) {
+      const int chunk = li / kWords, wl = li % kWords;
+      const int w = wl & 3, lane = (wl >> 2) & 31, tau = wl >> 7;
+      const int ch = 16 * F * tau + (lane >> 2) + 8 * (w & 1);
+      const int tok = chunk * 32 + 16 * (w >> 1) + 4 * (lane & 3);
+      unsigned int word = 0;
+#pragma unroll
+      for (int j = 0; j < F; ++j)
+        word |= *reinterpret_cast<const unsigned int*>(&codes[(ch + 16 * j) * kCodePitchV + tok]) << (BITS * j);
+      dst[li] = word;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
 // Power iteration (Algorithm 2).  A "tile" is one (batch, head, K|V) residual
 // R_h [n_c, 128] in the workspace.  Factor buffers are [128][16] fp32, zero
 // beyond the rank.
@@ -1079,6 +1247,10 @@ static cudaError_t launch_quant(const CompressArgs& a, int nbh, int kmax_needed,
   const int T = a.seg.T;
   const size_t smem = round_up(T * kXPitch * 2, 16) + (size_t)T * kRPitch * 4;
   dim3 grid(a.seg.nblk, nbh, 2);
+  if (T == kFastLen && a.cc.g_v == kFastLen && a.seg.k_k == 1 && a.cc.k_v == 1) {
+    quant_fast_kernel<BITS><<<grid, 128, 0, st>>>(a);
+    return cudaGetLastError();
+  }
 #define GEAR_LAUNCH_Q(KM)                                                                                   \
   {                                                                                                         \
     cudaError_t e = cudaFuncSetAttribute(quant_pack_kernel<BITS, KM>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
