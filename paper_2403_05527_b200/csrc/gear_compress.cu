@@ -279,14 +279,24 @@ constexpr int kFastLen = 64;
 constexpr int kCodePitchK = kHeadDim + 4;   // bytes per token row of the key codes  [token][channel]
 constexpr int kCodePitchV = kFastLen + 4;   // bytes per channel row of the value codes [channel][token]
 
-template <int BITS>
+// Value side, shared-memory staging (a thread's 64 channels are contiguous in memory, so direct accesses of a warp
+// would touch 32 lines each): the fp16 tile comes in with coalesced loads, the fp32 residual tile leaves the same way.
+// Row (c, token) of the fp16 tile holds the 64 channels of group c; rows are 36 words apart and the second group
+// starts 16 words late, rows of the residual tile are 164 words with group 1 at word 80: both make the 128-bit
+// accesses of a quarter warp (four tokens x two groups) hit 32 different banks.
+constexpr int kStageRowWords = 36, kStageGroupSkew = 16;
+constexpr int kResPitch = 164, kResGroup = 80;
+constexpr int kFastSmemV = kFastLen * kResPitch * 4;     // the residual tile; the fp16 tile lives in it first
+
+template <int BITS, int SIDE>
 __global__ void __launch_bounds__(128) quant_fast_kernel(CompressArgs p) {
   constexpr int L = kFastLen, F = 8 / BITS;
-  __shared__ __align__(16) unsigned char codes[kHeadDim * kCodePitchV > L * kCodePitchK ? kHeadDim * kCodePitchV
-                                                                                      : L * kCodePitchK];
+  constexpr int side = SIDE;
+  extern __shared__ __align__(16) unsigned char stage_raw[];    // value side only
+  __shared__ __align__(16) unsigned char codes[SIDE == 0 ? L * kCodePitchK : kHeadDim * kCodePitchV];
   __shared__ unsigned int dmax_bits, smax_bits, rmax_bits;
   const SegDesc& sd = p.seg;
-  const int side = blockIdx.z, bhl = blockIdx.y, blk = blockIdx.x, tid = threadIdx.x;
+  const int bhl = blockIdx.y, blk = blockIdx.x, tid = threadIdx.x;
   if (tid == 0) { dmax_bits = 0u; smax_bits = 0u; rmax_bits = 0u; }
   const __half* X = (side == 0 ? p.K : p.V) + ((size_t)bhl * sd.n_c + (size_t)blk * L) * kHeadDim;
   float* R = p.R ? p.R + (((size_t)bhl * 2 + side) * sd.n_c + (size_t)blk * L) * kHeadDim : nullptr;
@@ -295,40 +305,72 @@ __global__ void __launch_bounds__(128) quant_fast_kernel(CompressArgs p) {
   // element e of this thread's group sits at X[first + e * step]
   const int first = side == 0 ? tid : (tid >> 1) * kHeadDim + (tid & 1) * L;
   const int step = side == 0 ? kHeadDim : 1;
+  float* rs = reinterpret_cast<float*>(stage_raw);
 
-  float x[L];
+  // the group as 32 packed pairs (entries 2q, 2q + 1)
+  __half2 xp[L / 2];
   if (side == 0) {
 #pragma unroll
-    for (int e = 0; e < L; ++e) x[e] = __half2float(X[first + e * kHeadDim]);
+    for (int q = 0; q < L / 2; ++q) xp[q] = __halves2half2(X[first + (2 * q) * kHeadDim], X[first + (2 * q + 1) * kHeadDim]);
   } else {
-    const uint4* src = reinterpret_cast<const uint4*>(X + first);
+    uint4* xs = reinterpret_cast<uint4*>(stage_raw);
+    for (int i = tid; i < L * 16; i += 128) {           // 16-byte pieces of the tile, in memory order
+      const int tok = i >> 4, c = (i >> 3) & 1, q = i & 7;
+      xs[(((c * L + tok) * kStageRowWords + c * kStageGroupSkew) >> 2) + q] = reinterpret_cast<const uint4*>(X)[i];
+    }
+    __syncthreads();
+    const int tok = tid >> 1, c = tid & 1;
+    const uint4* src = xs + (((c * L + tok) * kStageRowWords + c * kStageGroupSkew) >> 2);
 #pragma unroll
     for (int q = 0; q < L / 8; ++q) {
       const uint4 v = src[q];
-      const unsigned int w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
-        x[8 * q + 2 * i] = f.x;
-        x[8 * q + 2 * i + 1] = f.y;
-      }
+      xp[4 * q] = *reinterpret_cast<const __half2*>(&v.x);
+      xp[4 * q + 1] = *reinterpret_cast<const __half2*>(&v.y);
+      xp[4 * q + 2] = *reinterpret_cast<const __half2*>(&v.z);
+      xp[4 * q + 3] = *reinterpret_cast<const __half2*>(&v.w);
     }
+    __syncthreads();                                     // the residual tile takes the place of the fp16 tile
   }
   // Filter_s (Eq. 4), one entry per side: the largest and the smallest entry leave the group, the second largest and
-  // second smallest instances bound what is kept; ties go to the lower index
-  float max1 = -INFINITY, max2 = -INFINITY, min1 = INFINITY, min2 = INFINITY;
+  // second smallest instances bound what is kept.  Comparisons of fp16 values are exact in fp16, so the search runs on
+  // the packed pairs: even and odd entries keep their own two largest / smallest and are merged at the end.
+  float max1, max2, min1, min2;
+  {
+    const __half2 ninf = __float2half2_rn(-INFINITY), pinf = __float2half2_rn(INFINITY);
+    __half2 M1 = ninf, M2 = ninf, m1 = pinf, m2 = pinf;
 #pragma unroll
-  for (int e = 0; e < L; ++e) {
-    max2 = fmaxf(max2, fminf(x[e], max1));
-    max1 = fmaxf(max1, x[e]);
-    min2 = fminf(min2, fmaxf(x[e], min1));
-    min1 = fminf(min1, x[e]);
+    for (int q = 0; q < L / 2; ++q) {
+      M2 = __hmax2(M2, __hmin2(xp[q], M1));
+      M1 = __hmax2(M1, xp[q]);
+      m2 = __hmin2(m2, __hmax2(xp[q], m1));
+      m1 = __hmin2(m1, xp[q]);
+    }
+    const float2 fM1 = __half22float2(M1), fM2 = __half22float2(M2), fm1 = __half22float2(m1), fm2 = __half22float2(m2);
+    max1 = fmaxf(fM1.x, fM1.y);
+    max2 = fmaxf(fminf(fM1.x, fM1.y), fmaxf(fM2.x, fM2.y));
+    min1 = fminf(fm1.x, fm1.y);
+    min2 = fminf(fmaxf(fm1.x, fm1.y), fminf(fm2.x, fm2.y));
   }
-  int imax = 0, imin = 0;
+  // first index of the maximum and of the minimum (ties go to the lower index): one mask bit per entry
+  int imax, imin;
+  {
+    const __half2 vM = __float2half2_rn(max1), vm = __float2half2_rn(min1);
+    unsigned int a0 = 0u, a1 = 0u, b0 = 0u, b1 = 0u;   // bit q of a half word: pair q (a0, b0) or pair 16 + q (a1, b1)
 #pragma unroll
-  for (int e = L - 1; e >= 0; --e) {
-    imax = x[e] == max1 ? e : imax;
-    imin = x[e] == min1 ? e : imin;
+    for (int q = 0; q < L / 2; ++q) {
+      const unsigned int bit = 0x00010001u << (q & 15);
+      const unsigned int eM = __heq2_mask(xp[q], vM) & bit, em = __heq2_mask(xp[q], vm) & bit;
+      if (q < 16) { a0 |= eM; b0 |= em; } else { a1 |= eM; b1 |= em; }
+    }
+    auto first_set = [](unsigned int lo16, unsigned int hi16) {
+      const unsigned int even = __byte_perm(lo16, hi16, 0x5410);   // bit q: entry 2 q
+      const unsigned int odd = __byte_perm(lo16, hi16, 0x7632);    // bit q: entry 2 q + 1
+      const int fe = even ? 2 * (__ffs((int)even) - 1) : L;
+      const int fo = odd ? 2 * (__ffs((int)odd) - 1) + 1 : L;
+      return min(fe, fo);
+    };
+    imax = first_set(a0, a1);
+    imin = first_set(b0, b1);
   }
   if (imin == imax) imin = 1;               // all entries equal: the bottom entry is the next index
   const float mn = min2, mx = max2;
@@ -339,39 +381,57 @@ __global__ void __launch_bounds__(128) quant_fast_kernel(CompressArgs p) {
   const __half d16 = __float2half_rn(d32);
   const float d = __half2float(d16);
   const float inv = d != 0.f ? __fdiv_rn(1.0f, d) : 0.f;
-  float rmax = 0.f;
+  // Codes and residuals are computed for every entry as if it were kept; the two filtered entries are cleared
+  // afterwards.  round-to-nearest-even of the clamped quotient by adding 1.5 * 2^23: the code is the low byte of the sum.
+  constexpr float kRound = 12582912.0f;
+  auto quantize = [&](float x, unsigned int& code) {
+    const float t = __fmul_rn(__fsub_rn(x, mn), inv);
+    const float y = __fadd_rn(fminf(fmaxf(t, 0.f), levels), kRound);
+    code = __float_as_uint(y) & 0xFFu;
+    return x - fmaf(__fsub_rn(y, kRound), d, mn);
+  };
   if (side == 0) {
 #pragma unroll
-    for (int e = 0; e < L; ++e) {
-      const bool out = e == imax || e == imin;
-      const float t = __fmul_rn(__fsub_rn(x[e], mn), inv);
-      float cf = fminf(fmaxf(rintf(t), 0.f), levels);
-      float resid = x[e] - fmaf(cf, d, mn);
-      if (out) { cf = 0.f; resid = 0.f; }
-      codes[e * kCodePitchK + tid] = (unsigned char)(int)cf;
-      if (R != nullptr) R[e * kHeadDim + tid] = resid;
-      rmax = fmaxf(rmax, fabsf(resid));
+    for (int q = 0; q < L / 2; ++q) {
+      const float2 f = __half22float2(xp[q]);
+      unsigned int c0, c1;
+      const float r0 = quantize(f.x, c0), r1 = quantize(f.y, c1);
+      codes[(2 * q) * kCodePitchK + tid] = (unsigned char)c0;
+      codes[(2 * q + 1) * kCodePitchK + tid] = (unsigned char)c1;
+      if (R != nullptr) {
+        R[(2 * q) * kHeadDim + tid] = r0;
+        R[(2 * q + 1) * kHeadDim + tid] = r1;
+      }
+    }
+    codes[imax * kCodePitchK + tid] = 0;
+    codes[imin * kCodePitchK + tid] = 0;
+    if (R != nullptr) {
+      R[imax * kHeadDim + tid] = 0.f;
+      R[imin * kHeadDim + tid] = 0.f;
     }
   } else {
     const int tok = tid >> 1, c0 = (tid & 1) * L;
+    float* rrow = rs + tok * kResPitch + (tid & 1) * kResGroup;
 #pragma unroll
     for (int q = 0; q < L / 4; ++q) {
-      float rr[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int e = 4 * q + i;
-        const bool out = e == imax || e == imin;
-        const float t = __fmul_rn(__fsub_rn(x[e], mn), inv);
-        float cf = fminf(fmaxf(rintf(t), 0.f), levels);
-        float resid = x[e] - fmaf(cf, d, mn);
-        if (out) { cf = 0.f; resid = 0.f; }
-        codes[(c0 + e) * kCodePitchV + tok] = (unsigned char)(int)cf;
-        rr[i] = resid;
-        rmax = fmaxf(rmax, fabsf(resid));
-      }
-      if (R != nullptr) *reinterpret_cast<float4*>(R + first + 4 * q) = make_float4(rr[0], rr[1], rr[2], rr[3]);
+      const float2 f0 = __half22float2(xp[2 * q]), f1 = __half22float2(xp[2 * q + 1]);
+      unsigned int k0, k1, k2, k3;
+      const float4 rr = make_float4(quantize(f0.x, k0), quantize(f0.y, k1), quantize(f1.x, k2), quantize(f1.y, k3));
+      codes[(c0 + 4 * q) * kCodePitchV + tok] = (unsigned char)k0;
+      codes[(c0 + 4 * q + 1) * kCodePitchV + tok] = (unsigned char)k1;
+      codes[(c0 + 4 * q + 2) * kCodePitchV + tok] = (unsigned char)k2;
+      codes[(c0 + 4 * q + 3) * kCodePitchV + tok] = (unsigned char)k3;
+      *reinterpret_cast<float4*>(rrow + 4 * q) = rr;
     }
+    codes[(c0 + imax) * kCodePitchV + tok] = 0;
+    codes[(c0 + imin) * kCodePitchV + tok] = 0;
+    rrow[imax] = 0.f;
+    rrow[imin] = 0.f;
   }
+  // A bound on the group's residuals instead of their maximum (it only picks the power of two the power iteration
+  // scales by): half a step for a kept entry, the whole range if the step rounded to zero, plus the rounding of the
+  // dequantised value
+  float rmax = (d != 0.f ? 0.50390625f * d : range) + 2.4e-7f * (fabsf(mn) + fabsf(mx));
   // the group's scale, zero point and its two outliers (in-group index ascending)
   {
     const __half vmax = X[first + imax * step], vmin = X[first + imin * step];
@@ -402,6 +462,12 @@ __global__ void __launch_bounds__(128) quant_fast_kernel(CompressArgs p) {
     reinterpret_cast<float*>(rec)[side] = __uint_as_float(dmax_bits);
     reinterpret_cast<float*>(rec)[2 + side] = __uint_as_float(smax_bits);
     if (R != nullptr) atomicMax(p.Rmax + bhl * 2 + side, rmax_bits);
+  }
+  if (side == 1 && R != nullptr) {
+    for (int i = tid; i < L * 32; i += 128) {            // 16-byte pieces of the residual tile, in memory order
+      const int tok = i >> 5, c = (i >> 4) & 1, q = i & 15;
+      reinterpret_cast<float4*>(R)[i] = *reinterpret_cast<const float4*>(rs + tok * kResPitch + c * kResGroup + 4 * q);
+    }
   }
   // pack the codes into mma-fragment order (code_coord_k / code_coord_v): the four codes of a byte row are neighbours
   // in shared memory, a field of the word is one 32-bit load shifted into place
@@ -1242,13 +1308,23 @@ __global__ void append_kernel(__half* buf_k, __half* buf_v, const __half* k_new,
 // ---------------------------------------------------------------------------
 // host side: launch sequence for a range of (batch, head) pairs
 // ---------------------------------------------------------------------------
+// the shape quant_fast_kernel is written for (two launches, keys then values)
+static bool quant_is_fast(const SegDesc& sd, const CacheConst& cc) {
+  return sd.T == kFastLen && cc.g_v == kFastLen && sd.k_k == 1 && cc.k_v == 1;
+}
+
 template <int BITS>
 static cudaError_t launch_quant(const CompressArgs& a, int nbh, int kmax_needed, cudaStream_t st) {
   const int T = a.seg.T;
   const size_t smem = round_up(T * kXPitch * 2, 16) + (size_t)T * kRPitch * 4;
   dim3 grid(a.seg.nblk, nbh, 2);
-  if (T == kFastLen && a.cc.g_v == kFastLen && a.seg.k_k == 1 && a.cc.k_v == 1) {
-    quant_fast_kernel<BITS><<<grid, 128, 0, st>>>(a);
+  if (quant_is_fast(a.seg, a.cc)) {
+    cudaError_t e = cudaFuncSetAttribute(quant_fast_kernel<BITS, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kFastSmemV);
+    if (e != cudaSuccess) return e;
+    grid.z = 1;
+    quant_fast_kernel<BITS, 0><<<grid, 128, 0, st>>>(a);
+    quant_fast_kernel<BITS, 1><<<grid, 128, kFastSmemV, st>>>(a);
     return cudaGetLastError();
   }
 #define GEAR_LAUNCH_Q(KM)                                                                                   \
@@ -1317,7 +1393,7 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
   const int kneed = sd.k_k > job.cc.k_v ? sd.k_k : job.cc.k_v;
   cudaError_t e = job.cc.bits == 2 ? launch_quant<2>(ca, nbh, kneed, st) : launch_quant<4>(ca, nbh, kneed, st);
   if (e != cudaSuccess) return e;
-  count_launches(1);
+  count_launches(quant_is_fast(sd, job.cc) ? 2 : 1);
   if (sd.rank == 0) return cudaSuccess;
   // init + per early loop (pass, reduce) + last loop (pass, gram, chol, gram, chol, store, reduce)
   count_launches(1 + 2 * (job.iters - 1) + 7 + (job.iters == 1 ? 1 : 0));
