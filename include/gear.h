@@ -61,6 +61,8 @@ typedef void* (*gear_alloc_fn)(size_t bytes, void* ctx);
 typedef void (*gear_free_fn)(void* ptr, void* ctx);
 
 /* Hyper-parameters in the paper's notation (Section 2 and 3; Algorithm 1, 2). */
+#define GEAR_GROUP_PER_VECTOR 0
+
 typedef struct gear_config {
   int32_t batch;        /* sequences in the batch                                              */
   int32_t n_q_heads;    /* H_q query heads; n_q_heads % n_kv_heads == 0                        */
@@ -69,7 +71,13 @@ typedef struct gear_config {
   int32_t bits;         /* b in {2, 4}                                                           */
   int32_t group;        /* g in {16, 32, 64, 128}: keys are grouped per channel over
                            min(g, n_c) consecutive tokens of a segment, values per token over
-                           min(g, d_H) consecutive channels (KIVI grouping, Section 2)          */
+                           min(g, d_H) consecutive channels (KIVI grouping, Section 2).
+                           GEAR_GROUP_PER_VECTOR: the per-vector grouping of the same section (KCVT):
+                           one key group per channel over all tokens of a segment, one value group
+                           per token; Filter_s then acts on those whole vectors, so a channel of an
+                           n-token segment gives up ceil(s n / 200) entries per side (any count
+                           below n / 2).  Needs buffer_cap <= 128; segments longer than 128 tokens
+                           must be multiples of 64 and at most 8192 tokens long.                  */
   float   outlier_pct;  /* s in percent, 0 <= s <= 10.  Filter_s (Eq. 4) takes
                            k = ceil(s * len / 200) largest and k smallest entries of every
                            group of length len; need k <= 8 and 2k < len                        */

@@ -208,7 +208,7 @@ def compress_tile(x16: np.ndarray, kind: str, bits: int, g: int, s_pct: float,
     Returns a dict with the canonical (unpacked) pieces:
       codes u8 [n_c, d_H]; scale, zero fp16 ('K': [n_c/g_K, d_H]; 'V': [n_c, d_H/g_V]);
       mask bool [n_c, d_H] (support of S); S float64 (exact fp16 values on the mask);
-      out_idx u8 / out_val fp16 [n_groups, 2k] (in-group index ascending);
+      out_idx u8 (int32 for groups longer than 256) / out_val fp16 [n_groups, 2k] (in-group index ascending);
       D float64 (dequantised backbone, 0 on the mask); R; A [n_c, r]; B [d_H, r]."""
     x16 = np.asarray(x16, dtype=F16)
     n_c, d_h = x16.shape
@@ -243,7 +243,8 @@ def compress_tile(x16: np.ndarray, kind: str, bits: int, g: int, s_pct: float,
     resid = x - d_hat - s_mat                                      # R = X - (D^ + S)
 
     if k and (filter_len is None or filter_len == g_len):
-        out_idx = np.nonzero(gmask)[1].reshape(-1, 2 * k).astype(np.uint8)   # ascending per group
+        idx_t = np.uint8 if g_len <= 256 else np.int32                       # an index inside a long vector needs more than a byte
+        out_idx = np.nonzero(gmask)[1].reshape(-1, 2 * k).astype(idx_t)      # ascending per group
         out_val = gr[gmask].reshape(-1, 2 * k).astype(F16)
     else:                                        # none, or a varying number per group: the mask and S carry them
         out_idx = np.zeros((gr.shape[0], 0), np.uint8)

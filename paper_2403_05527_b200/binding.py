@@ -291,7 +291,9 @@ def gear_export(cache, segment: int, what: str, batch: int, n_kv_heads: int):
         elif base in ("OUT_IDX", "OUT_VAL"):
             shape = ((batch, n_kv_heads, n_c // si.g_k, 128, 2 * si.k_k) if side_k
                      else (batch, n_kv_heads, n_c, 128 // si.g_v, 2 * si.k_v))
-            arr = np.empty(shape, np.uint8 if base == "OUT_IDX" else np.float16)
+            # a key group longer than 128 tokens (per-vector grouping): token indices come as 32-bit integers
+            idx_t = np.int32 if side_k and si.g_k > 128 else np.uint8
+            arr = np.empty(shape, idx_t if base == "OUT_IDX" else np.float16)
         elif base in ("A", "A_FP32"):
             arr = np.empty((batch, n_kv_heads, n_c, r), np.float32)
         elif base in ("B", "B_FP32"):

@@ -14,7 +14,8 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libgear_b200.so")
 STAMP = os.path.join(HERE, "libgear_b200.stamp")
-SOURCES = ["gear_api.cu", "gear_compress.cu", "gear_decode.cu", "gear_export.cu", "gear_fp16_attn.cu"]
+SOURCES = ["gear_api.cu", "gear_compress.cu", "gear_decode.cu", "gear_export.cu", "gear_fp16_attn.cu",
+           "gear_kcvt.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "--threads", "0"]
 

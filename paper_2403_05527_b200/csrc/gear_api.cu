@@ -129,19 +129,20 @@ static gear_status check_config(const gear_config* c) {
   if (c->n_q_heads % c->n_kv_heads) return GEAR_ERR_SHAPE;
   if (c->head_dim != kHeadDim) return GEAR_ERR_SHAPE;
   if (c->bits != 2 && c->bits != 4) return GEAR_ERR_ARG;
-  if (c->group != 16 && c->group != 32 && c->group != 64 && c->group != 128) return GEAR_ERR_ARG;
+  const bool per_vector = c->group == GEAR_GROUP_PER_VECTOR;
+  if (!per_vector && c->group != 16 && c->group != 32 && c->group != 64 && c->group != 128) return GEAR_ERR_ARG;
   if (!(c->outlier_pct >= 0.f) || c->outlier_pct > 10.f) return GEAR_ERR_ARG;
   if (c->buffer_cap < 16 || c->buffer_cap % 16 || c->buffer_cap > 1024) return GEAR_ERR_ARG;
-  if (c->buffer_cap > c->group && c->buffer_cap % c->group) return GEAR_ERR_SHAPE;
+  if (per_vector ? c->buffer_cap > 128 : (c->buffer_cap > c->group && c->buffer_cap % c->group)) return GEAR_ERR_SHAPE;
   if (c->rank_flush < 0 || c->rank_flush > kMaxRank || c->rank_max < 0 || c->rank_max > kMaxRank) return GEAR_ERR_ARG;
   if (c->rank_flush > c->rank_max) return GEAR_ERR_ARG;
   if (c->rank_flush > c->buffer_cap) return GEAR_ERR_SHAPE;
   if (c->max_queries > 64) return GEAR_ERR_ARG;
   if (c->power_iters < 1 || c->power_iters > 64) return GEAR_ERR_ARG;
-  const int gv = c->group < kHeadDim ? c->group : kHeadDim;
+  const int gv = per_vector || c->group > kHeadDim ? kHeadDim : c->group;
   const int kv = outlier_count(c->outlier_pct, gv);
   if (kv > kMaxOutliers || (kv > 0 && 2 * kv >= gv)) return GEAR_ERR_SHAPE;
-  const int tf = c->buffer_cap < c->group ? c->buffer_cap : c->group;
+  const int tf = per_vector || c->buffer_cap < c->group ? c->buffer_cap : c->group;
   const int kf = outlier_count(c->outlier_pct, tf);
   if (kf > kMaxOutliers || (kf > 0 && 2 * kf >= tf)) return GEAR_ERR_SHAPE;
   return GEAR_OK;
@@ -151,9 +152,18 @@ static SegDesc shape_segment(const gear_cache* c, int n_c, int rank) {
   SegDesc s;
   memset(&s, 0, sizeof(s));
   s.n_c = n_c;
-  s.T = n_c < c->cfg.group ? n_c : c->cfg.group;
   s.rank = rank;
-  s.k_k = outlier_count(c->cfg.outlier_pct, s.T);
+  if (c->cfg.group == GEAR_GROUP_PER_VECTOR && n_c > 128) {
+    // one key group per channel over the whole segment: 64-token record blocks without outlier slots, the
+    // outliers in a list behind the records (csr_base16 is set when the segment is placed)
+    s.T = 64;
+    s.k_k = 0;
+    s.csr_k = 2 * outlier_count(c->cfg.outlier_pct, n_c);
+    s.csr_base16 = 1;
+  } else {
+    s.T = c->cfg.group == GEAR_GROUP_PER_VECTOR || n_c < c->cfg.group ? n_c : c->cfg.group;
+    s.k_k = outlier_count(c->cfg.outlier_pct, s.T);
+  }
   layout_segment(s, c->cc);
   return s;
 }
@@ -198,7 +208,7 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   for (int i = 0; i < gear_cache::kHostSlots; ++i) { c->host_ring[i] = nullptr; c->host_ev[i] = nullptr; c->host_used[i] = false; }
   c->host_next = 0;
   c->cc.bits = cfg->bits;
-  c->cc.g_v = cfg->group < kHeadDim ? cfg->group : kHeadDim;
+  c->cc.g_v = cfg->group == GEAR_GROUP_PER_VECTOR || cfg->group > kHeadDim ? kHeadDim : cfg->group;
   c->cc.ngv = kHeadDim / c->cc.g_v;
   c->cc.k_v = outlier_count(cfg->outlier_pct, c->cc.g_v);
   c->cc.BH = cfg->batch * cfg->n_kv_heads;
@@ -214,13 +224,17 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   // arena: worst bytes per token over the two segment shapes the cache can see (full groups at rank_max,
   // flushed buffers at rank_flush), plus the per-segment B factors
   const int n_b = cfg->buffer_cap;
-  SegDesc sp = shape_segment(c, cfg->group, cfg->rank_max);
+  const bool per_vector = cfg->group == GEAR_GROUP_PER_VECTOR;
+  SegDesc sp = shape_segment(c, per_vector ? 192 : cfg->group, cfg->rank_max);
   SegDesc sf = shape_segment(c, n_b, cfg->rank_flush);
   const double dens_p = (double)sp.rec_bytes / sp.T, dens_f = (double)sf.rec_bytes / sf.T;
   const double dens = dens_p > dens_f ? dens_p : dens_f;
   const size_t n_flush_max = (size_t)(cfg->max_tokens / n_b) + 1;
   size_t per_bh = (size_t)(dens * (double)cfg->max_tokens) + n_flush_max * sf.bfac_bytes + 8 * (size_t)sp.bfac_bytes +
                   16 * (size_t)(sp.rec_bytes > sf.rec_bytes ? sp.rec_bytes : sf.rec_bytes);
+  if (per_vector)      // outlier lists of per-vector key segments: offsets per block, entries per channel (rounded up per segment)
+    per_bh += (size_t)(cfg->max_tokens / 64 + 8) * 4 + 64 * 16 +
+              (size_t)kHeadDim * 4 * (2 * (size_t)outlier_count(cfg->outlier_pct, (int)cfg->max_tokens) + 2 * 8);
   c->arena_bytes = align_up(per_bh, 256) * BH + 4096;
   c->arena_used = 0;
   GEAR_TRY_ALLOC(c->arena, c->arena_bytes);
@@ -280,8 +294,14 @@ static gear_status compress_segment(gear_cache* c, const void* K, const void* V,
   SegDesc sd = shape_segment(c, n, rank);
   if (c->n_blocks_c + sd.nblk > c->blk_cap) return GEAR_ERR_CAPACITY;
   if (sd.k_k > kMaxOutliers || (sd.k_k > 0 && 2 * sd.k_k >= sd.T)) return GEAR_ERR_SHAPE;
-  const size_t need = align_up((size_t)sd.bh_stride, 16) * c->cc.BH;
+  size_t need = align_up((size_t)sd.bh_stride, 16) * c->cc.BH;
   sd.bh_stride = (long long)align_up((size_t)sd.bh_stride, 16);
+  const bool per_vector = sd.csr_base16 != 0;
+  if (per_vector) {
+    if (!kcvt_fits(n) || sd.csr_k >= n || (need >> 4) > 0xFFFFFFFFull) return GEAR_ERR_SHAPE;
+    sd.csr_base16 = (unsigned int)(need >> 4);
+    need += align_up((size_t)csr_stride_bytes(sd.nblk, sd.csr_k) * c->cc.BH, 16);
+  }
   if (c->arena_used + need > c->arena_bytes) return GEAR_ERR_CAPACITY;
   sd.seg_base = (long long)c->arena_used;
   sd.tok_start = (int)c->n_compressed;
@@ -303,19 +323,20 @@ static gear_status compress_segment(gear_cache* c, const void* K, const void* V,
   job.seed = c->cfg.seed; job.segment_index = (int)c->segs.size(); job.iters = c->cfg.power_iters;
 
   cudaError_t e = cudaSuccess;
-  if (compress_tile_fits(sd.T, sd.n_c, sd.rank)) {
+  if (!per_vector && compress_tile_fits(sd.T, sd.n_c, sd.rank)) {
     e = compress_tile(job, c->cc.BH, st);              // short segment: one launch, residual in shared memory
   } else if (is_flush) {
     e = compress_range(job, 0, c->cc.BH, c->flush_ws, st);
   } else {
     // bounded transient workspace, (batch, head) pairs processed in ranges
-    const size_t per_bh = compress_workspace_bytes(1, n, rank);
+    const int csr_k = per_vector ? sd.csr_k : -1;
+    const size_t per_bh = compress_workspace_bytes(1, n, rank, csr_k);
     const size_t budget = (size_t)3 << 30;
     int chunk = (int)(budget / per_bh);
     if (chunk < 1) chunk = 1;
     if (chunk > c->cc.BH) chunk = c->cc.BH;
     unsigned char* ws = nullptr;
-    const size_t ws_bytes = compress_workspace_bytes(chunk, n, rank);
+    const size_t ws_bytes = compress_workspace_bytes(chunk, n, rank, csr_k);
     cudaMemPool_t pool = workspace_pool(c->device);
     if (pool == nullptr || cudaMallocFromPoolAsync((void**)&ws, ws_bytes, pool, st) != cudaSuccess) {
       cudaGetLastError();
@@ -349,7 +370,7 @@ extern "C" gear_status gear_compress(gear_cache** cache, const gear_config* cfg,
   gear_status st = check_config(use);
   if (st != GEAR_OK) return st;
   if (n < 16 || n % 16 || n > (1 << 30)) return GEAR_ERR_SHAPE;
-  if (n >= use->group && n % use->group) return GEAR_ERR_SHAPE;
+  if (use->group == GEAR_GROUP_PER_VECTOR ? (n > 128 && n % 64) : (n >= use->group && n % use->group)) return GEAR_ERR_SHAPE;
   if (rank < 0 || rank > use->rank_max || rank > n) return GEAR_ERR_ARG;
   bool created = false;
   if (!*cache) {
@@ -592,10 +613,12 @@ static size_t export_elems(const gear_cache* c, const SegDesc& s, int what, size
   const size_t BH = c->cc.BH, d = kHeadDim;
   switch (what) {
     case GEAR_EXP_K_CODES: case GEAR_EXP_V_CODES: *elem_bytes = 1; return BH * s.n_c * d;
-    case GEAR_EXP_K_SCALE: case GEAR_EXP_K_ZERO: *elem_bytes = 2; return BH * s.nblk * d;
+    case GEAR_EXP_K_SCALE: case GEAR_EXP_K_ZERO: *elem_bytes = 2; return BH * (s.csr_base16 ? 1 : s.nblk) * d;
     case GEAR_EXP_V_SCALE: case GEAR_EXP_V_ZERO: *elem_bytes = 2; return BH * s.n_c * c->cc.ngv;
-    case GEAR_EXP_K_OUT_IDX: *elem_bytes = 1; return BH * s.nblk * d * 2 * s.k_k;
-    case GEAR_EXP_K_OUT_VAL: *elem_bytes = 2; return BH * s.nblk * d * 2 * s.k_k;
+    case GEAR_EXP_K_OUT_IDX:
+      if (s.csr_base16) { *elem_bytes = 4; return BH * d * s.csr_k; }      // token in the segment, 32-bit
+      *elem_bytes = 1; return BH * s.nblk * d * 2 * s.k_k;
+    case GEAR_EXP_K_OUT_VAL: *elem_bytes = 2; return s.csr_base16 ? BH * d * s.csr_k : BH * s.nblk * d * 2 * s.k_k;
     case GEAR_EXP_V_OUT_IDX: *elem_bytes = 1; return BH * s.n_c * c->cc.ngv * 2 * c->cc.k_v;
     case GEAR_EXP_V_OUT_VAL: *elem_bytes = 2; return BH * s.n_c * c->cc.ngv * 2 * c->cc.k_v;
     case GEAR_EXP_K_A: case GEAR_EXP_V_A: case GEAR_EXP_K_A_FP32: case GEAR_EXP_V_A_FP32:
@@ -668,6 +691,7 @@ extern "C" gear_status gear_segment_info_get(const gear_cache* c, int32_t segmen
   if (!c || !info || segment < 0 || segment >= (int)c->segs.size()) return GEAR_ERR_ARG;
   const SegDesc& s = c->segs[segment];
   info->n_c = s.n_c; info->rank = s.rank; info->g_k = s.T; info->g_v = c->cc.g_v; info->k_k = s.k_k; info->k_v = c->cc.k_v;
+  if (s.csr_base16 != 0) { info->g_k = s.n_c; info->k_k = s.csr_k / 2; }      // per-vector keys: the whole segment
   return GEAR_OK;
 }
 
@@ -682,6 +706,11 @@ extern "C" gear_status gear_cache_bytes(const gear_cache* c, gear_bytes* out) {
     out->lowrank_a += BH * 2 * (long long)s.n_c * s.rank * 2;
     out->lowrank_b += BH * 2 * d * s.rank * 2;
     out->stored_total += BH * s.bh_stride;
+    if (s.csr_base16 != 0) {     // per-vector keys: the list of the segment's key outliers (the records repeat the scales)
+      const long long list = BH * (long long)csr_stride_bytes(s.nblk, s.csr_k);
+      out->outliers += list;
+      out->stored_total += list;
+    }
   }
   out->buffer = BH * 2 * (long long)c->buf_len * d * 2;
   out->stored_total += out->buffer;

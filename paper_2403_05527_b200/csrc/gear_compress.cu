@@ -189,7 +189,7 @@ __global__ void __launch_bounds__(128) quant_pack_kernel(CompressArgs p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const SegDesc& sd = p.seg;
   const int T = sd.T;
-  const int side = blockIdx.z, bhl = blockIdx.y, blk = blockIdx.x, tid = threadIdx.x;
+  const int side = blockIdx.z + p.side0, bhl = blockIdx.y, blk = blockIdx.x, tid = threadIdx.x;
   unsigned short* xs = reinterpret_cast<unsigned short*>(smem_raw);   // fp16 bits of the block; each entry is replaced by its code
   float* rs = reinterpret_cast<float*>(smem_raw + round_up(T * kXPitch * 2, 16));
   auto x_of = [&](int idx) { return __half2float(__ushort_as_half(xs[idx])); };
@@ -1317,8 +1317,8 @@ template <int BITS>
 static cudaError_t launch_quant(const CompressArgs& a, int nbh, int kmax_needed, cudaStream_t st) {
   const int T = a.seg.T;
   const size_t smem = round_up(T * kXPitch * 2, 16) + (size_t)T * kRPitch * 4;
-  dim3 grid(a.seg.nblk, nbh, 2);
-  if (quant_is_fast(a.seg, a.cc)) {
+  dim3 grid(a.seg.nblk, nbh, 2 - a.side0);         // side0 = 1: the value side only
+  if (a.side0 == 0 && quant_is_fast(a.seg, a.cc)) {
     cudaError_t e = cudaFuncSetAttribute(quant_fast_kernel<BITS, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          kFastSmemV);
     if (e != cudaSuccess) return e;
@@ -1350,7 +1350,8 @@ static void launch_pass(const PiArgs& p, cudaStream_t st) {
   pi_pass_kernel<MODE><<<grid, kPassWarps * 32, 0, st>>>(p);
 }
 
-size_t compress_workspace_bytes(int nbh, int n_c, int rank) {
+// bytes of the power iteration's part of the workspace (a multiple of 256)
+static size_t pi_workspace_bytes(int nbh, int n_c, int rank) {
   if (rank == 0) return 256;
   const size_t ntiles = (size_t)nbh * 2;
   const size_t nchunk = (n_c + kChunkRows - 1) / kChunkRows;
@@ -1362,7 +1363,12 @@ size_t compress_workspace_bytes(int nbh, int n_c, int rank) {
   b += ntiles * nchunk * 256 * 4;                 // Gp
   b += ntiles * 256 * 4;                          // W
   b += ntiles * 4;                                // Rmax
-  return b + 1024;
+  return (b + 1024 + 255) / 256 * 256;
+}
+
+// csr_k < 0: a segment with per-block key groups; otherwise one with per-vector keys and csr_k outliers per channel
+size_t compress_workspace_bytes(int nbh, int n_c, int rank, int csr_k) {
+  return pi_workspace_bytes(nbh, n_c, rank) + (csr_k >= 0 ? kcvt_workspace_bytes(nbh, n_c, csr_k) : 0);
 }
 
 cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned char* ws, cudaStream_t st) {
@@ -1391,9 +1397,17 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
   ca.V = job.V + (size_t)bh0 * sd.n_c * kHeadDim;
   ca.R = pa.R; ca.Rmax = pa.Rmax;
   const int kneed = sd.k_k > job.cc.k_v ? sd.k_k : job.cc.k_v;
+  const bool per_vector = sd.csr_base16 != 0;          // keys: one group per channel over the whole segment
+  ca.side0 = per_vector ? 1 : 0;
   cudaError_t e = job.cc.bits == 2 ? launch_quant<2>(ca, nbh, kneed, st) : launch_quant<4>(ca, nbh, kneed, st);
   if (e != cudaSuccess) return e;
-  count_launches(quant_is_fast(sd, job.cc) ? 2 : 1);
+  count_launches(!per_vector && quant_is_fast(sd, job.cc) ? 2 : 1);
+  if (per_vector) {
+    KcvtArgs ka;
+    ka.seg = sd; ka.arena = job.arena; ka.K = ca.K; ka.R = pa.R; ka.Rmax = pa.Rmax; ka.bh0 = bh0;
+    e = launch_kcvt_keys(ka, nbh, job.cc.bits, ws + pi_workspace_bytes(nbh, sd.n_c, sd.rank), st);
+    if (e != cudaSuccess) return e;
+  }
   if (sd.rank == 0) return cudaSuccess;
   // init + per early loop (pass, reduce) + last loop (pass, gram, chol, gram, chol, store, reduce)
   count_launches(1 + 2 * (job.iters - 1) + 7 + (job.iters == 1 ? 1 : 0));

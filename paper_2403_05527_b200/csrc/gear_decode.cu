@@ -744,6 +744,26 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
                   for (int e = 0; e < k2k; ++e) k_entry(j, __half2float(ov[j * k2k + e]), oi[j * k2k + e]);
               }
             }
+            if (S::kDyn && sdc->csr_base16 != 0) {
+              // per-vector keys: the block's outliers come from the list of the (batch, head), any channel to any lane
+              const unsigned char* csr = a.arena + sdc->seg_base + (size_t)sdc->csr_base16 * 16 +
+                                         (size_t)bh * csr_stride_bytes(sdc->nblk, sdc->csr_k);
+              const unsigned int* offs = reinterpret_cast<const unsigned int*>(csr);
+              const unsigned int* ent = reinterpret_cast<const unsigned int*>(csr + csr_offsets_bytes(sdc->nblk));
+              const unsigned int e_hi = offs[blk - c_seg_lo + 1];
+              const __half2* szp = reinterpret_cast<const __half2*>(kp + off_kscale);
+              for (unsigned int e = offs[blk - c_seg_lo] + lane; e < e_hi; e += 32) {
+                const unsigned int w = ent[e];
+                const int tok = (int)(w & 0xFFu), ch = (int)((w >> 8) & 0xFFu);
+                const float d = __half2float(__ushort_as_half((unsigned short)(w >> 16))) - __high2float(szp[ch]);
+#pragma unroll
+                for (int h = 0; h < HP; ++h)
+                  if (h < HC) {
+                    const float qv = __half2float(qs[h * kHeadDim + ch]) * a.scale_log2;
+                    atomicAdd(&corr_k[h * maxT + tok], __float2int_rn(qv * pow2i(sexp_k[h]) * d));
+                  }
+              }
+            }
           }
           __syncwarp();
           // this lane's B registers: limb gid % 4 of head hcol(nt) for the four 32-channel chunks
@@ -846,7 +866,7 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
                 if (tp < T) {
                   v = *reinterpret_cast<const float2*>(ps + h * maxT + tp);
                   v.x += c_zero[h]; v.y += c_zero[h];
-                  if (k2k > 0) {
+                  if (k2k > 0 || (S::kDyn && sdc->csr_base16 != 0)) {
                     const int2 c = *reinterpret_cast<const int2*>(corr_k + h * maxT + tp);
                     v.x = fmaf((float)c.x, Sik, v.x);
                     v.y = fmaf((float)c.y, Sik, v.y);

@@ -41,7 +41,8 @@ __global__ void export_kernel(const unsigned char* arena, SegDesc sd, CacheConst
       break;
     }
     case GEAR_EXP_K_SCALE: case GEAR_EXP_K_ZERO: {
-      const int ch = i % d; const size_t r = i / d; const int blk = r % sd.nblk, bh = r / sd.nblk;
+      const int rows = sd.csr_base16 ? 1 : sd.nblk;       // per-vector keys: every block repeats the segment's pair
+      const int ch = i % d; const size_t r = i / d; const int blk = r % rows, bh = r / rows;
       const __half2 z = reinterpret_cast<const __half2*>(record_of(arena, sd, bh, blk) + sd.off_kscale)[ch];
       reinterpret_cast<__half*>(dst)[i] = what == GEAR_EXP_K_SCALE ? __low2half(z) : __high2half(z);
       break;
@@ -89,9 +90,33 @@ __global__ void export_kernel(const unsigned char* arena, SegDesc sd, CacheConst
   }
 }
 
+// Key outliers of a segment with per-vector keys: one thread per (batch, head, channel) walks the list of its
+// (batch, head) -- sorted by block, channel, token -- and writes the channel's entries, token ascending.
+__global__ void export_list_kernel(const unsigned char* arena, SegDesc sd, int what, void* dst, int BH) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= BH * kHeadDim) return;
+  const int bh = i / kHeadDim, ch = i % kHeadDim;
+  const unsigned char* csr = arena + sd.seg_base + (size_t)sd.csr_base16 * 16 + (size_t)bh * csr_stride_bytes(sd.nblk, sd.csr_k);
+  const unsigned int* offs = reinterpret_cast<const unsigned int*>(csr);
+  const unsigned int* ent = reinterpret_cast<const unsigned int*>(csr + csr_offsets_bytes(sd.nblk));
+  int n = 0;
+  for (int b = 0; b < sd.nblk; ++b)
+    for (unsigned int e = offs[b]; e < offs[b + 1]; ++e) {
+      const unsigned int w = ent[e];
+      if ((int)((w >> 8) & 0xFFu) != ch || n >= sd.csr_k) continue;
+      if (what == GEAR_EXP_K_OUT_IDX) reinterpret_cast<int*>(dst)[(size_t)i * sd.csr_k + n] = b * sd.T + (int)(w & 0xFFu);
+      else reinterpret_cast<unsigned short*>(dst)[(size_t)i * sd.csr_k + n] = (unsigned short)(w >> 16);
+      ++n;
+    }
+}
+
 cudaError_t launch_export(const unsigned char* arena, const SegDesc& sd, const CacheConst& cc, int what, void* dst,
                           size_t n_elems, cudaStream_t st) {
   if (n_elems == 0) return cudaSuccess;
+  if (sd.csr_base16 != 0 && (what == GEAR_EXP_K_OUT_IDX || what == GEAR_EXP_K_OUT_VAL)) {
+    export_list_kernel<<<(cc.BH * kHeadDim + 127) / 128, 128, 0, st>>>(arena, sd, what, dst, cc.BH);
+    return cudaGetLastError();
+  }
   export_kernel<<<(unsigned int)((n_elems + 255) / 256), 256, 0, st>>>(arena, sd, cc, what, dst, n_elems);
   return cudaGetLastError();
 }

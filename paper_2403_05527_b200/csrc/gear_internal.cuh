@@ -21,7 +21,24 @@ struct CompressArgs {
   float* R;             // residual workspace [nbh][2][n_c][128] or nullptr (rank 0)
   unsigned int* Rmax;   // [nbh][2] bit patterns of max |R| per tile (zeroed before the launch), with R
   int bh0;              // first (batch, head) of the range, for addressing the records
+  int side0;            // first side the launch covers (blockIdx.z + side0: 0 keys, 1 values)
 };
+
+// Key side of a segment with per-vector grouping (gear_kcvt.cu)
+struct KcvtArgs {
+  SegDesc seg;
+  unsigned char* arena;
+  const __half* K;      // [nbh][n_c][128], already offset to the first (batch, head) of the range
+  float* R;             // residual workspace [nbh][2][n_c][128] or nullptr (rank 0)
+  unsigned int* Rmax;   // [nbh][2] (see CompressArgs) or nullptr
+  int bh0;
+  unsigned char* codes8;   // workspace: [nbh][n_c][128] one code per byte
+  unsigned int* olist;     // workspace: [nbh][128][csr_k] token | fp16 value << 16, token ascending
+  __half2* sz;             // workspace: [nbh][128] (scale, zero)
+};
+bool kcvt_fits(int n_c);
+size_t kcvt_workspace_bytes(int nbh, int n_c, int csr_k);
+cudaError_t launch_kcvt_keys(KcvtArgs a, int nbh, int bits, unsigned char* ws, cudaStream_t st);
 
 struct PiArgs {
   SegDesc seg;
@@ -52,7 +69,7 @@ struct CompressJob {
   int iters;
 };
 
-size_t compress_workspace_bytes(int nbh, int n_c, int rank);
+size_t compress_workspace_bytes(int nbh, int n_c, int rank, int csr_k = -1);
 // whole-tile path for short segments (one launch): usable when compress_tile_fits()
 bool compress_tile_fits(int T, int n_c, int rank);
 cudaError_t compress_tile(const CompressJob& job, int BH, cudaStream_t st);

@@ -56,7 +56,18 @@ struct SegDesc {
   int slab_a;            // bytes of A rows per slab and side
   int off_vpart;         // start of the value part inside a record (= bytes of the key part)
   int shape_id;          // compile-time block shape of the decode kernel that fits this segment, 0 = none
+  // Per-vector key grouping over a whole segment (one key group per channel over all n_c tokens): the records keep
+  // their 64-token blocks, every block repeats the channel's (scale, zero), k_k is 0 and the outliers of the
+  // segment live in a list per (batch, kv head) behind the records (see csr_stride_bytes).
+  int csr_k;             // outliers per channel, both sides together (0: the segment has per-block key groups)
+  unsigned int csr_base16;   // the list of (batch, kv head) 0: offset from seg_base in units of 16 bytes
 };
+static_assert(sizeof(SegDesc) == 128, "a warp copies a descriptor with one 32-bit load per lane");
+
+// Outlier list of one (batch, kv head) of such a segment: offsets u32 [nblk + 1] (padded to 16 bytes), then
+// 128 * csr_k entries sorted by block, then channel, then token: token in block | channel << 8 | fp16 value << 16.
+__host__ __device__ inline int csr_offsets_bytes(int nblk) { return ((nblk + 1) * 4 + 15) / 16 * 16; }
+__host__ __device__ inline int csr_stride_bytes(int nblk, int csr_k) { return csr_offsets_bytes(nblk) + 128 * csr_k * 4; }
 
 // Cache-wide constants the kernels need.
 struct CacheConst {

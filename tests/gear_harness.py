@@ -26,7 +26,8 @@ class Pair:
         self.dev = torch.device("cuda:0")
         self.cid, self.B, self.Hq, self.Hkv = config_id, batch, hq, hkv
         self.r_flush = r_flush
-        self.oracle = O.OracleCache(batch, hq, hkv, 128, bits, group, s, nb, r_flush, iters)
+        # group 0: per-vector grouping -- for the oracle, a group length no vector reaches
+        self.oracle = O.OracleCache(batch, hq, hkv, 128, bits, group if group else 1 << 30, s, nb, r_flush, iters)
         flags = G.GEAR_FLAG_KEEP_FP32_FACTORS if keep_fp32 else 0
         self.cfg = G.make_config(batch, hq, hkv, bits, group, s, nb, r_flush, max_tokens,
                                  rank_max=r_max if r_max is not None else max(r_flush, 0), power_iters=iters, flags=flags)

@@ -1,0 +1,89 @@
+"""Per-vector grouping (Section 2, "Group-wise Quantization"; the KCVT backbone of Section 4): one key group per
+channel over the whole segment, one value group per token, Filter_s (Eq. 4) on those whole vectors.  The CUDA path
+(C ABI, group = GEAR_GROUP_PER_VECTOR) against the float64 oracle run with a group length no vector reaches:
+bit-exact on codes, scales, zero-points and outlier sets / values, <= 1e-3 on the low-rank product and on attention."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture
+def pair_factory():
+    from tests.gear_harness import Pair
+    made = []
+
+    def make(*a, **k):
+        p = Pair(*a, **k)
+        made.append(p)
+        return p
+    yield make
+    for p in made:
+        if p.cache is not None:
+            p.close()
+
+
+def test_four_bit_prefill_of_4096_tokens_then_flushed_buffers(pair_factory):
+    """The paper's 4-bit setting (s = 2 %, r = 4) at n = 4096: 41 entries per side leave every key channel."""
+    from paper_2403_05527_b200 import binding as G
+    p = pair_factory(2, 1, 4, 2, 4, 0, 2.0, 32, 2, 4096 + 128, r_max=4)
+    p.compress(4096, 4)
+    si = G.gear_segment_info_get(p.cache, 0)
+    assert (si.g_k, si.k_k, si.g_v, si.k_v) == (4096, 41, 128, 2)
+    p.check_segment(0)
+    p.check_attention()
+    assert p.append(40) == 1                      # one flushed 32-token segment (a key group = its 32 tokens), 8 buffered
+    si = G.gear_segment_info_get(p.cache, 1)
+    assert (si.g_k, si.k_k) == (32, 1)
+    p.check_segment(1)
+    p.check_attention(extra=1)
+
+
+@pytest.mark.parametrize("bits,n,s,rank", [(2, 512, 2.0, 2), (4, 1024, 5.0, 0), (2, 192, 0.0, 4), (4, 8192, 1.0, 2)])
+def test_other_shapes(pair_factory, bits, n, s, rank):
+    p = pair_factory(3, 2, 2, 2, bits, 0, s, 64, 2, n + 128, r_max=max(rank, 2))
+    p.compress(n, rank)
+    p.check_segment(0)
+    p.check_attention()
+    p.append(70)
+    p.check_segment(1)
+    p.check_attention(extra=2)
+
+
+def test_ties_go_to_the_lower_token(pair_factory):
+    """Keys drawn from a handful of values: the thresholds of Filter_s sit inside long runs of equal entries, and a
+    channel that is constant has its k largest and k smallest in the first 2k tokens."""
+    import torch
+    from oracle import gear_oracle as O
+    from paper_2403_05527_b200 import binding as G, synth
+    B, H, n = 1, 2, 512
+    rng = np.random.default_rng(7)
+    k16 = rng.choice(np.array([-1.5, -0.25, 0.0, 0.25, 2.0], np.float16), size=(B, H, n, 128))
+    k16[:, :, :, 5] = np.float16(0.75)            # a constant channel
+    k16[:, :, ::7, 9] = np.float16(-0.0)          # both zeros in one channel
+    _, v16 = synth.make_kv(3, B, H, n, 128)
+    p = pair_factory(3, B, H, H, 4, 0, 3.0, 64, 0, n + 64, r_max=0)
+    p.oracle.compress(k16, v16, 0, None)
+    dev = p.dev
+    G.gear_compress(p.cache, None, torch.from_numpy(k16).to(dev), torch.from_numpy(v16).to(dev), n, 0, None)
+    torch.cuda.synchronize()
+    p.check_segment(0)
+    p.check_attention()
+    assert O.outlier_count(3.0, n) == 8
+
+
+def test_limits_are_errors(pair_factory):
+    import torch
+    from paper_2403_05527_b200 import binding as G
+    with pytest.raises(G.GearError):              # a buffer longer than one block of per-vector keys
+        G.gear_create(G.make_config(1, 1, 1, 4, 0, 2.0, 256, 0, 1024))
+    cfg = G.make_config(1, 1, 1, 4, 0, 2.0, 64, 0, 16384)
+    cache = G.gear_create(cfg)
+    try:
+        x = torch.zeros(1, 1, 16384, 128, dtype=torch.float16, device="cuda:0")
+        with pytest.raises(G.GearError):          # longer than the select kernel's shared memory holds
+            G.gear_compress(cache, None, x, x, 16384, 0, None)
+        with pytest.raises(G.GearError):          # not a multiple of the 64-token record block
+            G.gear_compress(cache, None, x, x, 208, 0, None)
+    finally:
+        G.gear_free(cache)

@@ -334,3 +334,29 @@ def test_literal_eq5_codes_the_zeros_left_by_the_outliers():
     assert np.all(np.abs(lit2["D"][m2]) <= scale[m2] * (0.5 + 2.0 ** -10))
     assert np.any(lit2["D"][m2] != 0.0)
     assert np.array_equal(lit2["R"][m2], -lit2["D"][m2])
+
+
+def test_per_vector_grouping_on_a_long_segment_by_brute_force():
+    """With g beyond every vector (Section 2, per-vector grouping) a key group is a whole channel: Eq. 4 takes the
+    k = ceil(s n / 200) largest and smallest of its n tokens (ties to the lower token, the smallest among what the
+    largest left), and Eq. 2 sees the rest.  Checked entry by entry against a sort written out here; the index of an
+    outlier no longer fits a byte."""
+    rng = np.random.default_rng(11)
+    n = 320
+    x = np.round(rng.standard_normal((n, 128)) * 4).astype(np.float16) / np.float16(4)      # many equal entries
+    t = O.compress_tile(x, "K", 4, 1 << 30, 2.0, 0, 3, None)
+    k = O.outlier_count(2.0, n)
+    assert (t["g_len"], k, t["out_idx"].dtype, t["scale"].shape) == (n, 4, np.int32, (1, 128))
+    for ch in (0, 17, 127):
+        col = x[:, ch].astype(np.float64)
+        order = sorted(range(n), key=lambda i: (-col[i], i))
+        top = order[:k]
+        rest = [i for i in range(n) if i not in top]
+        bot = sorted(rest, key=lambda i: (col[i], i))[:k]
+        out = sorted(top + bot)
+        assert list(t["out_idx"][ch]) == out
+        kept = [i for i in range(n) if i not in out]
+        lo, hi = col[kept].min(), col[kept].max()
+        assert float(t["zero"][0, ch]) == lo
+        assert float(t["scale"][0, ch]) == float(np.float16(np.float32(hi - lo) / np.float32(15)))
+        assert not t["mask"][kept, ch].any() and t["mask"][out, ch].all()
