@@ -40,7 +40,7 @@ UNIT = "tokens/s"
 # kernel on one layer cache (C2: 137.65 MB of DRAM traffic for 134.26 MB; C4: 125.65 MB for 118.48 MB); traffic grows in
 # proportion to the cache
 DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {2: 1.0253, 4: 1.0605}
-EXTRA_CONFIGS = (3, 32, 4)
+EXTRA_CONFIGS = (3, 32, 4, 6)
 
 
 def workload_name(w, layers):
@@ -101,7 +101,8 @@ def oracle_unit_cycle(w, unit_seed, n_decode):
     from oracle import gear_oracle as O
     k16, v16 = synth.make_kv(w.config_id, 1, 1, w.n, 128, extra=unit_seed)
     b0 = synth.make_b0(w.config_id, 1, 1, 128, w.rank, extra=unit_seed)
-    cache = O.OracleCache(1, 1, 1, 128, w.bits, w.group, w.s_pct, w.buffer_cap, w.rank, w.power_iters)
+    group = w.group if w.group else 1 << 30      # group 0 = per-vector grouping: no vector reaches this length
+    cache = O.OracleCache(1, 1, 1, 128, w.bits, group, w.s_pct, w.buffer_cap, w.rank, w.power_iters)
     cache.compress(k16, v16, w.rank, b0)
     ks, vs = synth.make_appended(w.config_id, 1, 1, 128, w.buffer_cap)
     q = synth.make_query(w.config_id, 1, 1, 128, extra=unit_seed)

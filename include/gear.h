@@ -81,7 +81,10 @@ typedef struct gear_config {
   float   outlier_pct;  /* s in percent, 0 <= s <= 10.  Filter_s (Eq. 4) takes
                            k = ceil(s * len / 200) largest and k smallest entries of every
                            group of length len; need k <= 8 and 2k < len                        */
-  int32_t buffer_cap;   /* n_b >= 1, multiple of 16: streaming-buffer capacity in tokens         */
+  int32_t buffer_cap;   /* n_b: streaming-buffer capacity in tokens, 16..1024.  A multiple of 16, and of
+                           `group` when larger than it; or a multiple of 4 that is smaller than `group`
+                           (at most 128 with per-vector grouping), e.g. the paper's n_b = 20: the
+                           flushed buffer is then one block whose last 16-token slab is partly empty   */
   int32_t rank_flush;   /* r_g: rank used when a full buffer is compressed, 0..16               */
   int32_t rank_max;     /* largest rank any gear_compress call will use (sizes the arena), 0..16 */
   int32_t power_iters;  /* L >= 1 loops of Algorithm 2                                           */

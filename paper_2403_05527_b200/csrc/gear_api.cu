@@ -132,8 +132,10 @@ static gear_status check_config(const gear_config* c) {
   const bool per_vector = c->group == GEAR_GROUP_PER_VECTOR;
   if (!per_vector && c->group != 16 && c->group != 32 && c->group != 64 && c->group != 128) return GEAR_ERR_ARG;
   if (!(c->outlier_pct >= 0.f) || c->outlier_pct > 10.f) return GEAR_ERR_ARG;
-  if (c->buffer_cap < 16 || c->buffer_cap % 16 || c->buffer_cap > 1024) return GEAR_ERR_ARG;
+  if (c->buffer_cap < 16 || c->buffer_cap % 4 || c->buffer_cap > 1024) return GEAR_ERR_ARG;
   if (per_vector ? c->buffer_cap > 128 : (c->buffer_cap > c->group && c->buffer_cap % c->group)) return GEAR_ERR_SHAPE;
+  // a capacity that is not a multiple of 16 (the paper's n_b = 20): the flushed buffer must be a single block
+  if (c->buffer_cap % 16 && !per_vector && c->buffer_cap > c->group) return GEAR_ERR_SHAPE;
   if (c->rank_flush < 0 || c->rank_flush > kMaxRank || c->rank_max < 0 || c->rank_max > kMaxRank) return GEAR_ERR_ARG;
   if (c->rank_flush > c->rank_max) return GEAR_ERR_ARG;
   if (c->rank_flush > c->buffer_cap) return GEAR_ERR_SHAPE;
@@ -323,6 +325,10 @@ static gear_status compress_segment(gear_cache* c, const void* K, const void* V,
   job.seed = c->cfg.seed; job.segment_index = (int)c->segs.size(); job.iters = c->cfg.power_iters;
 
   cudaError_t e = cudaSuccess;
+  if (sd.T % 16) {     // the last slab of every block is partly empty: its codes, factor rows and scales read as zero
+    if (cudaMemsetAsync(c->arena + sd.seg_base, 0, need, st) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
+    if (!compress_tile_fits(sd.T, sd.n_c, sd.rank)) return GEAR_ERR_SHAPE;
+  }
   if (!per_vector && compress_tile_fits(sd.T, sd.n_c, sd.rank)) {
     e = compress_tile(job, c->cc.BH, st);              // short segment: one launch, residual in shared memory
   } else if (is_flush) {
@@ -424,7 +430,7 @@ static gear_status plan_decode(gear_cache* c, int Gq) {
     if (s.off_vpart > max_k) max_k = s.off_vpart;
     if (s.rec_bytes - s.off_vpart > max_v) max_v = s.rec_bytes - s.off_vpart;
     if (s.bfac_bytes > max_bfac) max_bfac = s.bfac_bytes;
-    if (s.T > max_T) max_T = s.T;
+    if ((s.T + 31) / 32 * 32 > max_T) max_T = (s.T + 31) / 32 * 32;
   }
   if (!decode_plan(c->cc.bits, Gq, c->cc.ngv, max_k, max_v, max_bfac, max_T, 227 * 1024, warps_cap, &c->plan))
     return GEAR_ERR_SHAPE;

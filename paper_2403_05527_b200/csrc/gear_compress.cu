@@ -149,7 +149,7 @@ __device__ __forceinline__ void pack_block_codes(const unsigned short* xs, int T
   constexpr int F = 8 / BITS;
   if (side == 0) {
     constexpr int kWords = kSlab * kHeadDim * BITS / 32;            // words per slab
-    for (int li = tid; li < (T / kSlab) * kWords; li += nthreads) {
+    for (int li = tid; li < ((T + kSlab - 1) / kSlab) * kWords; li += nthreads) {
       const int slab = li / kWords, wl = li % kWords;
       const int w = wl & 3, lane = (wl >> 2) & 31, tau = wl >> 7;
       unsigned int word = 0;
@@ -159,7 +159,8 @@ __device__ __forceinline__ void pack_block_codes(const unsigned short* xs, int T
         for (int j = 0; j < F; ++j) {
           int tok, ch;
           code_coord_k(BITS, lane, tau, w, i, j, tok, ch);
-          word |= (unsigned int)xs[(slab * kSlab + tok) * kXPitch + ch] << (8 * i + BITS * j);
+          tok += slab * kSlab;
+          if (tok < T) word |= (unsigned int)xs[tok * kXPitch + ch] << (8 * i + BITS * j);
         }
       dst[li] = word;
     }

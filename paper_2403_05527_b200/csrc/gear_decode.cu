@@ -214,14 +214,14 @@ bool decode_plan(int bits, int heads, int ngv, int max_kpart, int max_vpart, int
 // group.  The shapes of the usual configurations are compile-time constants (every offset inside the record becomes
 // an immediate and the loops unroll); any other segment runs through the same code with run-time values.
 struct DynShape {                      // values read from the segment descriptor
-  static constexpr bool kDyn = true;
+  static constexpr bool kDyn = true, kCsr = true;     // kCsr: the segment may keep its key outliers in a list
   static constexpr int T = 0, k2k = 0, r_pad = 0, k2v = 0, unroll = 1;
   static constexpr int off_kscale = 0, off_koval = 0, off_koidx = 0, off_kcodes = 0, off_ak = 0, off_av = 0, off_vscale = 0,
                        off_voval = 0, off_voidx = 0;
 };
-template <int BITS, int NGV, int T_, int KK, int RP, int KV>
+template <int BITS, int NGV, int T_, int KK, int RP, int KV, bool CSR = false>
 struct StaticShape {                   // mirrors layout_segment(); checked against it on the host (static_shape_id)
-  static constexpr bool kDyn = false;
+  static constexpr bool kDyn = false, kCsr = CSR;
   static constexpr int T = T_, k2k = 2 * KK, r_pad = RP, k2v = 2 * KV, unroll = 2;
   static constexpr int nslab = T_ / kSlab, slab_codes = kSlab * kHeadDim * BITS / 8, nchunk = (T_ + 31) / 32;
   static constexpr int off_kscale = kRecHeader;
@@ -238,6 +238,7 @@ struct StaticShape {                   // mirrors layout_segment(); checked agai
   static constexpr int rec_bytes = off_vpart + off_voidx + (T_ * NGV * 2 * KV + 15) / 16 * 16;
   static bool matches(const SegDesc& s, const CacheConst& c) {
     return c.bits == BITS && c.ngv == NGV && c.k_v == KV && s.T == T_ && s.k_k == KK && s.r_pad == RP &&
+           (s.csr_base16 != 0) == CSR &&
            s.off_kscale == off_kscale && s.off_koval == off_koval && s.off_koidx == off_koidx &&
            s.off_kcodes == off_kcodes && s.off_ak == off_ak && s.off_vpart == off_vpart &&
            s.off_vcodes == off_vpart && s.off_av == off_vpart + off_av && s.off_vscale == off_vpart + off_vscale &&
@@ -249,12 +250,14 @@ template <int BITS> using ShapeA1 = StaticShape<BITS, 2, 64, 1, 4, 1>;     // g 
 template <int BITS> using ShapeA2 = StaticShape<BITS, 2, 64, 1, 8, 1>;     // g 64, rank 5..8
 template <int BITS> using ShapeB1 = StaticShape<BITS, 1, 128, 2, 4, 2>;    // g 128 prefill blocks
 template <int BITS> using ShapeB2 = StaticShape<BITS, 1, 64, 1, 4, 2>;     // g 128, flushed 64-token buffers
+template <int BITS> using ShapeP1 = StaticShape<BITS, 1, 64, 0, 4, 2, true>;   // per-vector keys (outlier list), rank 3..4
 
 int static_shape_id(const SegDesc& s, const CacheConst& c) {
   if (ShapeA1<2>::matches(s, c) || ShapeA1<4>::matches(s, c)) return 1;
   if (ShapeA2<2>::matches(s, c) || ShapeA2<4>::matches(s, c)) return 2;
   if (ShapeB1<2>::matches(s, c) || ShapeB1<4>::matches(s, c)) return 3;
   if (ShapeB2<2>::matches(s, c) || ShapeB2<4>::matches(s, c)) return 4;
+  if (ShapeP1<2>::matches(s, c) || ShapeP1<4>::matches(s, c)) return 5;
   return 0;
 }
 
@@ -551,7 +554,7 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
           const int o_voidx = S::kDyn ? sdc->off_voidx - sdc->off_vpart : S::off_voidx;
           const bool with_bk = r_pad > 0 && (blk == c_seg_lo || blk == blk_lo);
           const bool with_bv = r_pad > 0 && (blk == c_seg_hi - 1 || blk == blk_hi - 1);
-          const int nslab = T / kSlab;
+          const int nslab = (T + kSlab - 1) / kSlab;        // a block may end inside a slab (tokens past T: no score)
           const int nchunk = (T + 31) / 32;
 
           // ================================================================ key item
@@ -744,7 +747,7 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
                   for (int e = 0; e < k2k; ++e) k_entry(j, __half2float(ov[j * k2k + e]), oi[j * k2k + e]);
               }
             }
-            if (S::kDyn && sdc->csr_base16 != 0) {
+            if (S::kCsr && sdc->csr_base16 != 0) {
               // per-vector keys: the block's outliers come from the list of the (batch, head), any channel to any lane
               const unsigned char* csr = a.arena + sdc->seg_base + (size_t)sdc->csr_base16 * 16 +
                                          (size_t)bh * csr_stride_bytes(sdc->nblk, sdc->csr_k);
@@ -866,7 +869,7 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
                 if (tp < T) {
                   v = *reinterpret_cast<const float2*>(ps + h * maxT + tp);
                   v.x += c_zero[h]; v.y += c_zero[h];
-                  if (k2k > 0 || (S::kDyn && sdc->csr_base16 != 0)) {
+                  if (k2k > 0 || (S::kCsr && sdc->csr_base16 != 0)) {
                     const int2 c = *reinterpret_cast<const int2*>(corr_k + h * maxT + tp);
                     v.x = fmaf((float)c.x, Sik, v.x);
                     v.y = fmaf((float)c.y, Sik, v.y);
@@ -1123,6 +1126,7 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
         else if (NGV == 2 && c_shape == 2) body(ShapeA2<BITS>{});
         else if (NGV == 1 && c_shape == 3) body(ShapeB1<BITS>{});
         else if (NGV == 1 && c_shape == 4) body(ShapeB2<BITS>{});
+        else if (NGV == 1 && c_shape == 5) body(ShapeP1<BITS>{});
         else body(DynShape{});
         if (!alive) break;
       }

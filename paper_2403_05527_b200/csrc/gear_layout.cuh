@@ -14,11 +14,11 @@
 //     kscale     128 x (scale fp16, zero fp16)                 one pair per channel
 //     koval      128 x 2k_K fp16   outlier values, per channel, in-group index ascending
 //     koidx      128 x 2k_K u8     their token index inside the block
-//     kcodes     T/16 slabs x 16*128*b/8 bytes, in mma-fragment order (see code_coord_k)
-//     ak         T/16 slabs x [16 tokens][r_pad] fp16          rows of A_K
+//     kcodes     ceil(T/16) slabs x 16*128*b/8 bytes, in mma-fragment order (see code_coord_k; tokens past T: code 0)
+//     ak         ceil(T/16) slabs x [16 tokens][r_pad] fp16    rows of A_K (zero past T)
 //   -- off_vpart --
 //     vcodes     ceil(T/32) chunks x 32*128*b/8 bytes (see code_coord_v; tokens past T hold code 0)
-//     av         T/16 slabs x [r_pad][16 tokens] fp16          rows of A_V, transposed per slab
+//     av         ceil(T/16) slabs x [r_pad][16 tokens] fp16    rows of A_V, transposed per slab (zero past T)
 //     vscale     T x (d_H/g_V) x (scale fp16, zero fp16)
 //     voval      T x (d_H/g_V) x 2k_V fp16
 //     voidx      T x (d_H/g_V) x 2k_V u8   channel index inside the group
@@ -87,7 +87,7 @@ __host__ __device__ inline int rank_pad(int r) {
 
 // Fill the size / offset fields of a descriptor from (T, n_c, rank, k_k) and the cache constants.
 __host__ __device__ inline void layout_segment(SegDesc& s, const CacheConst& c) {
-  const int nslab = s.T / kSlab;
+  const int nslab = (s.T + kSlab - 1) / kSlab;     // a flushed buffer may end inside a slab: its tail rows hold zeros
   const int nchunk_v = (s.T + 31) / 32;
   s.r_pad = rank_pad(s.rank);
   s.nblk = s.n_c / s.T;

@@ -39,6 +39,24 @@ def test_four_bit_prefill_of_4096_tokens_then_flushed_buffers(pair_factory):
     p.check_attention(extra=1)
 
 
+@pytest.mark.parametrize("bits,group,n", [(4, 0, 1024), (2, 64, 256), (4, 128, 128)])
+def test_buffer_of_twenty_tokens(pair_factory, bits, group, n):
+    """n_b = 20 (Section 4, "Implementation details"): a flushed buffer is one block of 20 tokens, a key group its
+    20 tokens of a channel; the record keeps two 16-token slabs, the second one partly empty."""
+    from paper_2403_05527_b200 import binding as G
+    p = pair_factory(2, 2, 4, 2, bits, group, 2.0, 20, 2, n + 100, r_max=4)
+    p.compress(n, 4)
+    assert p.append(67) == 3                      # three flushed 20-token segments, seven tokens buffered
+    for si in (1, 2, 3):
+        info = G.gear_segment_info_get(p.cache, si)
+        assert (info.n_c, info.g_k, info.k_k) == (20, 20, 1)
+        p.check_segment(si)
+    p.check_attention(extra=3)
+    assert p.append(13) == 1                      # the buffer is empty right after a flush
+    p.check_segment(4)
+    p.check_attention(extra=4)
+
+
 @pytest.mark.parametrize("bits,n,s,rank", [(2, 512, 2.0, 2), (4, 1024, 5.0, 0), (2, 192, 0.0, 4), (4, 8192, 1.0, 2)])
 def test_other_shapes(pair_factory, bits, n, s, rank):
     p = pair_factory(3, 2, 2, 2, bits, 0, s, 64, 2, n + 128, r_max=max(rank, 2))
