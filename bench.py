@@ -343,9 +343,9 @@ def measure_config(torch, G, dev, w, layers, steps, warmup, rank, e2e_steps=0, d
     ms_total = max_over_ranks(s0.elapsed_time(s1), dist, dev)
     status = [G.gear_last_device_status(c) for c in caches]
     if any(status):
-        raise SystemExit(f"device status word set: {status}")
+        raise SystemExit(f"device status word set: {status} ({w.name})")
     if not all(torch.isfinite(o).all().item() for o in outs):
-        raise SystemExit("non-finite attention output")
+        raise SystemExit(f"non-finite attention output ({w.name})")
 
     dec_ms = [a.elapsed_time(b) for a, b in events]       # one entry per group of L back-to-back decode launches
     flush_ms = [a.elapsed_time(b) for a, b in flush_events]

@@ -929,9 +929,22 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
 #pragma unroll
           for (int i = 0; i < NPR; ++i) {
             const int pr = lane + 32 * i, tp = 2 * pr;
-            if (S::kDyn && tp >= T) break;
-            if (!S::kDyn && S::T < 64 && tp >= T) break;
             const int s = pr >> 3, pi = pr & 7, tw = pi & 3, rg = pi >> 2;
+            if (S::kDyn && tp >= T) {
+              // a block that ends inside a slab: the absent tokens of that slab get probability zero in the fp16
+              // fragments (the region held other operands before; their A_V rows are zero, but 0 x NaN is not)
+              if (r_pad > 0 && tp < nslab * kSlab) {
+#pragma unroll
+                for (int h = 0; h < HP; ++h)
+                  if (h < HC) {
+                    uint32_t* bp = fragPc + s * kFragStride + rg;
+                    bp[(2 * (h & 3) * 4 + tw) * 2] = 0u;
+                    bp[((2 * (h & 3) + 1) * 4 + tw) * 2] = 0u;
+                  }
+              }
+              break;
+            }
+            if (!S::kDyn && S::T < 64 && tp >= T) break;
             // where this pair's two bytes go in a row of the value B operand: chunk, register (tokens 4t.. / 16+4t..),
             // lane column, half word
             const int vboff = (((pr >> 4) * 8 + ((pr & 7) >> 1) * 2 + ((pr & 15) >> 3)) << 2) + ((pr & 1) << 1);

@@ -39,12 +39,13 @@ def test_four_bit_prefill_of_4096_tokens_then_flushed_buffers(pair_factory):
     p.check_attention(extra=1)
 
 
-@pytest.mark.parametrize("bits,group,n", [(4, 0, 1024), (2, 64, 256), (4, 128, 128)])
-def test_buffer_of_twenty_tokens(pair_factory, bits, group, n):
+@pytest.mark.parametrize("bits,group,n,hq,r_flush", [(4, 0, 1024, 4, 2), (2, 64, 256, 4, 2), (4, 128, 128, 4, 2),
+                                                     (4, 0, 1024, 2, 4), (2, 128, 256, 2, 4), (2, 64, 256, 2, 3)])
+def test_buffer_of_twenty_tokens(pair_factory, bits, group, n, hq, r_flush):
     """n_b = 20 (Section 4, "Implementation details"): a flushed buffer is one block of 20 tokens, a key group its
     20 tokens of a channel; the record keeps two 16-token slabs, the second one partly empty."""
     from paper_2403_05527_b200 import binding as G
-    p = pair_factory(2, 2, 4, 2, bits, group, 2.0, 20, 2, n + 100, r_max=4)
+    p = pair_factory(2, 2, hq, 2, bits, group, 2.0, 20, r_flush, n + 100, r_max=4)     # hq = 2: the one-head kernel
     p.compress(n, 4)
     assert p.append(67) == 3                      # three flushed 20-token segments, seven tokens buffered
     for si in (1, 2, 3):
