@@ -368,7 +368,8 @@ def measure_config(torch, G, dev, w, layers, steps, warmup, rank, e2e_steps=0, d
                 for li, c in enumerate(caches):
                     G.gear_append_buffer_host(c, hk_np[i % n_tok], hv_np[i % n_tok])
                     G.gear_decode_attn_host_async(c, hq_np, hout_np[li])
-                G.gear_stream_wait()
+                for c in caches:
+                    G.gear_cache_wait(c)
         step_e2e()
         barrier()
         t0 = time.perf_counter()

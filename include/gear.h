@@ -164,17 +164,18 @@ gear_status gear_release_workspace(void);
  * the call then synchronises `stream`).  Calls on one cache must use one stream. */
 gear_status gear_append_buffer_host(gear_cache* cache, const void* k_new_host, const void* v_new_host,
                                     const float* B0_flush_host, void* stream);
-/* gear_decode_attn with q and out in HOST memory; synchronises `stream` (out_host is valid on return). */
+/* gear_decode_attn with q and out in HOST memory; waits for the result (out_host is valid on return). */
 gear_status gear_decode_attn_host(gear_cache* cache, const void* q_host, float* out_host,
                                   float softmax_scale, void* stream);
-/* The same without the wait: the copies and the kernel are queued on `stream` and the call returns.  q_host must
- * stay unchanged, and out_host is not valid, until gear_stream_wait(stream) (or the caller's own wait on that
- * stream) has returned.  A model step queues all its layers this way and waits once.  Errors as gear_decode_attn. */
+/* The same without the wait: the copies and the kernel are queued and the call returns.  q_host must stay
+ * unchanged, and out_host is not valid, until gear_cache_wait(cache) has returned.  A model step queues all its
+ * layers this way and then waits for each cache once.  Errors as gear_decode_attn. */
 gear_status gear_decode_attn_host_async(gear_cache* cache, const void* q_host, float* out_host,
                                         float softmax_scale, void* stream);
-/* Blocks the calling host thread until everything queued on `stream` (0: the default stream) has finished.
- * GEAR_ERR_CUDA if the stream reports an error. */
-gear_status gear_stream_wait(void* stream);
+/* Blocks the calling host thread until the host-buffer calls queued on `cache` so far have finished: their copies
+ * run on a stream of the cache's own (ordered against the caller's stream by events, so that one cache's copies run
+ * beside another cache's kernels), which this call waits for.  GEAR_ERR_CUDA if that stream reports an error. */
+gear_status gear_cache_wait(gear_cache* cache);
 
 /* ---- FP16-cache reference point for the same decode step (Eq. 1 on uncompressed K, V) ---- */
 

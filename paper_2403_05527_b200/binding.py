@@ -65,7 +65,7 @@ _SIGNATURES = {
     "gear_append_buffer_host": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "gear_decode_attn_host": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
     "gear_decode_attn_host_async": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
-    "gear_stream_wait": (C.c_int32, [C.c_void_p]),
+    "gear_cache_wait": (C.c_int32, [C.c_void_p]),
     "gear_fp16_decode_attn": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                           C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_float, C.c_void_p,
                                           C.c_size_t, C.c_void_p]),
@@ -181,8 +181,8 @@ def gear_decode_attn_host_async(cache, q_host, out_host, softmax_scale: float = 
                                                     _stream(stream)), "gear_decode_attn_host_async")
 
 
-def gear_stream_wait(stream=None) -> int:
-    return _check(lib().gear_stream_wait(_stream(stream)), "gear_stream_wait")
+def gear_cache_wait(cache) -> int:
+    return _check(lib().gear_cache_wait(cache), "gear_cache_wait")
 
 
 def gear_fp16_attn_scratch_bytes(batch, n_q_heads, head_dim=128) -> int:

@@ -103,6 +103,10 @@ struct gear_cache {
   // holds on to the caller's memory.  A slot is reused once the copy that read it has finished (its event).
   static constexpr int kHostSlots = 4;
   unsigned char* host_ring[kHostSlots]; cudaEvent_t host_ev[kHostSlots]; bool host_used[kHostSlots]; int host_next;
+  // The host-buffer entry points copy on a stream of the cache's own, tied to the caller's stream by events, so that
+  // the copies of one cache run beside the kernels of another that shares the caller's stream.
+  cudaStream_t copy_st;
+  cudaEvent_t ev_rows_up, ev_rows_used, ev_q_up, ev_attn_done, ev_out_down;
   // host state
   std::vector<SegDesc> segs;
   std::vector<long long> dbgA_off, dbgB_off;             // float offsets into dbg (or -1)
@@ -172,6 +176,7 @@ static SegDesc shape_segment(const gear_cache* c, int n_c, int rank) {
 
 extern "C" void gear_free(gear_cache* c) {
   if (!c) return;
+  if (c->copy_st) cudaStreamSynchronize(c->copy_st);      // copies queued by the host-buffer calls still use the staging rows
   const DeviceAllocator& m = c->mem;
   m.put(c->arena); m.put(c->dbg); m.put(c->table_dev); m.put(c->blk2seg); m.put(c->buf_k); m.put(c->buf_v);
   m.put(c->flush_ws); m.put(c->partial); m.put(c->tickets); m.put(c->status);
@@ -180,6 +185,10 @@ extern "C" void gear_free(gear_cache* c) {
     if (c->host_ring[i]) cudaFreeHost(c->host_ring[i]);
     if (c->host_ev[i]) cudaEventDestroy(c->host_ev[i]);
   }
+  cudaEvent_t* evs[5] = {&c->ev_rows_up, &c->ev_rows_used, &c->ev_q_up, &c->ev_attn_done, &c->ev_out_down};
+  for (cudaEvent_t* e : evs)
+    if (*e) cudaEventDestroy(*e);
+  if (c->copy_st) cudaStreamDestroy(c->copy_st);
   delete c;
 }
 
@@ -209,6 +218,8 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   c->stage_k = c->stage_v = c->stage_q = nullptr; c->stage_out = nullptr; c->stage_b0 = nullptr;
   for (int i = 0; i < gear_cache::kHostSlots; ++i) { c->host_ring[i] = nullptr; c->host_ev[i] = nullptr; c->host_used[i] = false; }
   c->host_next = 0;
+  c->copy_st = nullptr;
+  c->ev_rows_up = c->ev_rows_used = c->ev_q_up = c->ev_attn_done = c->ev_out_down = nullptr;
   c->cc.bits = cfg->bits;
   c->cc.g_v = cfg->group == GEAR_GROUP_PER_VECTOR || cfg->group > kHeadDim ? kHeadDim : cfg->group;
   c->cc.ngv = kHeadDim / c->cc.g_v;
@@ -275,6 +286,16 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   for (int i = 0; i < gear_cache::kHostSlots; ++i) {
     if (cudaHostAlloc((void**)&c->host_ring[i], 2 * tok_bytes, cudaHostAllocDefault) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->host_ev[i], cudaEventDisableTiming) != cudaSuccess) {
+      cudaGetLastError();
+      gear_free(c);
+      return GEAR_ERR_ALLOC;
+    }
+  }
+  {
+    cudaEvent_t* evs[5] = {&c->ev_rows_up, &c->ev_rows_used, &c->ev_q_up, &c->ev_attn_done, &c->ev_out_down};
+    bool ok = cudaStreamCreateWithFlags(&c->copy_st, cudaStreamNonBlocking) == cudaSuccess;
+    for (cudaEvent_t* e : evs) ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
       cudaGetLastError();
       gear_free(c);
       return GEAR_ERR_ALLOC;
@@ -530,8 +551,12 @@ extern "C" gear_status gear_append_buffer_host(gear_cache* c, const void* k_host
   if (c->host_used[slot] && cudaEventSynchronize(c->host_ev[slot]) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
   memcpy(c->host_ring[slot], k_host, tok_bytes);
   memcpy(c->host_ring[slot] + tok_bytes, v_host, tok_bytes);
-  if (cudaMemcpyAsync(c->stage_k, c->host_ring[slot], 2 * tok_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaEventRecord(c->host_ev[slot], st) != cudaSuccess) {
+  // copy stream: after the previous push has read the staging rows; caller's stream: after the copy
+  if (cudaStreamWaitEvent(c->copy_st, c->ev_rows_used, 0) != cudaSuccess ||
+      cudaMemcpyAsync(c->stage_k, c->host_ring[slot], 2 * tok_bytes, cudaMemcpyHostToDevice, c->copy_st) != cudaSuccess ||
+      cudaEventRecord(c->host_ev[slot], c->copy_st) != cudaSuccess ||
+      cudaEventRecord(c->ev_rows_up, c->copy_st) != cudaSuccess ||
+      cudaStreamWaitEvent(st, c->ev_rows_up, 0) != cudaSuccess) {
     cudaGetLastError();
     return GEAR_ERR_CUDA;
   }
@@ -548,6 +573,7 @@ extern "C" gear_status gear_append_buffer_host(gear_cache* c, const void* k_host
   }
   gear_status s = gear_append_buffer(c, c->stage_k, c->stage_v, b0, stream);
   if (s < 0) return s;
+  if (cudaEventRecord(c->ev_rows_used, st) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
   // the start vectors are read straight from the caller's memory: only then wait for the copy
   if (with_b0 && cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
   return s;
@@ -558,14 +584,23 @@ static gear_status decode_host(gear_cache* c, const void* q_host, float* out_hos
   if (!c || !q_host || !out_host) return GEAR_ERR_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t nq = (size_t)c->cfg.batch * c->cfg.n_q_heads * kHeadDim;
-  if (cudaMemcpyAsync(c->stage_q, q_host, nq * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+  // query up on the copy stream once the previous call's kernel has read the staging query; the kernel after that
+  // copy and after the previous call's result has left the staging output
+  if (cudaStreamWaitEvent(c->copy_st, c->ev_attn_done, 0) != cudaSuccess ||
+      cudaMemcpyAsync(c->stage_q, q_host, nq * 2, cudaMemcpyHostToDevice, c->copy_st) != cudaSuccess ||
+      cudaEventRecord(c->ev_q_up, c->copy_st) != cudaSuccess ||
+      cudaStreamWaitEvent(st, c->ev_q_up, 0) != cudaSuccess ||
+      cudaStreamWaitEvent(st, c->ev_out_down, 0) != cudaSuccess) {
     cudaGetLastError();
     return GEAR_ERR_CUDA;
   }
   gear_status s = gear_decode_attn(c, c->stage_q, c->stage_out, softmax_scale, stream);
   if (s != GEAR_OK) return s;
-  if (cudaMemcpyAsync(out_host, c->stage_out, nq * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-      (wait && cudaStreamSynchronize(st) != cudaSuccess)) {
+  if (cudaEventRecord(c->ev_attn_done, st) != cudaSuccess ||
+      cudaStreamWaitEvent(c->copy_st, c->ev_attn_done, 0) != cudaSuccess ||
+      cudaMemcpyAsync(out_host, c->stage_out, nq * 4, cudaMemcpyDeviceToHost, c->copy_st) != cudaSuccess ||
+      cudaEventRecord(c->ev_out_down, c->copy_st) != cudaSuccess ||
+      (wait && cudaStreamSynchronize(c->copy_st) != cudaSuccess)) {
     cudaGetLastError();
     return GEAR_ERR_CUDA;
   }
@@ -582,8 +617,9 @@ extern "C" gear_status gear_decode_attn_host_async(gear_cache* c, const void* q_
   return decode_host(c, q_host, out_host, softmax_scale, stream, false);
 }
 
-extern "C" gear_status gear_stream_wait(void* stream) {
-  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) {
+extern "C" gear_status gear_cache_wait(gear_cache* c) {
+  if (!c) return GEAR_ERR_ARG;
+  if (cudaStreamSynchronize(c->copy_st) != cudaSuccess) {
     cudaGetLastError();
     return GEAR_ERR_CUDA;
   }

@@ -159,7 +159,7 @@ def test_host_buffer_entry_points(pair_factory):
     # the queued form: nothing is valid before the wait, the same bits after it
     out2 = np.zeros((1, 2, 128), np.float32)
     G.gear_decode_attn_host_async(p.cache, q, out2)
-    G.gear_stream_wait()
+    G.gear_cache_wait(p.cache)
     assert np.array_equal(out, out2)
 
 
