@@ -37,7 +37,7 @@ def _device_inputs(torch, w, dev, seed, n_app):
 
 
 @pytest.mark.parametrize("config_id,units", [(2, [(0, 0), (3, 17), (7, 31)]), (4, [(0, 0), (3, 7)]), (3, [(5, 11), (15, 39)]), (32, [(2, 3)]),
-                                             (21, [(1, 30)]), (22, [(0, 5), (3, 31)])])
+                                             (21, [(1, 30)]), (22, [(0, 5), (3, 31)]), (6, [(0, 0), (6, 29)])])
 def test_full_size_layer_sampled_units_match_the_oracle(config_id, units):
     import torch
     from oracle import gear_oracle as O
@@ -71,7 +71,8 @@ def test_full_size_layer_sampled_units_match_the_oracle(config_id, units):
             return exported[(seg, what)]
 
         for b, h in units:
-            ref = O.OracleCache(1, rep, 1, 128, w.bits, w.group, w.s_pct, w.buffer_cap, w.rank, w.power_iters)
+            group = w.group if w.group else 1 << 30          # group 0: per-vector grouping
+            ref = O.OracleCache(1, rep, 1, 128, w.bits, group, w.s_pct, w.buffer_cap, w.rank, w.power_iters)
             ref.compress(k[b:b + 1, h:h + 1].cpu().numpy(), v[b:b + 1, h:h + 1].cpu().numpy(), w.rank,
                          b0[b:b + 1, h:h + 1].cpu().numpy())
             for i in range(n_app):
