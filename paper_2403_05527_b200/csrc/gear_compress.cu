@@ -503,6 +503,262 @@ __global__ void __launch_bounds__(128) quant_fast_kernel(CompressArgs p) {
 }
 
 // ---------------------------------------------------------------------------
+// Groups of 128 entries with two outliers per side (g = 128 at s = 2 %: keys in blocks of 128 tokens, values one
+// group per token), again with the group in registers.  Per half of the packed pairs a chain keeps the three largest
+// and three smallest instances; the halves are merged; the entries above / equal to the second largest instance (and
+// below / equal to the second smallest) are found as bit masks, which give the two filtered entries per side in
+// (value, index) order.  A group in which the two sides would share an entry (nearly constant groups) takes the
+// general routine instead.  Same binary32 sequence per entry as everywhere else.
+// ---------------------------------------------------------------------------
+constexpr int kFast2Len = 128;
+constexpr int kCodePitch2 = kFast2Len + 4;
+
+// first set entry of the pair of 64-bit masks (even entries, odd entries), removed from them; 2 * 64 if none
+__device__ __forceinline__ int take_first(unsigned long long& even, unsigned long long& odd) {
+  const int fe = even ? 2 * (__ffsll((long long)even) - 1) : 2 * 64;
+  const int fo = odd ? 2 * (__ffsll((long long)odd) - 1) + 1 : 2 * 64;
+  if (fe < fo) { even &= even - 1; return fe; }
+  if (fo < 2 * 64) odd &= odd - 1;
+  return fo;
+}
+// four accumulators (bit q of the low / high half word: even / odd entry of pair 16 w + q) -> the two 64-bit masks
+__device__ __forceinline__ void masks_of(const unsigned int (&a)[4], unsigned long long& even, unsigned long long& odd) {
+  const unsigned int e0 = __byte_perm(a[0], a[1], 0x5410), e1 = __byte_perm(a[2], a[3], 0x5410);
+  const unsigned int o0 = __byte_perm(a[0], a[1], 0x7632), o1 = __byte_perm(a[2], a[3], 0x7632);
+  even = ((unsigned long long)e1 << 32) | e0;
+  odd = ((unsigned long long)o1 << 32) | o0;
+}
+// the three largest of six values (with multiplicity), in order
+__device__ __forceinline__ void top3_of6(float (&v)[6], float (&out)[3]) {
+#pragma unroll
+  for (int r = 0; r < 3; ++r) {
+    float m = v[0];
+#pragma unroll
+    for (int i = 1; i < 6; ++i) m = fmaxf(m, v[i]);
+    out[r] = m;
+    bool gone = false;
+#pragma unroll
+    for (int i = 0; i < 6; ++i) {
+      const bool hit = !gone && v[i] == m;
+      v[i] = hit ? -INFINITY : v[i];
+      gone = gone || hit;
+    }
+  }
+}
+
+template <int BITS, int SIDE>
+__global__ void __launch_bounds__(128) quant_fast2_kernel(CompressArgs p) {
+  constexpr int L = kFast2Len, F = 8 / BITS;
+  __shared__ __align__(16) unsigned char codes[L * kCodePitch2];    // keys [token][channel], values [channel][token]
+  __shared__ unsigned int dmax_bits, smax_bits, rmax_bits;
+  const SegDesc& sd = p.seg;
+  const int T = sd.T;                               // keys: 128; values: tokens (= groups) of the block
+  const int bhl = blockIdx.y, blk = blockIdx.x, tid = threadIdx.x;
+  if (tid == 0) { dmax_bits = 0u; smax_bits = 0u; rmax_bits = 0u; }
+  __syncthreads();
+  const __half* X = (SIDE == 0 ? p.K : p.V) + ((size_t)bhl * sd.n_c + (size_t)blk * T) * kHeadDim;
+  float* R = p.R ? p.R + (((size_t)bhl * 2 + SIDE) * sd.n_c + (size_t)blk * T) * kHeadDim : nullptr;
+  unsigned char* rec = p.arena + sd.seg_base + (size_t)(p.bh0 + bhl) * sd.bh_stride + sd.bfac_bytes +
+                       (size_t)blk * sd.rec_bytes;
+  const int first = SIDE == 0 ? tid : tid * kHeadDim;      // element e of the group: X[first + e * step]
+  const int step = SIDE == 0 ? kHeadDim : 1;
+  // where code / residual of element e go
+  auto code_at = [&](int e) -> unsigned char& { return codes[e * kCodePitch2 + tid]; };   // row: token (keys) / channel (values)
+  const bool active = SIDE == 0 || tid < T;
+
+  if (active) {
+    __half2 xp[L / 2];
+    if (SIDE == 0) {
+#pragma unroll
+      for (int q = 0; q < L / 2; ++q) xp[q] = __halves2half2(X[first + (2 * q) * kHeadDim], X[first + (2 * q + 1) * kHeadDim]);
+    } else {
+      const uint4* src = reinterpret_cast<const uint4*>(X + first);
+#pragma unroll
+      for (int q = 0; q < L / 8; ++q) {
+        const uint4 v = src[q];
+        xp[4 * q] = *reinterpret_cast<const __half2*>(&v.x);
+        xp[4 * q + 1] = *reinterpret_cast<const __half2*>(&v.y);
+        xp[4 * q + 2] = *reinterpret_cast<const __half2*>(&v.z);
+        xp[4 * q + 3] = *reinterpret_cast<const __half2*>(&v.w);
+      }
+    }
+    // the three largest / smallest instances of the even and of the odd entries, then of all
+    float top[3], bot[3];
+    {
+      const __half2 ninf = __float2half2_rn(-INFINITY), pinf = __float2half2_rn(INFINITY);
+      __half2 M1 = ninf, M2 = ninf, M3 = ninf, m1 = pinf, m2 = pinf, m3 = pinf;
+#pragma unroll
+      for (int q = 0; q < L / 2; ++q) {
+        const __half2 t = __hmin2(xp[q], M1);
+        M1 = __hmax2(M1, xp[q]);
+        const __half2 u = __hmin2(t, M2);
+        M2 = __hmax2(M2, t);
+        M3 = __hmax2(M3, u);
+        const __half2 tb = __hmax2(xp[q], m1);
+        m1 = __hmin2(m1, xp[q]);
+        const __half2 ub = __hmax2(tb, m2);
+        m2 = __hmin2(m2, tb);
+        m3 = __hmin2(m3, ub);
+      }
+      float v[6] = {__low2float(M1), __low2float(M2), __low2float(M3), __high2float(M1), __high2float(M2), __high2float(M3)};
+      top3_of6(v, top);
+      float w[6] = {-__low2float(m1), -__low2float(m2), -__low2float(m3), -__high2float(m1), -__high2float(m2), -__high2float(m3)};
+      top3_of6(w, bot);
+      bot[0] = -bot[0]; bot[1] = -bot[1]; bot[2] = -bot[2];
+    }
+    // entries above / equal to the second largest instance, below / equal to the second smallest
+    int it[2], ib[2];
+    {
+      const __half2 vT = __float2half2_rn(top[1]), vB = __float2half2_rn(bot[1]);
+      unsigned int gt[4] = {0u, 0u, 0u, 0u}, et[4] = {0u, 0u, 0u, 0u}, lt[4] = {0u, 0u, 0u, 0u}, eb[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+      for (int q = 0; q < L / 2; ++q) {
+        const unsigned int bit = 0x00010001u << (q & 15);
+        gt[q >> 4] |= __hgt2_mask(xp[q], vT) & bit;
+        et[q >> 4] |= __heq2_mask(xp[q], vT) & bit;
+        lt[q >> 4] |= __hlt2_mask(xp[q], vB) & bit;
+        eb[q >> 4] |= __heq2_mask(xp[q], vB) & bit;
+      }
+      unsigned long long ge, go, ee, eo;
+      masks_of(gt, ge, go); masks_of(et, ee, eo);
+      it[0] = take_first(ge, go);                      // the one entry above the second largest instance, if any
+      if (it[0] >= L) it[0] = take_first(ee, eo);
+      it[1] = take_first(ee, eo);
+      masks_of(lt, ge, go); masks_of(eb, ee, eo);
+      ib[0] = take_first(ge, go);
+      if (ib[0] >= L) ib[0] = take_first(ee, eo);
+      ib[1] = take_first(ee, eo);
+    }
+    const bool shared_entry = it[0] == ib[0] || it[0] == ib[1] || it[1] == ib[0] || it[1] == ib[1];
+    const float levels = (float)((1 << BITS) - 1);
+    float d, mn, dm, rmax;
+    __half d16;
+    unsigned char* orec_v = rec + (SIDE == 0 ? sd.off_koval : sd.off_voval) + tid * 8;
+    unsigned char* orec_i = rec + (SIDE == 0 ? sd.off_koidx : sd.off_voidx) + tid * 4;
+    if (!shared_entry) {
+      mn = bot[2];
+      const float mx = top[2];
+      // Eq. 2 on the kept entries: binary32, one rounding per operation
+      const float range = __fsub_rn(mx, mn);
+      const float d32 = __fdiv_rn(range, levels);
+      d16 = __float2half_rn(d32);
+      d = __half2float(d16);
+      const float inv = d != 0.f ? __fdiv_rn(1.0f, d) : 0.f;
+      constexpr float kRound = 12582912.0f;
+      auto quantize = [&](float x, unsigned int& code) {
+        const float t = __fmul_rn(__fsub_rn(x, mn), inv);
+        const float y = __fadd_rn(fminf(fmaxf(t, 0.f), levels), kRound);
+        code = __float_as_uint(y) & 0xFFu;
+        return x - fmaf(__fsub_rn(y, kRound), d, mn);
+      };
+      if (SIDE == 0) {
+#pragma unroll
+        for (int q = 0; q < L / 2; ++q) {
+          const float2 f = __half22float2(xp[q]);
+          unsigned int c0, c1;
+          const float r0 = quantize(f.x, c0), r1 = quantize(f.y, c1);
+          code_at(2 * q) = (unsigned char)c0;
+          code_at(2 * q + 1) = (unsigned char)c1;
+          if (R != nullptr) {
+            R[(2 * q) * kHeadDim + tid] = r0;
+            R[(2 * q + 1) * kHeadDim + tid] = r1;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int q = 0; q < L / 4; ++q) {
+          const float2 f0 = __half22float2(xp[2 * q]), f1 = __half22float2(xp[2 * q + 1]);
+          unsigned int k0, k1, k2, k3;
+          const float4 rr = make_float4(quantize(f0.x, k0), quantize(f0.y, k1), quantize(f1.x, k2), quantize(f1.y, k3));
+          code_at(4 * q) = (unsigned char)k0;
+          code_at(4 * q + 1) = (unsigned char)k1;
+          code_at(4 * q + 2) = (unsigned char)k2;
+          code_at(4 * q + 3) = (unsigned char)k3;
+          if (R != nullptr) *reinterpret_cast<float4*>(R + first + 4 * q) = rr;
+        }
+      }
+      // the four filtered entries: cleared, and stored in-group index ascending
+      int oi[4] = {it[0], it[1], ib[0], ib[1]};
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        code_at(oi[a]) = 0;
+        if (R != nullptr) R[SIDE == 0 ? oi[a] * kHeadDim + tid : first + oi[a]] = 0.f;
+      }
+      auto order = [&](int a, int b) { if (oi[a] > oi[b]) { const int t = oi[a]; oi[a] = oi[b]; oi[b] = t; } };
+      order(0, 1); order(2, 3); order(0, 2); order(1, 3); order(1, 2);
+      unsigned short ov[4];
+      dm = 0.f;
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const __half h = X[first + oi[a] * step];
+        ov[a] = __half_as_ushort(h);
+        dm = fmaxf(dm, fabsf(__half2float(h) - mn));
+      }
+      *reinterpret_cast<uint2*>(orec_v) = make_uint2(ov[0] | ((unsigned int)ov[1] << 16), ov[2] | ((unsigned int)ov[3] << 16));
+      *reinterpret_cast<unsigned int*>(orec_i) = (unsigned int)oi[0] | ((unsigned int)oi[1] << 8) |
+                                                 ((unsigned int)oi[2] << 16) | ((unsigned int)oi[3] << 24);
+      rmax = (d != 0.f ? 0.50390625f * d : range) + 2.4e-7f * (fabsf(mn) + fabsf(mx));
+    } else {
+      rmax = 0.f;
+      GroupResult g = process_group<BITS, 2>(
+          L, 2, [&](int e) { return __half2float(X[first + e * step]); },
+          [&](int e, int code, float r) {
+            code_at(e) = (unsigned char)code;
+            if (R != nullptr) R[SIDE == 0 ? e * kHeadDim + tid : first + e] = r;
+            rmax = fmaxf(rmax, fabsf(r));
+          },
+          [&](int slot, int idx, float v) {
+            reinterpret_cast<__half*>(orec_v)[slot] = __float2half_rn(v);
+            orec_i[slot] = (unsigned char)idx;
+          });
+      d16 = g.scale;
+      d = __half2float(d16);
+      mn = __half2float(g.zero);
+      dm = g.dmax;
+    }
+    reinterpret_cast<__half2*>(rec + (SIDE == 0 ? sd.off_kscale : sd.off_vscale))[tid] = __halves2half2(d16, __float2half_rn(mn));
+    atomicMax(&dmax_bits, __float_as_uint(dm));       // non-negative floats order like their bit patterns
+    atomicMax(&smax_bits, __float_as_uint(d));
+    atomicMax(&rmax_bits, __float_as_uint(rmax));
+  }
+  __syncthreads();
+  if (tid == 0) {
+    reinterpret_cast<float*>(rec)[SIDE] = __uint_as_float(dmax_bits);
+    reinterpret_cast<float*>(rec)[2 + SIDE] = __uint_as_float(smax_bits);
+    if (R != nullptr) atomicMax(p.Rmax + bhl * 2 + SIDE, rmax_bits);
+  }
+  // pack the codes into mma-fragment order (code_coord_k / code_coord_v), one 32-bit load per field
+  unsigned int* dst = reinterpret_cast<unsigned int*>(rec + (SIDE == 0 ? sd.off_kcodes : sd.off_vcodes));
+  if (SIDE == 0) {
+    constexpr int kWords = kSlab * kHeadDim * BITS / 32;            // words per slab
+    for (int li = tid; li < (L / kSlab) * kWords; li += 128) {
+      const int slab = li / kWords, wl = li % kWords;
+      const int w = wl & 3, lane = (wl >> 2) & 31, tau = wl >> 7;
+      const int tok = slab * kSlab + (lane >> 2) + 8 * (w & 1);
+      const int ch = 32 * F * tau + 16 * (w >> 1) + 4 * (lane & 3);
+      unsigned int word = 0;
+#pragma unroll
+      for (int j = 0; j < F; ++j)
+        word |= *reinterpret_cast<const unsigned int*>(&codes[tok * kCodePitch2 + ch + 32 * j]) << (BITS * j);
+      dst[li] = word;
+    }
+  } else {
+    constexpr int kWords = 32 * kHeadDim * BITS / 32;               // words per 32-token chunk
+    for (int li = tid; li < (T / 32) * kWords; li += 128) {
+      const int chunk = li / kWords, wl = li % kWords;
+      const int w = wl & 3, lane = (wl >> 2) & 31, tau = wl >> 7;
+      const int ch = 16 * F * tau + (lane >> 2) + 8 * (w & 1);
+      const int tok = chunk * 32 + 16 * (w >> 1) + 4 * (lane & 3);
+      unsigned int word = 0;
+#pragma unroll
+      for (int j = 0; j < F; ++j)
+        word |= *reinterpret_cast<const unsigned int*>(&codes[(ch + 16 * j) * kCodePitch2 + tok]) << (BITS * j);
+      dst[li] = word;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
 // Power iteration (Algorithm 2).  A "tile" is one (batch, head, K|V) residual
 // R_h [n_c, 128] in the workspace.  Factor buffers are [128][16] fp32, zero
 // beyond the rank.
@@ -1309,37 +1565,46 @@ __global__ void append_kernel(__half* buf_k, __half* buf_v, const __half* k_new,
 // ---------------------------------------------------------------------------
 // host side: launch sequence for a range of (batch, head) pairs
 // ---------------------------------------------------------------------------
-// the shape quant_fast_kernel is written for (two launches, keys then values)
-static bool quant_is_fast(const SegDesc& sd, const CacheConst& cc) {
-  return sd.T == kFastLen && cc.g_v == kFastLen && sd.k_k == 1 && cc.k_v == 1;
-}
-
+// Filter / Quant / pack / residual of a long segment: per side, the register-resident kernel that fits the group
+// shape, else the general one.  side0 = 1: the value side only.  Returns the number of launches through *launches.
 template <int BITS>
-static cudaError_t launch_quant(const CompressArgs& a, int nbh, int kmax_needed, cudaStream_t st) {
+static cudaError_t launch_quant(CompressArgs a, int nbh, int kmax_needed, cudaStream_t st, int* launches) {
   const int T = a.seg.T;
   const size_t smem = round_up(T * kXPitch * 2, 16) + (size_t)T * kRPitch * 4;
-  dim3 grid(a.seg.nblk, nbh, 2 - a.side0);         // side0 = 1: the value side only
-  if (a.side0 == 0 && quant_is_fast(a.seg, a.cc)) {
-    cudaError_t e = cudaFuncSetAttribute(quant_fast_kernel<BITS, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kFastSmemV);
-    if (e != cudaSuccess) return e;
-    grid.z = 1;
-    quant_fast_kernel<BITS, 0><<<grid, 128, 0, st>>>(a);
-    quant_fast_kernel<BITS, 1><<<grid, 128, kFastSmemV, st>>>(a);
-    return cudaGetLastError();
-  }
+  const dim3 grid(a.seg.nblk, nbh, 1);
+  const int first_side = a.side0;
+  *launches = 0;
+  for (int side = first_side; side < 2; ++side) {
+    const int len = side == 0 ? T : a.cc.g_v, k = side == 0 ? a.seg.k_k : a.cc.k_v;
+    cudaError_t e = cudaSuccess;
+    if (T == kFastLen && len == kFastLen && k == 1) {
+      if (side == 0) {
+        quant_fast_kernel<BITS, 0><<<grid, 128, 0, st>>>(a);
+      } else {
+        e = cudaFuncSetAttribute(quant_fast_kernel<BITS, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFastSmemV);
+        if (e != cudaSuccess) return e;
+        quant_fast_kernel<BITS, 1><<<grid, 128, kFastSmemV, st>>>(a);
+      }
+    } else if (len == kFast2Len && k == 2 && T % 32 == 0 && T <= kFast2Len) {
+      if (side == 0) quant_fast2_kernel<BITS, 0><<<grid, 128, 0, st>>>(a);
+      else quant_fast2_kernel<BITS, 1><<<grid, 128, 0, st>>>(a);
+    } else {
+      a.side0 = side;
 #define GEAR_LAUNCH_Q(KM)                                                                                   \
   {                                                                                                         \
-    cudaError_t e = cudaFuncSetAttribute(quant_pack_kernel<BITS, KM>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                         (int)smem);                                                       \
+    e = cudaFuncSetAttribute(quant_pack_kernel<BITS, KM>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                             (int)smem);                                                                   \
     if (e != cudaSuccess) return e;                                                                         \
     quant_pack_kernel<BITS, KM><<<grid, 128, smem, st>>>(a);                                                \
   }
-  if (kmax_needed <= 1) GEAR_LAUNCH_Q(1)
-  else if (kmax_needed <= 2) GEAR_LAUNCH_Q(2)
-  else if (kmax_needed <= 4) GEAR_LAUNCH_Q(4)
-  else GEAR_LAUNCH_Q(8)
+      if (kmax_needed <= 1) GEAR_LAUNCH_Q(1)
+      else if (kmax_needed <= 2) GEAR_LAUNCH_Q(2)
+      else if (kmax_needed <= 4) GEAR_LAUNCH_Q(4)
+      else GEAR_LAUNCH_Q(8)
 #undef GEAR_LAUNCH_Q
+    }
+    *launches += 1;
+  }
   return cudaGetLastError();
 }
 
@@ -1400,9 +1665,10 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
   const int kneed = sd.k_k > job.cc.k_v ? sd.k_k : job.cc.k_v;
   const bool per_vector = sd.csr_base16 != 0;          // keys: one group per channel over the whole segment
   ca.side0 = per_vector ? 1 : 0;
-  cudaError_t e = job.cc.bits == 2 ? launch_quant<2>(ca, nbh, kneed, st) : launch_quant<4>(ca, nbh, kneed, st);
+  int n_quant = 0;
+  cudaError_t e = job.cc.bits == 2 ? launch_quant<2>(ca, nbh, kneed, st, &n_quant) : launch_quant<4>(ca, nbh, kneed, st, &n_quant);
   if (e != cudaSuccess) return e;
-  count_launches(!per_vector && quant_is_fast(sd, job.cc) ? 2 : 1);
+  count_launches(n_quant);
   if (per_vector) {
     KcvtArgs ka;
     ka.seg = sd; ka.arena = job.arena; ka.K = ca.K; ka.R = pa.R; ka.Rmax = pa.Rmax; ka.bh0 = bh0;

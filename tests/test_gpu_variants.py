@@ -99,3 +99,33 @@ def test_several_query_rows_per_head(hq, hkv, nq, bits, group):
         assert e.value.status == G.GEAR_ERR_ARG
     finally:
         G.gear_free(cache)
+
+
+def test_groups_of_128_with_ties_and_constant_groups():
+    """g = 128, s = 2 %: two entries per side leave every group.  Entries drawn from five values put the thresholds of
+    Filter_s inside runs of equal entries (ties go to the lower index); constant groups make the smallest entries the
+    ones right after the largest.  Codes, scales and outlier sets must still match the oracle bit for bit."""
+    import torch
+    from tests.gear_harness import Pair
+    from paper_2403_05527_b200 import binding as G
+    B, H, n = 1, 2, 256
+    rng = np.random.default_rng(19)
+    vals = np.array([-1.5, -0.25, 0.0, 0.25, 2.0], np.float16)
+    k16 = rng.choice(vals, size=(B, H, n, 128))
+    v16 = rng.choice(vals, size=(B, H, n, 128))
+    k16[:, :, :, 7] = np.float16(0.5)              # a constant key channel
+    k16[:, :, 5, 8] = np.float16(3.0)              # one entry above a sea of ties
+    v16[:, :, 3, :] = np.float16(-0.75)            # a constant value row
+    v16[:, :, 9, :] = np.float16(1.0); v16[:, :, 9, 100] = np.float16(-4.0)
+    k16[:, :, 130:140, :] = (rng.standard_normal((B, H, 10, 128)) * 3).astype(np.float16)    # and ordinary entries
+    p = Pair(4, B, H, H, 2, 128, 2.0, 64, 0, n + 64, r_max=0)
+    try:
+        p.oracle.compress(k16, v16, 0, None)
+        G.gear_compress(p.cache, None, torch.from_numpy(k16).to(p.dev), torch.from_numpy(v16).to(p.dev), n, 0, None)
+        torch.cuda.synchronize()
+        si = G.gear_segment_info_get(p.cache, 0)
+        assert (si.g_k, si.k_k, si.g_v, si.k_v) == (128, 2, 128, 2)
+        p.check_segment(0)
+        p.check_attention()
+    finally:
+        p.close()
