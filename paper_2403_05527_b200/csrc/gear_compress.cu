@@ -848,17 +848,21 @@ __global__ void pi_init_kernel(PiArgs p, const float* B0, int bh0, int BH_total_
 // each 16-channel step c as one 128-bit load; since a contraction does not care about the order of its index, these
 // four channels serve as the step's k indices 2t, 2t+1, 2t+8, 2t+9 of the A fragment.  For R^T a the same registers,
 // transposed 8 x 8 by movmatrix, are the A fragment of R^T (rows: channels 4j, 4j+1 | 4j+2, 4j+3 of the step).
-template <int MODE>
-__global__ void __launch_bounds__(kPassWarps * 32, 3) pi_pass_kernel(PiArgs p) {
-  constexpr int RP = 4;                            // rank columns per CTA: 4 x (head, remainder) = the 8 columns of n
+// NT = 8-column tiles of n per CTA: one (four rank columns; three CTAs per SM) or two (eight columns, the residual is
+// converted once for both; two CTAs per SM).
+template <int MODE, int NT>
+__global__ void __launch_bounds__(kPassWarps * 32, NT == 1 ? 3 : 2) pi_pass_kernel(PiArgs p) {
+  constexpr int RP = 4 * NT;                       // rank columns per CTA: each gives a (head, remainder) column pair of n
   __shared__ float red[kHeadDim * RP];             // cross-warp sum, accumulated warp by warp
   __shared__ __align__(16) __half bsplit[2 * RP][kHeadDim];   // [2 rho + (0: head, 1: remainder)][channel]
   __shared__ float colmax[kPassWarps][RP];
-  const int tile = blockIdx.y, chunk = blockIdx.x;
+  // grid (rank column groups, chunks, tiles): the CTAs that read the same chunk of R are neighbours in launch order,
+  // so all but the first find it in L2
+  const int tile = blockIdx.z, chunk = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, t = lane & 3;
   const int row0 = chunk * kChunkRows;
   const int row1 = min(p.n_c, row0 + kChunkRows);
-  const int rho0 = blockIdx.z * RP;                // this CTA's rank columns [rho0, rho0 + RP)
+  const int rho0 = blockIdx.x * RP;                // this CTA's rank columns [rho0, rho0 + RP)
   const float* R = p.R + (size_t)tile * p.n_c * kHeadDim;
   float* A0 = p.A0 + (size_t)tile * p.n_c * kMaxRank + rho0;
 
@@ -892,24 +896,34 @@ __global__ void __launch_bounds__(kPassWarps * 32, 3) pi_pass_kernel(PiArgs p) {
     for (int i = threadIdx.x; i < kHeadDim * RP; i += blockDim.x) red[i] = 0.f;
     __syncthreads();
   }
-  // B fragments of a = R b: column n = gid is (rho = gid >> 1, head | remainder), k as described above
-  uint32_t bf[8][2];
-#pragma unroll
-  for (int c = 0; c < 8; ++c) {
-    const uint2 v = *reinterpret_cast<const uint2*>(&bsplit[gid][16 * c + 4 * t]);
-    bf[c][0] = v.x; bf[c][1] = v.y;
-  }
-  // |R sr| < 2 and |b 2^-eb| < 2, so |a| < 512 in these units: a 2^-10 stays below one half
-  constexpr float kScaleA = 1.0f / 1024.0f;
-  const int ebt = t == 0 ? eb[0] : (t == 1 ? eb[1] : (t == 2 ? eb[2] : eb[3]));
-  const float inv_a = exp2_int(er + ebt);                   // back to a = R b for column rho = t
-  const float inv_acc = exp2_int(2 * er + ebt + 10);        // back to R^T a
-
-  float acc[8][4];        // R^T a: [step c][(channel 4 gid/2 + gid%2 of the step | the same + 2) x (head, remainder) of rho = t]
+  // B fragments of a = R b: column n = gid of tile nt is (rho = 4 nt + gid / 2, head | remainder), k as described above
+  uint32_t bf[8][NT][2];
 #pragma unroll
   for (int c = 0; c < 8; ++c)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) acc[c][i] = 0.f;
+    for (int nt = 0; nt < NT; ++nt) {
+      const uint2 v = *reinterpret_cast<const uint2*>(&bsplit[8 * nt + gid][16 * c + 4 * t]);
+      bf[c][nt][0] = v.x; bf[c][nt][1] = v.y;
+    }
+  // |R sr| < 2 and |b 2^-eb| < 2, so |a| < 512 in these units: a 2^-10 stays below one half
+  constexpr float kScaleA = 1.0f / 1024.0f;
+  float inv_a[NT], inv_acc[NT];                    // back to a = R b and to R^T a for column rho = 4 nt + t
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    int ebt = eb[4 * nt];
+#pragma unroll
+    for (int q = 1; q < 4; ++q) ebt = t == q ? eb[4 * nt + q] : ebt;
+    inv_a[nt] = exp2_int(er + ebt);
+    inv_acc[nt] = exp2_int(2 * er + ebt + 10);
+  }
+
+  float acc[8][NT][4];    // R^T a: [step c][tile][(channel 4 gid/2 + gid%2 of the step | the same + 2) x (head, remainder)]
+#pragma unroll
+  for (int c = 0; c < 8; ++c)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[c][nt][i] = 0.f;
 
   for (int rb = row0 + warp * 16; rb < row1; rb += kPassWarps * 16) {
     const int ra = rb + gid, rc = rb + gid + 8;
@@ -921,26 +935,36 @@ __global__ void __launch_bounds__(kPassWarps * 32, 3) pi_pass_kernel(PiArgs p) {
       xc[c] = vc ? *reinterpret_cast<const float4*>(R + (size_t)rc * kHeadDim + 16 * c + 4 * t) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     uint32_t fh[8][4], fl[8][4];
-    float d[4] = {0.f, 0.f, 0.f, 0.f};
+    float d[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) d[nt][0] = d[nt][1] = d[nt][2] = d[nt][3] = 0.f;
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
       split_pair(xa[c].x * sr, xa[c].y * sr, fh[c][0], fl[c][0]);
       split_pair(xc[c].x * sr, xc[c].y * sr, fh[c][1], fl[c][1]);
       split_pair(xa[c].z * sr, xa[c].w * sr, fh[c][2], fl[c][2]);
       split_pair(xc[c].z * sr, xc[c].w * sr, fh[c][3], fl[c][3]);
-      mma16816(d, fh[c], bf[c][0], bf[c][1]);
-      mma16816(d, fl[c], bf[c][0], bf[c][1]);
-    }
-    const float a_lo_rows = d[0] + d[1], a_hi_rows = d[2] + d[3];   // a[row gid][rho t], a[row gid + 8][rho t] (scaled)
-    if (MODE == 1) {
-      if (va) A0[(size_t)ra * kMaxRank + t] = a_lo_rows * inv_a;
-      if (vc) A0[(size_t)rc * kMaxRank + t] = a_hi_rows * inv_a;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        mma16816(d[nt], fh[c], bf[c][nt][0], bf[c][nt][1]);
+        mma16816(d[nt], fl[c], bf[c][nt][0], bf[c][nt][1]);
+      }
     }
     // B fragment of R^T a: k = row, n = (rho, head | remainder): the 8 x 8 tiles [row][2 rho + part], transposed
-    uint32_t m0, m1;
-    split_pair_hl(a_lo_rows * kScaleA, m0);
-    split_pair_hl(a_hi_rows * kScaleA, m1);
-    const uint32_t ab0 = movmatrix_trans(m0), ab1 = movmatrix_trans(m1);
+    uint32_t ab[NT][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float a_lo_rows = d[nt][0] + d[nt][1], a_hi_rows = d[nt][2] + d[nt][3];   // a[row gid | gid + 8][rho 4 nt + t], scaled
+      if (MODE == 1) {
+        if (va) A0[(size_t)ra * kMaxRank + 4 * nt + t] = a_lo_rows * inv_a[nt];
+        if (vc) A0[(size_t)rc * kMaxRank + 4 * nt + t] = a_hi_rows * inv_a[nt];
+      }
+      uint32_t m0, m1;
+      split_pair_hl(a_lo_rows * kScaleA, m0);
+      split_pair_hl(a_hi_rows * kScaleA, m1);
+      ab[nt][0] = movmatrix_trans(m0);
+      ab[nt][1] = movmatrix_trans(m1);
+    }
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
       uint32_t th[4], tl[4];
@@ -948,8 +972,11 @@ __global__ void __launch_bounds__(kPassWarps * 32, 3) pi_pass_kernel(PiArgs p) {
       th[2] = movmatrix_trans(fh[c][1]); th[3] = movmatrix_trans(fh[c][3]);
       tl[0] = movmatrix_trans(fl[c][0]); tl[1] = movmatrix_trans(fl[c][2]);
       tl[2] = movmatrix_trans(fl[c][1]); tl[3] = movmatrix_trans(fl[c][3]);
-      mma16816(acc[c], th, ab0, ab1);
-      mma16816(acc[c], tl, ab0, ab1);
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        mma16816(acc[c][nt], th, ab[nt][0], ab[nt][1]);
+        mma16816(acc[c][nt], tl, ab[nt][0], ab[nt][1]);
+      }
     }
   }
   // combine the warps of this block in a fixed order, write the chunk's partial
@@ -958,8 +985,11 @@ __global__ void __launch_bounds__(kPassWarps * 32, 3) pi_pass_kernel(PiArgs p) {
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         const int ch = 16 * c + 4 * (gid >> 1) + (gid & 1);
-        red[ch * RP + t] += (acc[c][0] + acc[c][1]) * inv_acc;
-        red[(ch + 2) * RP + t] += (acc[c][2] + acc[c][3]) * inv_acc;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          red[ch * RP + 4 * nt + t] += (acc[c][nt][0] + acc[c][nt][1]) * inv_acc[nt];
+          red[(ch + 2) * RP + 4 * nt + t] += (acc[c][nt][2] + acc[c][nt][3]) * inv_acc[nt];
+        }
       }
     }
     __syncthreads();
@@ -1610,10 +1640,10 @@ static cudaError_t launch_quant(CompressArgs a, int nbh, int kmax_needed, cudaSt
 
 template <int MODE>
 static void launch_pass(const PiArgs& p, cudaStream_t st) {
-  // Four rank columns per CTA; a higher rank is spread over gridDim.z CTAs that read the same chunk of R (the second
-  // reader finds it in L2).
-  dim3 grid(p.nchunk, p.ntiles, p.rank <= 4 ? 1 : (p.rank <= 8 ? 2 : 4));
-  pi_pass_kernel<MODE><<<grid, kPassWarps * 32, 0, st>>>(p);
+  // Four or eight rank columns per CTA; rank 16 is spread over two CTAs that read the same chunk of R one after the
+  // other (the second finds it in L2).
+  if (p.rank <= 4) pi_pass_kernel<MODE, 1><<<dim3(1, p.nchunk, p.ntiles), kPassWarps * 32, 0, st>>>(p);
+  else pi_pass_kernel<MODE, 2><<<dim3(p.rank <= 8 ? 1 : 2, p.nchunk, p.ntiles), kPassWarps * 32, 0, st>>>(p);
 }
 
 // bytes of the power iteration's part of the workspace (a multiple of 256)
