@@ -36,10 +36,11 @@ from paper_2403_05527_b200 import synth  # noqa: E402
 
 METRIC = "compressed-KV decode attn tokens/s"
 UNIT = "tokens/s"
-# dram__bytes_read + dram__bytes_write of one gear_decode_kernel launch per algorithmic byte, from an ncu capture of the
-# kernel on one layer cache (C2: 137.65 MB of DRAM traffic for 134.26 MB; C4: 125.65 MB for 118.48 MB); traffic grows in
-# proportion to the cache
-DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {2: 1.0253, 4: 1.0605}
+# dram__bytes_read + dram__bytes_write of one gear_decode_kernel launch per algorithmic byte, by configuration, from ncu
+# captures of the kernel on one layer cache (C2: 137.65 MB of DRAM traffic for 134.26 MB; C4: 125.65 MB for 118.48 MB;
+# C3 4-bit: 1071.46 MB for 1077.91 MB; C3 2-bit: 735.96 MB for 738.39 MB; C6: 193.66 MB for 191.34 MB -- a ratio below
+# one: the segment flushed just before the captured launch was still in L2); traffic grows in proportion to the cache
+DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {2: 1.0253, 4: 1.0605, 3: 0.9940, 32: 0.9967, 6: 1.0121}
 EXTRA_CONFIGS = (3, 32, 4, 6)
 
 
@@ -405,7 +406,7 @@ def compress_roofline(w, res, peak):
     in_bytes = 2 * B * H * w.n * 128 * 2
     pre_ms = statistics.median(res["compress_ms"])
     pre_alg = in_bytes + res["prefill_out_bytes"]
-    out = {"prefill": {"bound": "hbm", "kernel": "quant_pack_kernel + pi_pass_kernel (dominant)", "ms": pre_ms,
+    out = {"prefill": {"bound": "hbm", "kernel": "Filter/Quant kernel of the group shape (quant_fast*_kernel, quant_pack_kernel, kcvt_*) + pi_pass_kernel (dominant)", "ms": pre_ms,
                        "input_gbs": in_bytes / (pre_ms * 1e-3) / 1e9, "algorithmic_bytes": pre_alg,
                        "achieved": pre_alg / (pre_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
                        "frac": pre_alg / (pre_ms * 1e-3) / 1e9 / peak}}
