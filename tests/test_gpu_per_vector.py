@@ -106,3 +106,38 @@ def test_limits_are_errors(pair_factory):
             G.gear_compress(cache, None, x, x, 208, 0, None)
     finally:
         G.gear_free(cache)
+
+
+def test_two_long_segments_a_short_one_and_a_buffer(pair_factory):
+    """Two prefill calls of per-vector keys (each its own groups and outlier list), a 128-token segment that is a
+    single ordinary block, then a flushed buffer and buffered tokens."""
+    import torch
+    from paper_2403_05527_b200 import binding as G, synth
+    p = pair_factory(5, 2, 2, 2, 2, 0, 2.0, 32, 2, 2048, r_max=4)
+    p.compress(512, 4)
+    p.compress(256, 2, extra=1)
+    p.compress(128, 3, extra=2)
+    infos = [G.gear_segment_info_get(p.cache, i) for i in range(3)]
+    assert [(i.n_c, i.g_k, i.k_k) for i in infos] == [(512, 512, 6), (256, 256, 3), (128, 128, 2)]
+    for si in range(3):
+        p.check_segment(si)
+    p.append(37)
+    p.check_segment(3)
+    p.check_attention(extra=5)
+    b = G.gear_cache_bytes(p.cache)
+    assert b.stored_total >= b.codes + b.scale_zero + b.outliers + b.lowrank_a + b.lowrank_b + b.buffer
+
+
+def test_capacity_of_the_arena_is_an_error_not_a_fault():
+    import torch
+    from paper_2403_05527_b200 import binding as G
+    cfg = G.make_config(1, 1, 1, 4, 0, 2.0, 32, 0, 512)
+    cache = G.gear_create(cfg)
+    try:
+        x = torch.randn(1, 1, 512, 128, device="cuda:0").half()
+        G.gear_compress(cache, None, x, x, 512, 0, None)
+        with pytest.raises(G.GearError):          # the cache was sized for 512 tokens
+            G.gear_compress(cache, None, x, x, 192, 0, None)
+        assert G.gear_last_device_status(cache) == 0
+    finally:
+        G.gear_free(cache)
