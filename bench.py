@@ -367,8 +367,7 @@ def measure_config(torch, G, dev, w, layers, steps, warmup, rank, e2e_steps=0, d
             # back, and the host waits once, for the last of them
             for i in range(nb):
                 for li, c in enumerate(caches):
-                    G.gear_append_buffer_host(c, hk_np[i % n_tok], hv_np[i % n_tok])
-                    G.gear_decode_attn_host_async(c, hq_np, hout_np[li])
+                    G.gear_step_host(c, hk_np[i % n_tok], hv_np[i % n_tok], hq_np, hout_np[li])
                 for c in caches:
                     G.gear_cache_wait(c)
         step_e2e()

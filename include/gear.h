@@ -172,6 +172,13 @@ gear_status gear_decode_attn_host(gear_cache* cache, const void* q_host, float* 
  * layers this way and then waits for each cache once.  Errors as gear_decode_attn. */
 gear_status gear_decode_attn_host_async(gear_cache* cache, const void* q_host, float* out_host,
                                         float softmax_scale, void* stream);
+/* One decoding step of one layer through HOST buffers, queued like gear_decode_attn_host_async: the new key / value
+ * rows and the query go up in one copy (through pinned memory of the library: k_new_host, v_new_host and q_host may
+ * be reused on return), the rows are pushed (gear_append_buffer with library-drawn start vectors if the push
+ * flushes), the query attends to the cache including the new token, and the result comes down into out_host, valid
+ * after gear_cache_wait(cache).  Returns GEAR_OK, GEAR_FLUSHED or an error of the two calls it combines. */
+gear_status gear_step_host(gear_cache* cache, const void* k_new_host, const void* v_new_host, const void* q_host,
+                           float* out_host, float softmax_scale, void* stream);
 /* Blocks the calling host thread until the host-buffer calls queued on `cache` so far have finished: their copies
  * run on a stream of the cache's own (ordered against the caller's stream by events, so that one cache's copies run
  * beside another cache's kernels), which this call waits for.  GEAR_ERR_CUDA if that stream reports an error. */

@@ -66,6 +66,7 @@ _SIGNATURES = {
     "gear_decode_attn_host": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
     "gear_decode_attn_host_async": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
     "gear_cache_wait": (C.c_int32, [C.c_void_p]),
+    "gear_step_host": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
     "gear_fp16_decode_attn": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                           C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_float, C.c_void_p,
                                           C.c_size_t, C.c_void_p]),
@@ -179,6 +180,11 @@ def gear_decode_attn_host(cache, q_host, out_host, softmax_scale: float = 0.0, s
 def gear_decode_attn_host_async(cache, q_host, out_host, softmax_scale: float = 0.0, stream=None) -> int:
     return _check(lib().gear_decode_attn_host_async(cache, _ptr(q_host), _ptr(out_host), softmax_scale,
                                                     _stream(stream)), "gear_decode_attn_host_async")
+
+
+def gear_step_host(cache, k_new_host, v_new_host, q_host, out_host, softmax_scale: float = 0.0, stream=None) -> int:
+    return _check(lib().gear_step_host(cache, _ptr(k_new_host), _ptr(v_new_host), _ptr(q_host), _ptr(out_host),
+                                       softmax_scale, _stream(stream)), "gear_step_host")
 
 
 def gear_cache_wait(cache) -> int:

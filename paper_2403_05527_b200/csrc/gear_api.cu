@@ -180,7 +180,7 @@ extern "C" void gear_free(gear_cache* c) {
   const DeviceAllocator& m = c->mem;
   m.put(c->arena); m.put(c->dbg); m.put(c->table_dev); m.put(c->blk2seg); m.put(c->buf_k); m.put(c->buf_v);
   m.put(c->flush_ws); m.put(c->partial); m.put(c->tickets); m.put(c->status);
-  m.put(c->stage_k); m.put(c->stage_q); m.put(c->stage_out); m.put(c->stage_b0);
+  m.put(c->stage_k); m.put(c->stage_out); m.put(c->stage_b0);
   for (int i = 0; i < gear_cache::kHostSlots; ++i) {
     if (c->host_ring[i]) cudaFreeHost(c->host_ring[i]);
     if (c->host_ev[i]) cudaEventDestroy(c->host_ev[i]);
@@ -281,10 +281,13 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
   cudaMemset(c->tickets, 0, units * 4);
   cudaMemset(c->status, 0, 4);
   const size_t tok_bytes = BH * kHeadDim * 2;
-  GEAR_TRY_ALLOC(c->stage_k, 2 * tok_bytes);          // key row, then value row: one copy brings both
+  // key row, value row, query: one copy can bring all three (gear_step_host)
+  const size_t q_bytes = (size_t)cfg->batch * cfg->n_q_heads * kHeadDim * 2;
+  GEAR_TRY_ALLOC(c->stage_k, 2 * tok_bytes + q_bytes);
   c->stage_v = reinterpret_cast<unsigned char*>(c->stage_k) + tok_bytes;
+  c->stage_q = reinterpret_cast<unsigned char*>(c->stage_k) + 2 * tok_bytes;
   for (int i = 0; i < gear_cache::kHostSlots; ++i) {
-    if (cudaHostAlloc((void**)&c->host_ring[i], 2 * tok_bytes, cudaHostAllocDefault) != cudaSuccess ||
+    if (cudaHostAlloc((void**)&c->host_ring[i], 2 * tok_bytes + q_bytes, cudaHostAllocDefault) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->host_ev[i], cudaEventDisableTiming) != cudaSuccess) {
       cudaGetLastError();
       gear_free(c);
@@ -301,7 +304,6 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
       return GEAR_ERR_ALLOC;
     }
   }
-  GEAR_TRY_ALLOC(c->stage_q, (size_t)cfg->batch * cfg->n_q_heads * kHeadDim * 2);
   GEAR_TRY_ALLOC(c->stage_out, (size_t)cfg->batch * cfg->n_q_heads * kHeadDim * 4);
   GEAR_TRY_ALLOC(c->stage_b0, BH * 2 * kHeadDim * (size_t)(cfg->rank_flush > 0 ? cfg->rank_flush : 1) * 4);
   if (cudaDeviceSynchronize() != cudaSuccess) { gear_free(c); return GEAR_ERR_CUDA; }
@@ -615,6 +617,47 @@ extern "C" gear_status gear_decode_attn_host(gear_cache* c, const void* q_host, 
 extern "C" gear_status gear_decode_attn_host_async(gear_cache* c, const void* q_host, float* out_host,
                                                    float softmax_scale, void* stream) {
   return decode_host(c, q_host, out_host, softmax_scale, stream, false);
+}
+
+// One token of one layer through host buffers: push the rows, attend, all queued.  One copy up (rows and query
+// through one pinned slot), one copy down.
+extern "C" gear_status gear_step_host(gear_cache* c, const void* k_host, const void* v_host, const void* q_host,
+                                      float* out_host, float softmax_scale, void* stream) {
+  if (!c || !k_host || !v_host || !q_host || !out_host) return GEAR_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t tok_bytes = (size_t)c->cc.BH * kHeadDim * 2;
+  const size_t nq = (size_t)c->cfg.batch * c->cfg.n_q_heads * kHeadDim;
+  const int slot = c->host_next;
+  c->host_next = (slot + 1) % gear_cache::kHostSlots;
+  if (c->host_used[slot] && cudaEventSynchronize(c->host_ev[slot]) != cudaSuccess) { cudaGetLastError(); return GEAR_ERR_CUDA; }
+  memcpy(c->host_ring[slot], k_host, tok_bytes);
+  memcpy(c->host_ring[slot] + tok_bytes, v_host, tok_bytes);
+  memcpy(c->host_ring[slot] + 2 * tok_bytes, q_host, nq * 2);
+  // copy stream: after the previous push and the previous kernel have read the staging area; caller's stream: after the
+  // copy, and after the previous result has left the staging output
+  if (cudaStreamWaitEvent(c->copy_st, c->ev_rows_used, 0) != cudaSuccess ||
+      cudaStreamWaitEvent(c->copy_st, c->ev_attn_done, 0) != cudaSuccess ||
+      cudaMemcpyAsync(c->stage_k, c->host_ring[slot], 2 * tok_bytes + nq * 2, cudaMemcpyHostToDevice, c->copy_st) != cudaSuccess ||
+      cudaEventRecord(c->host_ev[slot], c->copy_st) != cudaSuccess ||
+      cudaStreamWaitEvent(st, c->host_ev[slot], 0) != cudaSuccess ||
+      cudaStreamWaitEvent(st, c->ev_out_down, 0) != cudaSuccess) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  c->host_used[slot] = true;
+  gear_status pushed = gear_append_buffer(c, c->stage_k, c->stage_v, nullptr, stream);
+  if (pushed < 0) return pushed;
+  gear_status s = gear_decode_attn(c, c->stage_q, c->stage_out, softmax_scale, stream);
+  if (s != GEAR_OK) return s;
+  if (cudaEventRecord(c->ev_attn_done, st) != cudaSuccess ||
+      cudaEventRecord(c->ev_rows_used, st) != cudaSuccess ||
+      cudaStreamWaitEvent(c->copy_st, c->ev_attn_done, 0) != cudaSuccess ||
+      cudaMemcpyAsync(out_host, c->stage_out, nq * 4, cudaMemcpyDeviceToHost, c->copy_st) != cudaSuccess ||
+      cudaEventRecord(c->ev_out_down, c->copy_st) != cudaSuccess) {
+    cudaGetLastError();
+    return GEAR_ERR_CUDA;
+  }
+  return pushed;
 }
 
 extern "C" gear_status gear_cache_wait(gear_cache* c) {

@@ -161,6 +161,15 @@ def test_host_buffer_entry_points(pair_factory):
     G.gear_decode_attn_host_async(p.cache, q, out2)
     G.gear_cache_wait(p.cache)
     assert np.array_equal(out, out2)
+    # push and attend in one call
+    k1, v1 = synth.make_appended(2, 1, 2, 128, 4)
+    p.oracle.append(k1[3], v1[3], None)
+    out3 = np.zeros((1, 2, 128), np.float32)
+    assert G.gear_step_host(p.cache, k1[3], v1[3], q, out3) == G.GEAR_OK
+    G.gear_cache_wait(p.cache)
+    ref3 = p.oracle.decode_attn(q)
+    assert np.abs(out3 - ref3).max() / np.abs(ref3).max() <= 1e-3
+    assert G.gear_cache_info(p.cache).buffer_len == 4
 
 
 def test_fp16_cache_attention_against_textbook():
