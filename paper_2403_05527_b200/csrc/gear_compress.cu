@@ -856,6 +856,7 @@ __global__ void __launch_bounds__(kPassWarps * 32, NT == 1 ? 3 : 2) pi_pass_kern
   __shared__ float red[kHeadDim * RP];             // cross-warp sum, accumulated warp by warp
   __shared__ __align__(16) __half bsplit[2 * RP][kHeadDim];   // [2 rho + (0: head, 1: remainder)][channel]
   __shared__ float colmax[kPassWarps][RP];
+  __shared__ float gred[MODE == 1 ? kPassWarps : 1][RP][RP];   // Gram partials of the rows a (last loop, all columns here)
   // grid (rank column groups, chunks, tiles): the CTAs that read the same chunk of R are neighbours in launch order,
   // so all but the first find it in L2
   const int tile = blockIdx.z, chunk = blockIdx.y;
@@ -917,6 +918,15 @@ __global__ void __launch_bounds__(kPassWarps * 32, NT == 1 ? 3 : 2) pi_pass_kern
     inv_acc[nt] = exp2_int(2 * er + ebt + 10);
   }
 
+  // Last loop, and this CTA holds every rank column: the Gram matrix of the rows a (first round of CholeskyQR) is
+  // summed here, so that A0 is not read again for it.  gram[nt][v]: row rho = 4 nt + t of the matrix, column v.
+  const bool with_gram = MODE == 1 && gridDim.x == 1;
+  float gram[NT][RP];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int v = 0; v < RP; ++v) gram[nt][v] = 0.f;
+
   float acc[8][NT][4];    // R^T a: [step c][tile][(channel 4 gid/2 + gid%2 of the step | the same + 2) x (head, remainder)]
 #pragma unroll
   for (int c = 0; c < 8; ++c)
@@ -952,6 +962,24 @@ __global__ void __launch_bounds__(kPassWarps * 32, NT == 1 ? 3 : 2) pi_pass_kern
     }
     // B fragment of R^T a: k = row, n = (rho, head | remainder): the 8 x 8 tiles [row][2 rho + part], transposed
     uint32_t ab[NT][2];
+    if (MODE == 1 && with_gram) {
+      float mine[2][NT];                            // a[row gid | gid + 8][rho 4 nt + t]; rows past the chunk are zero
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        mine[0][nt] = (d[nt][0] + d[nt][1]) * inv_a[nt];
+        mine[1][nt] = (d[nt][2] + d[nt][3]) * inv_a[nt];
+      }
+#pragma unroll
+      for (int half = 0; half < 2; ++half)
+#pragma unroll
+        for (int nv = 0; nv < NT; ++nv)
+#pragma unroll
+          for (int tv = 0; tv < 4; ++tv) {
+            const float other = __shfl_sync(0xffffffffu, mine[half][nv], (lane & ~3) | tv);   // a[row][4 nv + tv]
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) gram[nt][4 * nv + tv] = fmaf(mine[half][nt], other, gram[nt][4 * nv + tv]);
+          }
+    }
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       const float a_lo_rows = d[nt][0] + d[nt][1], a_hi_rows = d[nt][2] + d[nt][3];   // a[row gid | gid + 8][rho 4 nt + t], scaled
@@ -977,6 +1005,25 @@ __global__ void __launch_bounds__(kPassWarps * 32, NT == 1 ? 3 : 2) pi_pass_kern
         mma16816(acc[c][nt], th, ab[nt][0], ab[nt][1]);
         mma16816(acc[c][nt], tl, ab[nt][0], ab[nt][1]);
       }
+    }
+  }
+  if (MODE == 1 && with_gram) {      // rows of the warp (over gid), then the warps, in a fixed order
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int v = 0; v < RP; ++v) {
+        float g = gram[nt][v];
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
+        if (gid == 0) gred[MODE == 1 ? warp : 0][4 * nt + t][v] = g;
+      }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) {
+      const int u = i / kMaxRank, v = i % kMaxRank;
+      float g = 0.f;
+      if (u < RP && v < RP)
+        for (int w = 0; w < kPassWarps; ++w) g += gred[MODE == 1 ? w : 0][u][v];
+      p.Gp[((size_t)tile * p.nchunk + chunk) * 256 + i] = g;
     }
   }
   // combine the warps of this block in a fixed order, write the chunk's partial
@@ -1707,7 +1754,7 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
   }
   if (sd.rank == 0) return cudaSuccess;
   // init + per early loop (pass, reduce) + last loop (pass, gram, chol, gram, chol, store, reduce)
-  count_launches(1 + 2 * (job.iters - 1) + 7 + (job.iters == 1 ? 1 : 0));
+  count_launches(1 + 2 * (job.iters - 1) + (sd.rank > 8 ? 7 : 6) + (job.iters == 1 ? 1 : 0));
 
   const int tot = (int)ntiles * kHeadDim * kMaxRank;
   const float* b0 = job.B0 ? job.B0 : nullptr;
@@ -1726,8 +1773,8 @@ cudaError_t compress_range(const CompressJob& job, int bh0, int nbh, unsigned ch
         q.nchunk = 1;
         pi_reduce_b_kernel<<<(int)ntiles, kHeadDim, 0, st>>>(q, 1, 0, 0);
       }
-      launch_pass<1>(pa, st);                                   // A0 = R B, R^T A0
-      pi_gram2_kernel<<<dim3(nchunk, (int)ntiles), 256, 0, st>>>(pa, 1);
+      launch_pass<1>(pa, st);                                   // A0 = R B, R^T A0; for ranks up to 8 also A0^T A0
+      if (sd.rank > 8) pi_gram2_kernel<<<dim3(nchunk, (int)ntiles), 256, 0, st>>>(pa, 1);
       pi_chol_kernel<<<(int)ntiles, 32, 0, st>>>(pa, 1);        // A <- Q(A) by CholeskyQR, twice
       pi_gram2_kernel<<<dim3(nchunk, (int)ntiles), 256, 0, st>>>(pa, 0);
       pi_chol_kernel<<<(int)ntiles, 32, 0, st>>>(pa, 0);

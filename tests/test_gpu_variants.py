@@ -129,3 +129,17 @@ def test_groups_of_128_with_ties_and_constant_groups():
         p.check_attention()
     finally:
         p.close()
+
+
+@pytest.mark.parametrize("rank", [3, 6, 12, 16])
+def test_ranks_of_a_long_segment(rank):
+    """Long segments run the power iteration as streaming passes: four rank columns per CTA (ranks up to 4), eight
+    (5..8, with the first Gram matrix summed inside the last pass), two such CTAs per chunk above that."""
+    from tests.gear_harness import Pair
+    p = Pair(6, 1, 2, 2, 4, 64, 2.0, 64, 2, 512 + 128, r_max=16)
+    try:
+        p.compress(512, rank)
+        p.check_segment(0)
+        p.check_attention()
+    finally:
+        p.close()
