@@ -40,6 +40,7 @@ namespace gear {
 
 constexpr int kBufPitch = 272;                  // bytes per fp16 row of a buffer slab in shared memory
 constexpr int kBufItem = kSlab * kBufPitch;     // one slab of key rows or of value rows
+constexpr int kCsrAhead = 6;                    // outlier-list entries per lane requested one block ahead (per-vector keys)
 constexpr int kFragKRow = 40;                   // 32-bit words per (head, limb) row of the key B-operand staging area
 constexpr int kTokLimit = 16384;                // tokens a value accumulator takes before it is folded (int32 headroom)
 constexpr float kMagic = 12582912.0f;           // 1.5 * 2^23: x + kMagic carries rint(x) in its low mantissa bits, |x| < 2^22
@@ -528,6 +529,13 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
         __syncwarp();
       };
 
+      // outlier lists of per-vector key segments: this lane's offset, the entries requested ahead for block cs_blk
+      // (such segments have one value group per token: the state exists in the NGV = 1 kernels only)
+      constexpr int kAhead = NGV == 1 ? kCsrAhead : 1;
+      unsigned int cs_off = 0u, cs_e[kAhead];
+      int cs_seg = -1, cs_unit = -1, cs_base = 0, cs_blk = -1;
+#pragma unroll
+      for (int j = 0; j < kAhead; ++j) cs_e[j] = 0u;
 #pragma unroll 1
       for (int blk = blk_lo; blk < c_hi; ++blk) {
         if (blk >= c_seg_hi || blk < c_seg_lo) {
@@ -747,16 +755,23 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
                   for (int e = 0; e < k2k; ++e) k_entry(j, __half2float(ov[j * k2k + e]), oi[j * k2k + e]);
               }
             }
-            if (S::kCsr && sdc->csr_base16 != 0) {
-              // per-vector keys: the block's outliers come from the list of the (batch, head), any channel to any lane
+            if (NGV == 1 && S::kCsr && sdc->csr_base16 != 0) {
+              // per-vector keys: the block's outliers come from the list of the (batch, head), any channel to any lane.
+              // A lane keeps one offset of the list (31 blocks per load), and the entries of the next block are
+              // requested as soon as this block's are used, so that they arrive during the rest of the block.
               const unsigned char* csr = a.arena + sdc->seg_base + (size_t)sdc->csr_base16 * 16 +
                                          (size_t)bh * csr_stride_bytes(sdc->nblk, sdc->csr_k);
               const unsigned int* offs = reinterpret_cast<const unsigned int*>(csr);
               const unsigned int* ent = reinterpret_cast<const unsigned int*>(csr + csr_offsets_bytes(sdc->nblk));
-              const unsigned int e_hi = offs[blk - c_seg_lo + 1];
+              const int bi = blk - c_seg_lo;
+              if (cs_seg != c_seg_lo || cs_unit != u || bi < cs_base || bi + 1 > cs_base + 31) {
+                cs_seg = c_seg_lo; cs_unit = u; cs_base = bi; cs_blk = -1;
+                cs_off = bi + lane <= sdc->nblk ? offs[bi + lane] : 0u;
+              }
+              const unsigned int e_lo = __shfl_sync(0xffffffffu, cs_off, bi - cs_base);
+              const unsigned int e_hi = __shfl_sync(0xffffffffu, cs_off, bi - cs_base + 1);
               const __half2* szp = reinterpret_cast<const __half2*>(kp + off_kscale);
-              for (unsigned int e = offs[blk - c_seg_lo] + lane; e < e_hi; e += 32) {
-                const unsigned int w = ent[e];
+              auto apply = [&](unsigned int w) {
                 const int tok = (int)(w & 0xFFu), ch = (int)((w >> 8) & 0xFFu);
                 const float d = __half2float(__ushort_as_half((unsigned short)(w >> 16))) - __high2float(szp[ch]);
 #pragma unroll
@@ -765,6 +780,23 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
                     const float qv = __half2float(qs[h * kHeadDim + ch]) * a.scale_log2;
                     atomicAdd(&corr_k[h * maxT + tok], __float2int_rn(qv * pow2i(sexp_k[h]) * d));
                   }
+              };
+              const bool have = cs_blk == blk;
+#pragma unroll
+              for (int j = 0; j < kAhead; ++j) {
+                const unsigned int e = e_lo + lane + 32 * j;
+                if (e < e_hi) apply(have ? cs_e[j] : ent[e]);
+              }
+              for (unsigned int e = e_lo + lane + 32 * kAhead; e < e_hi; e += 32) apply(ent[e]);
+              if (blk + 1 < min(c_hi, c_seg_hi) && bi + 2 <= cs_base + 31) {
+                const unsigned int n_lo = __shfl_sync(0xffffffffu, cs_off, bi + 1 - cs_base);
+                const unsigned int n_hi = __shfl_sync(0xffffffffu, cs_off, bi + 2 - cs_base);
+#pragma unroll
+                for (int j = 0; j < kAhead; ++j) {
+                  const unsigned int e = n_lo + lane + 32 * j;
+                  cs_e[j] = e < n_hi ? ent[e] : 0u;
+                }
+                cs_blk = blk + 1;
               }
             }
           }
@@ -869,7 +901,7 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
                 if (tp < T) {
                   v = *reinterpret_cast<const float2*>(ps + h * maxT + tp);
                   v.x += c_zero[h]; v.y += c_zero[h];
-                  if (k2k > 0 || (S::kCsr && sdc->csr_base16 != 0)) {
+                  if (k2k > 0 || (NGV == 1 && S::kCsr && sdc->csr_base16 != 0)) {
                     const int2 c = *reinterpret_cast<const int2*>(corr_k + h * maxT + tp);
                     v.x = fmaf((float)c.x, Sik, v.x);
                     v.y = fmaf((float)c.y, Sik, v.y);
