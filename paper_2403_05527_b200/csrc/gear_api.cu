@@ -7,6 +7,7 @@
 #include <atomic>
 #include <mutex>
 #include <new>
+#include <unordered_map>
 #include <vector>
 
 #include "../../include/gear.h"
@@ -15,6 +16,15 @@
 using namespace gear;
 
 static std::atomic<unsigned long long> g_launches{0};
+// Calls of the library that launch kernels, numbered per stream: a decode call may request its first copies before
+// it waits for the kernel in front of it only if that kernel cannot be the one that last wrote the cache.
+static std::mutex g_seq_mutex;
+static std::unordered_map<cudaStream_t, unsigned long long> g_stream_seq;
+static unsigned long long next_call_number(cudaStream_t st) {
+  std::lock_guard<std::mutex> lock(g_seq_mutex);
+  return ++g_stream_seq[st];
+}
+
 void gear::count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 extern "C" uint64_t gear_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
@@ -118,6 +128,8 @@ struct gear_cache {
   DecodeArgs plan;
   int test_dead_wait;            // gear_test_dead_wait: the next decode calls wait on a barrier nothing completes
   int max_queries, units_alloc;  // query rows per head the scratch was sized for; units of that size
+  // the last call that wrote the cache (records, descriptors, buffer rows): its stream and its number on that stream
+  cudaStream_t write_stream; unsigned long long write_call; bool written;
 };
 
 static int outlier_count(float s_pct, int len) {
@@ -213,6 +225,7 @@ extern "C" gear_status gear_create(gear_cache** out, const gear_config* cfg) {
     c->mem.alloc = g_alloc; c->mem.free = g_free; c->mem.ctx = g_alloc_ctx;
   }
   c->test_dead_wait = 0;
+  c->write_stream = nullptr; c->write_call = 0; c->written = false;
   c->arena = nullptr; c->dbg = nullptr; c->table_dev = nullptr; c->blk2seg = nullptr; c->buf_k = c->buf_v = nullptr; c->flush_ws = nullptr;
   c->partial = nullptr; c->tickets = nullptr; c->status = nullptr;
   c->stage_k = c->stage_v = c->stage_q = nullptr; c->stage_out = nullptr; c->stage_b0 = nullptr;
@@ -387,6 +400,7 @@ static gear_status compress_segment(gear_cache* c, const void* K, const void* V,
   c->n_compressed += n;
   c->n_blocks_c += sd.nblk;
   c->plan_key = -1;
+  c->write_stream = st; c->write_call = next_call_number(st); c->written = true;
   return GEAR_OK;
 }
 
@@ -429,6 +443,7 @@ extern "C" gear_status gear_append_buffer(gear_cache* c, const void* k_new, cons
   }
   c->buf_len += 1;
   c->plan_key = -1;
+  c->write_stream = st; c->write_call = next_call_number(st); c->written = true;
   if (c->buf_len < n_b) return GEAR_OK;
   gear_status s = compress_segment(c, c->buf_k, c->buf_v, n_b, c->cfg.rank_flush, B0_flush, true, st);
   if (s != GEAR_OK) { c->buf_len -= 1; return s; }
@@ -480,6 +495,10 @@ static gear_status decode_rows(gear_cache* c, const void* q, float* out, int Gq,
   const float sc = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)kHeadDim);
   a.scale_log2 = sc * 1.4426950408889634f;
   a.test_dead_wait = c->test_dead_wait;
+  {
+    const unsigned long long call = next_call_number((cudaStream_t)stream);
+    a.early_reads = c->written && c->write_stream == (cudaStream_t)stream && call >= c->write_call + 2 ? 1 : 0;
+  }
   // one warp per CTA; never more warps than blocks of work
   const int passes = decode_passes(Gq);
   if ((long long)c->cc.BH * passes > c->units_alloc) return GEAR_ERR_CAPACITY;

@@ -340,10 +340,14 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
     blk_lo = (int)(f0 - (long long)u * NB);
   }
 
-  // Everything above used kernel parameters and shared memory only.  Let the launch after this one start its own
-  // prologue, and wait until the launches before this one have completed and their writes are visible.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Everything above used kernel parameters and shared memory only.  The launch is a programmatic dependent of the
+  // kernel before it on the stream: it waits (griddepcontrol.wait) until that kernel has completed and its writes
+  // are visible.  Only after its own wait does a decode kernel let its dependents start, so whoever starts early
+  // knows that everything two launches back is complete.  When the host has seen another launch of the library on
+  // this stream since the cache was last written (early_reads), the first copies of the ring -- descriptors,
+  // records and buffer rows, none of them written by the kernel right before this one -- are requested before the
+  // wait, so that they travel while that kernel drains; the query and everything else is read after it.
+  if (!a.early_reads) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   auto load_desc = [&](SegDesc* dst, int blk) {
     const int* src = reinterpret_cast<const int*>(a.table + a.blk2seg[blk]);
@@ -408,6 +412,8 @@ __global__ void __launch_bounds__(32, MINB) gear_decode_kernel(const __grid_cons
     }
   };
   for (int s = 0; s < NS; ++s) issue();
+  if (a.early_reads) asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   int c_stage = 0, c_par = 0, c_seg_lo = 0, c_seg_hi = 0, c_shape = 0;
   bool alive = true;

@@ -117,6 +117,7 @@ struct DecodeArgs {
   int spin_limit;             // polls a consumer spends on one ring stage before it gives up
   int test_dead_wait;         // test only: wait once on a barrier that nothing completes, with a short limit
   int wide;                   // one head per pass: use the kernel built for twelve resident warps (more registers)
+  int early_reads;            // the cache's data was last written at least two launches back on this stream (see the kernel)
   WarpSmem ws;
   float scale_log2;           // softmax scale * log2(e)
 };
