@@ -29,52 +29,66 @@ __device__ __forceinline__ float key_value(unsigned int key) {
   return __half2float(__ushort_as_half((unsigned short)h));
 }
 
-// The k-th largest key of keys[0 .. n) (flip = 0) or, with flip = 0xFFFF, the k-th smallest, by two 8-bit
-// histograms.  Returns the key; n_beyond = how many keys lie strictly beyond it.  One warp, hist = 256 words.
-__device__ __forceinline__ unsigned int warp_select(const unsigned short* keys, int n, int k, unsigned int flip,
-                                                    unsigned int* hist, int lane, int& n_beyond) {
-  unsigned int prefix = 0u;
-  int want = k, beyond = 0;
-#pragma unroll 1
-  for (int level = 0; level < 2; ++level) {
-    for (int i = lane; i < 256; i += 32) hist[i] = 0u;
-    __syncwarp();
-    for (int i = lane; i < n; i += 32) {
-      const unsigned int key = keys[i] ^ flip;
-      if (level == 0) atomicAdd(&hist[key >> 8], 1u);
-      else if ((key >> 8) == prefix) atomicAdd(&hist[key & 0xFFu], 1u);
-    }
-    __syncwarp();
-    // lane l owns bins 8 l .. 8 l + 7; count of the bins above the lane's
-    unsigned int mine = 0u;
+// Of a 256-bin histogram, the highest bin b with (count of the bins above b) < want <= (count of the bins >= b);
+// over = the count of the bins above it.  One warp; lane l owns bins 8 l .. 8 l + 7.
+__device__ __forceinline__ int pick_bin(const unsigned int* hist, int want, int lane, int& over) {
+  unsigned int mine = 0u;
 #pragma unroll
-    for (int b = 0; b < 8; ++b) mine += hist[8 * lane + b];
-    unsigned int incl = mine;                      // sum over lanes >= this one
+  for (int b = 0; b < 8; ++b) mine += hist[8 * lane + b];
+  unsigned int incl = mine;                      // sum over lanes >= this one
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned int v = __shfl_down_sync(0xffffffffu, incl, o);
-      if (lane + o < 32) incl += v;
-    }
-    const unsigned int above = incl - mine;
-    const bool here = above < (unsigned int)want && (unsigned int)want <= incl;
-    const int src = __ffs((int)__ballot_sync(0xffffffffu, here)) - 1;
-    int bin = 0, over = 0;
-    if (here) {
-      unsigned int acc = above;
-      for (int b = 7; b >= 0; --b) {
-        const unsigned int c = hist[8 * lane + b];
-        if (acc + c >= (unsigned int)want) { bin = 8 * lane + b; over = (int)acc; break; }
-        acc += c;
-      }
-    }
-    bin = __shfl_sync(0xffffffffu, bin, src);
-    over = __shfl_sync(0xffffffffu, over, src);
-    __syncwarp();
-    if (level == 0) { prefix = (unsigned int)bin; beyond = over; want -= over; }
-    else { prefix = (prefix << 8) | (unsigned int)bin; beyond += over; }
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned int v = __shfl_down_sync(0xffffffffu, incl, o);
+    if (lane + o < 32) incl += v;
   }
-  n_beyond = beyond;
-  return prefix ^ flip;
+  const unsigned int above = incl - mine;
+  const bool here = above < (unsigned int)want && (unsigned int)want <= incl;
+  const int src = __ffs((int)__ballot_sync(0xffffffffu, here)) - 1;
+  int bin = 0, ov = 0;
+  if (here) {
+    unsigned int acc = above;
+    for (int b = 7; b >= 0; --b) {
+      const unsigned int c = hist[8 * lane + b];
+      if (acc + c >= (unsigned int)want) { bin = 8 * lane + b; ov = (int)acc; break; }
+      acc += c;
+    }
+  }
+  over = __shfl_sync(0xffffffffu, ov, src);
+  return __shfl_sync(0xffffffffu, bin, src);
+}
+
+// The k-th largest key of keys[0 .. n) and the k-th smallest, by two 8-bit histogram levels; beyond_t / beyond_b: how
+// many keys lie strictly beyond them.  The smallest is the largest of the complemented keys: its first-level histogram
+// is the mirror image of the other one, its second level is counted in the same pass.  One warp, hist = 512 words.
+__device__ __forceinline__ void warp_select(const unsigned short* keys, int n, int k, unsigned int* hist, int lane,
+                                            unsigned int& key_t, int& beyond_t, unsigned int& key_b, int& beyond_b) {
+  unsigned int* hist_b = hist + 256;
+  for (int i = lane; i < 256; i += 32) hist[i] = 0u;
+  __syncwarp();
+  for (int i = lane; i < n; i += 32) atomicAdd(&hist[keys[i] >> 8], 1u);
+  __syncwarp();
+  for (int i = lane; i < 256; i += 32) hist_b[i] = hist[255 - i];
+  __syncwarp();
+  int over_t, over_b;
+  const unsigned int pre_t = (unsigned int)pick_bin(hist, k, lane, over_t);
+  const unsigned int pre_b = (unsigned int)pick_bin(hist_b, k, lane, over_b);
+  __syncwarp();
+  for (int i = lane; i < 512; i += 32) hist[i] = 0u;
+  __syncwarp();
+  for (int i = lane; i < n; i += 32) {
+    const unsigned int key = keys[i], kf = key ^ 0xFFFFu;
+    if ((key >> 8) == pre_t) atomicAdd(&hist[key & 0xFFu], 1u);
+    if ((kf >> 8) == pre_b) atomicAdd(&hist_b[kf & 0xFFu], 1u);
+  }
+  __syncwarp();
+  int over2_t, over2_b;
+  const unsigned int lo_t = (unsigned int)pick_bin(hist, k - over_t, lane, over2_t);
+  const unsigned int lo_b = (unsigned int)pick_bin(hist_b, k - over_b, lane, over2_b);
+  __syncwarp();
+  key_t = (pre_t << 8) | lo_t;
+  key_b = ((pre_b << 8) | lo_b) ^ 0xFFFFu;
+  beyond_t = over_t + over2_t;
+  beyond_b = over_b + over2_b;
 }
 
 template <int BITS>
@@ -84,15 +98,15 @@ __global__ void __launch_bounds__(kSelChannels * 32) kcvt_select_kernel(KcvtArgs
   const int n_c = sd.n_c, k = sd.csr_k / 2;
   const int cg = blockIdx.x, bhl = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int ch = cg * kSelChannels + warp;
-  // shared memory: keys [8][n_c] u16 | outlier bitmask [8][n_c / 32] | histograms [8][256] | stage of a chunk
+  // shared memory: keys [8][n_c] u16 | outlier bitmask [8][n_c / 32] | histograms [8][512] | stage of a chunk
   unsigned short* keys_all = reinterpret_cast<unsigned short*>(sm_raw);
   unsigned int* mask_all = reinterpret_cast<unsigned int*>(sm_raw + (size_t)kSelChannels * n_c * 2);
   unsigned int* hist_all = mask_all + kSelChannels * (n_c / 32);
-  float* stage_r = reinterpret_cast<float*>(hist_all + kSelChannels * 256);       // [kSelChunk][8]
+  float* stage_r = reinterpret_cast<float*>(hist_all + kSelChannels * 512);       // [kSelChunk][8]
   unsigned char* stage_c = reinterpret_cast<unsigned char*>(stage_r + kSelChunk * kSelChannels);   // [kSelChunk][8]
   unsigned short* keys = keys_all + (size_t)warp * n_c;
   unsigned int* omask = mask_all + warp * (n_c / 32);
-  unsigned int* hist = hist_all + warp * 256;
+  unsigned int* hist = hist_all + warp * 512;
 
   const __half* X = p.K + (size_t)bhl * n_c * kHeadDim;
   for (int tok = tid; tok < n_c; tok += blockDim.x) {          // 16 bytes (this CTA's 8 channels) of every token row
@@ -110,11 +124,10 @@ __global__ void __launch_bounds__(kSelChannels * 32) kcvt_select_kernel(KcvtArgs
   unsigned int key_t = 0xFFFFu, key_b = 0u;
   int need_t = 0, need_b = 0;                   // entries equal to the threshold key that still leave, lowest tokens first
   if (k > 0) {
-    int beyond;
-    key_t = warp_select(keys, n_c, k, 0u, hist, lane, beyond);
-    need_t = k - beyond;
-    key_b = warp_select(keys, n_c, k, 0xFFFFu, hist, lane, beyond);
-    need_b = k - beyond;
+    int beyond_t, beyond_b;
+    warp_select(keys, n_c, k, hist, lane, key_t, beyond_t, key_b, beyond_b);
+    need_t = k - beyond_t;
+    need_b = k - beyond_b;
   }
   const bool same = key_t == key_b;             // the thresholds meet only when all kept entries would be equal
   unsigned int kmin = 0xFFFFu, kmax = 0u;
@@ -125,13 +138,15 @@ __global__ void __launch_bounds__(kSelChannels * 32) kcvt_select_kernel(KcvtArgs
     bool out = false;
     if (k > 0) {
       const bool is_t = key == key_t, is_b = key == key_b;
-      const unsigned int bt = __ballot_sync(0xffffffffu, is_t), bb = __ballot_sync(0xffffffffu, is_b);
-      const unsigned int below = (1u << lane) - 1u;
-      const int rt = eq_t + __popc(bt & below), rb = eq_b + __popc(bb & below);
-      const bool top = key > key_t || (is_t && rt < need_t);
-      const bool bot = key < key_b || (is_b && (same ? (rt >= need_t && rt < need_t + need_b) : rb < need_b));
-      out = top || bot;
-      eq_t += __popc(bt); eq_b += __popc(bb);
+      out = key > key_t || key < key_b;
+      if (__any_sync(0xffffffffu, is_t || is_b)) {        // an entry on a threshold: ties go to the lower token
+        const unsigned int bt = __ballot_sync(0xffffffffu, is_t), bb = __ballot_sync(0xffffffffu, is_b);
+        const unsigned int below = (1u << lane) - 1u;
+        const int rt = eq_t + __popc(bt & below), rb = eq_b + __popc(bb & below);
+        out = out || (is_t && rt < need_t) ||
+              (is_b && (same ? (rt >= need_t && rt < need_t + need_b) : rb < need_b));
+        eq_t += __popc(bt); eq_b += __popc(bb);
+      }
     }
     const unsigned int bo = __ballot_sync(0xffffffffu, out);
     if (lane == 0) omask[base >> 5] = bo;
@@ -290,7 +305,7 @@ __global__ void __launch_bounds__(128) kcvt_pack_kernel(KcvtArgs p) {
 }
 
 size_t kcvt_select_smem(int n_c) {
-  return (size_t)kSelChannels * n_c * 2 + (size_t)kSelChannels * (n_c / 32) * 4 + kSelChannels * 256 * 4 +
+  return (size_t)kSelChannels * n_c * 2 + (size_t)kSelChannels * (n_c / 32) * 4 + kSelChannels * 512 * 4 +
          (size_t)kSelChunk * kSelChannels * 5;
 }
 size_t kcvt_list_smem(int nblk) { return ((size_t)nblk * kHeadDim + 2 * (size_t)nblk + 1) * 4; }
