@@ -37,10 +37,11 @@ from paper_2403_05527_b200 import synth  # noqa: E402
 METRIC = "compressed-KV decode attn tokens/s"
 UNIT = "tokens/s"
 # dram__bytes_read + dram__bytes_write of one gear_decode_kernel launch per algorithmic byte, by configuration, from ncu
-# captures of the kernel on one layer cache (C2: 137.65 MB of DRAM traffic for 134.26 MB; C4: 125.65 MB for 118.48 MB;
-# C3 4-bit: 1071.46 MB for 1077.91 MB; C3 2-bit: 735.96 MB for 738.39 MB; C6: 193.66 MB for 191.34 MB -- a ratio below
-# one: the segment flushed just before the captured launch was still in L2); traffic grows in proportion to the cache
-DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {2: 1.0253, 4: 1.0605, 3: 0.9940, 32: 0.9967, 6: 1.0121}
+# captures (one pass, the two counters) of the kernel as it stands on one layer cache: C2 137.40 MB of DRAM traffic for
+# 134.26 MB; C4 121.77 MB for 118.48 MB; C3 4-bit 1072.05 MB for 1077.91 MB; C3 2-bit 736.20 MB for 738.39 MB; C6
+# 193.67 MB for 191.34 MB (a ratio below one: the segment flushed just before the captured launch was still in L2);
+# traffic grows in proportion to the cache
+DECODE_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {2: 1.0234, 4: 1.0277, 3: 0.9946, 32: 0.9970, 6: 1.0122}
 EXTRA_CONFIGS = (3, 32, 4, 6)
 
 
